@@ -1,0 +1,793 @@
+// C ABI of the verification path (declared in include/ssd.h): argument checks, workspace
+// carving and the launch sequences.  All arithmetic runs in the kernels of gemm.cuh,
+// rowops.cuh, attention.cuh and tail.cuh; there is no CPU or library fallback.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "../../include/ssd.h"
+#include "attention.cuh"
+#include "common.cuh"
+#include "gemm.cuh"
+#include "rowops.cuh"
+#include "tail.cuh"
+
+using namespace ssd;
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+int g_num_sms = 0;
+bool g_attr_done = false;
+std::mutex g_mu;
+
+// ---- optional per-launch timing of the weight-streaming GEMM ----
+bool g_prof = false;
+std::vector<cudaEvent_t> g_prof_events;  // pairs
+size_t g_prof_used = 0;
+
+#define CUDA_OK(expr)                        \
+    do {                                     \
+        cudaError_t e__ = (expr);            \
+        if (e__ != cudaSuccess) return SSD_E_CUDA; \
+    } while (0)
+
+#define LAUNCH(kernel, grid, block, smem, stream, ...)                 \
+    do {                                                                \
+        kernel<<<grid, block, smem, stream>>>(__VA_ARGS__);             \
+        g_launches.fetch_add(1, std::memory_order_relaxed);             \
+        if (cudaPeekAtLastError() != cudaSuccess) return SSD_E_CUDA;    \
+    } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// bf16 matrix [rows, cols] row-major -> tensor map with a (box_rows x 64) box, 128-byte swizzle
+int make_map(CUtensorMap *map, const void *ptr, int rows, int cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return SSD_E_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? SSD_OK : SSD_E_CUDA;
+}
+
+template <int NT>
+constexpr int gemm_stage_bytes() { return kWTileBytes + 2 * NT * 8 * kTileK * 2; }
+constexpr int kSmemBudget = 227 * 1024;
+
+template <int NT>
+int gemm_stages() {
+    int s = (kSmemBudget - 1024 - 512) / gemm_stage_bytes<NT>();
+    return s > 12 ? 12 : s;
+}
+template <int NT>
+size_t gemm_smem() { return 1024 + (size_t)gemm_stages<NT>() * gemm_stage_bytes<NT>() + 16 * gemm_stages<NT>() + 16; }
+
+template <typename K>
+int set_smem(K kernel, size_t bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess ? 0 : -1;
+}
+
+template <typename T, int MR>
+size_t attn_smem(int Dh) {
+    return (size_t)MR * (Dh + kAttnTile + 3) * 4 + 2 * (size_t)kAttnTile * (Dh + 16 / sizeof(T)) * sizeof(T);
+}
+
+int init_device_once() {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (g_attr_done) return SSD_OK;
+    int dev = 0;
+    CUDA_OK(cudaGetDevice(&dev));
+    CUDA_OK(cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev));
+    int rc = 0;
+    rc |= set_smem(gemm_bf16_kernel<1>, gemm_smem<1>());
+    rc |= set_smem(gemm_bf16_kernel<2>, gemm_smem<2>());
+    rc |= set_smem(gemm_bf16_kernel<3>, gemm_smem<3>());
+    rc |= set_smem(gemm_bf16_kernel<4>, gemm_smem<4>());
+    rc |= set_smem(gemm_bf16_kernel<5>, gemm_smem<5>());
+    rc |= set_smem(gemm_bf16_kernel<6>, gemm_smem<6>());
+    rc |= set_smem(gemm_bf16_kernel<7>, gemm_smem<7>());
+    rc |= set_smem(gemm_bf16_kernel<8>, gemm_smem<8>());
+    rc |= set_smem(attn_partial_kernel<float, 8>, attn_smem<float, 8>(128));
+    rc |= set_smem(attn_partial_kernel<float, 16>, attn_smem<float, 16>(128));
+    rc |= set_smem(attn_partial_kernel<float, 32>, attn_smem<float, 32>(128));
+    rc |= set_smem(attn_partial_kernel<__nv_bfloat16, 8>, attn_smem<__nv_bfloat16, 8>(128));
+    rc |= set_smem(attn_partial_kernel<__nv_bfloat16, 16>, attn_smem<__nv_bfloat16, 16>(128));
+    rc |= set_smem(attn_partial_kernel<__nv_bfloat16, 32>, attn_smem<__nv_bfloat16, 32>(128));
+    if (rc) return SSD_E_CUDA;
+    g_attr_done = true;
+    return SSD_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+struct ssd_model {
+    ssd_arch a;
+    std::vector<const void *> w;  // 2 + 12 L + 3 tensors
+    std::vector<CUtensorMap> tm;  // bf16 models: per layer {qkv, o, in, out}, then lm head
+    int d_in;
+};
+
+struct ssd_kv {
+    ssd_arch a;
+    int B, S;
+    uint8_t *buf;
+    int32_t *status, *len, *keep;
+    uint8_t *cache;
+    size_t layer_bytes, esize;
+    int len_ub;   // host-side upper bound of the committed lengths
+    int last_rows;  // rows the last forward left uncommitted (upper bound bookkeeping)
+};
+
+namespace {
+
+enum { T_TOK = 0, T_POS = 1, T_L0 = 2, PER_LAYER = 12 };
+enum { L_LN1G, L_LN1B, L_WQKV, L_BQKV, L_WO, L_BO, L_LN2G, L_LN2B, L_WIN, L_BIN, L_WOUT, L_BOUT };
+
+const void *lw(const ssd_model *m, int layer, int which) { return m->w[T_L0 + PER_LAYER * layer + which]; }
+const void *fw(const ssd_model *m, int which) { return m->w[T_L0 + PER_LAYER * m->a.n_layers + which]; }
+const void *lm_matrix(const ssd_model *m) { return m->a.tie_lm_head ? m->w[T_TOK] : fw(m, 2); }
+
+int build_maps(ssd_model *m) {
+    if (m->a.dtype != 1) return SSD_OK;
+    const ssd_arch &a = m->a;
+    m->tm.resize((size_t)4 * a.n_layers + 1);
+    for (int l = 0; l < a.n_layers; ++l) {
+        int rc = 0;
+        rc |= make_map(&m->tm[4 * l + 0], lw(m, l, L_WQKV), 3 * a.d_model, a.d_model, kTileN);
+        rc |= make_map(&m->tm[4 * l + 1], lw(m, l, L_WO), a.d_model, a.d_model, kTileN);
+        rc |= make_map(&m->tm[4 * l + 2], lw(m, l, L_WIN), m->d_in, a.d_model, kTileN);
+        rc |= make_map(&m->tm[4 * l + 3], lw(m, l, L_WOUT), a.d_model, a.d_ff, kTileN);
+        if (rc) return SSD_E_CUDA;
+    }
+    return make_map(&m->tm[(size_t)4 * a.n_layers], lm_matrix(m), a.vocab, a.d_model, kTileN);
+}
+
+int check_arch(const ssd_arch &a) {
+    if (a.n_layers <= 0 || a.d_model <= 0 || a.n_heads <= 0 || a.head_dim <= 0 || a.d_ff <= 0 || a.vocab <= 0)
+        return SSD_E_ARG;
+    if (a.n_heads * a.head_dim != a.d_model) return SSD_E_SHAPE;
+    if (a.head_dim > 128 || a.head_dim % 8) return SSD_E_SHAPE;
+    if (a.norm < 0 || a.norm > 1 || a.act < 0 || a.act > 1 || a.pos < 0 || a.pos > 1 || a.dtype < 0 || a.dtype > 1)
+        return SSD_E_ARG;
+    if (a.pos == 1 && (a.rotary_dim <= 0 || a.rotary_dim % 2 || a.rotary_dim > a.head_dim)) return SSD_E_SHAPE;
+    if (a.pos == 0 && a.max_pos <= 0) return SSD_E_ARG;
+    if (a.dtype == 1) {
+        if (a.d_model < 128 || a.d_model % 8 || a.d_ff < 128 || a.d_ff % 8 || a.vocab < 128) return SSD_E_SHAPE;
+    }
+    return SSD_OK;
+}
+
+// ---- workspace ----
+struct Workspace {
+    RowInfo ri;
+    int32_t *n_rows_tmp;
+    float *x, *qkv, *qrot, *t_in, *logits;
+    RowStat *stats;
+    Operand xn1, xn2, ao, act;
+    float *part_m, *part_l, *part_o;
+    int max_split;
+    size_t bytes;
+};
+
+constexpr int kMaxSplit = 32;
+
+// Carve (or just size, base == nullptr) the workspace for B sequences x M rows.
+Workspace carve(const ssd_model *m, int B, int M, uint8_t *base) {
+    const ssd_arch &a = m->a;
+    const int R = B * M, Rp = (R + 7) / 8 * 8, d = a.d_model, F = a.d_ff;
+    size_t off = 0;
+    auto take = [&](size_t bytes) -> uint8_t * {
+        uint8_t *p = base ? base + off : nullptr;
+        off += align_up(bytes, 1024);
+        return p;
+    };
+    Workspace w;
+    memset(&w, 0, sizeof(w));
+    const int half = a.pos == 1 ? a.rotary_dim / 2 : 0;
+    w.ri.seq = (int32_t *)take(sizeof(int32_t) * R);
+    w.ri.pos = (int32_t *)take(sizeof(int32_t) * R);
+    w.ri.valid = (int32_t *)take(sizeof(int32_t) * R);
+    w.ri.n_eff = (int32_t *)take(sizeof(int32_t) * B);
+    w.ri.rope_cos = (float *)take(sizeof(float) * (size_t)R * (half ? half : 1));
+    w.ri.rope_sin = (float *)take(sizeof(float) * (size_t)R * (half ? half : 1));
+    w.n_rows_tmp = (int32_t *)take(sizeof(int32_t) * B);
+    w.x = (float *)take(sizeof(float) * (size_t)R * d);
+    w.qkv = (float *)take(sizeof(float) * (size_t)R * 3 * d);
+    w.qrot = (float *)take(sizeof(float) * (size_t)R * d);
+    w.t_in = (float *)take(sizeof(float) * (size_t)R * m->d_in);
+    w.logits = (float *)take(sizeof(float) * (size_t)R * a.vocab);
+    w.stats = (RowStat *)take(sizeof(RowStat) * R);
+    auto operand = [&](int ld, bool needed) {
+        Operand o;
+        o.f32 = nullptr; o.hi = nullptr; o.lo = nullptr; o.ld = ld;
+        if (!needed) return o;
+        if (a.dtype == 0) {
+            o.f32 = (float *)take(sizeof(float) * (size_t)Rp * ld);
+        } else {
+            o.hi = (__nv_bfloat16 *)take(2 * (size_t)Rp * ld);
+            o.lo = (__nv_bfloat16 *)take(2 * (size_t)Rp * ld);
+        }
+        return o;
+    };
+    w.xn1 = operand(d, true);
+    w.xn2 = operand(d, a.parallel_residual != 0);
+    w.ao = operand(d, true);
+    w.act = operand(F, true);
+    w.max_split = kMaxSplit;
+    size_t slots = (size_t)R * a.n_heads * kMaxSplit;
+    w.part_m = (float *)take(sizeof(float) * slots);
+    w.part_l = (float *)take(sizeof(float) * slots);
+    w.part_o = (float *)take(sizeof(float) * slots * a.head_dim);
+    w.bytes = off;
+    return w;
+}
+
+struct GemmCall {
+    const ssd_model *m;
+    cudaStream_t st;
+    int R, Rp;
+};
+
+template <int NT>
+int launch_gemm_nt(cudaStream_t st, const CUtensorMap &tw, const CUtensorMap &th, const CUtensorMap &tl, GemmArgs g,
+                   int grid) {
+    g.stages = gemm_stages<NT>();
+    LAUNCH(gemm_bf16_kernel<NT>, grid, kGemmThreads, gemm_smem<NT>(), st, tw, th, tl, g);
+    return SSD_OK;
+}
+
+// out[R, ldo] += X[R, Kd] * W[N, Kd]^T
+int gemm(const GemmCall &c, const void *W, const CUtensorMap *tw, const Operand &X, int Kd, int N, float *out, int ldo,
+         int32_t *status) {
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (g_prof) {
+        if (g_prof_used + 2 > g_prof_events.size()) {
+            for (int i = 0; i < 2; ++i) {
+                cudaEvent_t e;
+                CUDA_OK(cudaEventCreate(&e));
+                g_prof_events.push_back(e);
+            }
+        }
+        e0 = g_prof_events[g_prof_used];
+        e1 = g_prof_events[g_prof_used + 1];
+        g_prof_used += 2;
+        CUDA_OK(cudaEventRecord(e0, c.st));
+    }
+    int rc = SSD_OK;
+    if (c.m->a.dtype == 0) {
+        const int warps = 8;
+        LAUNCH(gemm_f32_kernel, ceil_div(N, warps), warps * 32, 0, c.st, (const float *)W, X.f32, X.ld, out, ldo, N,
+               Kd, c.R);
+    } else {
+        CUtensorMap th, tl;
+        if (make_map(&th, X.hi, c.Rp, Kd, c.Rp) || make_map(&tl, X.lo, c.Rp, Kd, c.Rp)) return SSD_E_CUDA;
+        GemmArgs g;
+        g.out = out; g.ldo = ldo; g.N = N; g.Kd = Kd; g.R = c.R;
+        g.n_tiles = ceil_div(N, kTileN);
+        g.kchunks = ceil_div(Kd, kTileK);
+        g.stages = 0;
+        g.status = status;
+        long long total = (long long)g.n_tiles * g.kchunks;
+        int grid = (int)(total < g_num_sms ? total : g_num_sms);
+        switch (c.Rp / 8) {
+            case 1: rc = launch_gemm_nt<1>(c.st, *tw, th, tl, g, grid); break;
+            case 2: rc = launch_gemm_nt<2>(c.st, *tw, th, tl, g, grid); break;
+            case 3: rc = launch_gemm_nt<3>(c.st, *tw, th, tl, g, grid); break;
+            case 4: rc = launch_gemm_nt<4>(c.st, *tw, th, tl, g, grid); break;
+            case 5: rc = launch_gemm_nt<5>(c.st, *tw, th, tl, g, grid); break;
+            case 6: rc = launch_gemm_nt<6>(c.st, *tw, th, tl, g, grid); break;
+            case 7: rc = launch_gemm_nt<7>(c.st, *tw, th, tl, g, grid); break;
+            case 8: rc = launch_gemm_nt<8>(c.st, *tw, th, tl, g, grid); break;
+            default: return SSD_E_CAPACITY;
+        }
+    }
+    if (rc) return rc;
+    if (e1) CUDA_OK(cudaEventRecord(e1, c.st));
+    return SSD_OK;
+}
+
+// Split of the position axis for a context of up to `ctx` positions.
+void plan_split(int B, int H, int ctx, int *chunk, int *n_split) {
+    if (ctx < 1) ctx = 1;
+    int want = ceil_div(2 * (g_num_sms > 0 ? g_num_sms : 148), B * H);
+    int max_by_len = ceil_div(ctx, kAttnTile);
+    int ns = want < 1 ? 1 : want;
+    if (ns > max_by_len) ns = max_by_len;
+    if (ns > kMaxSplit) ns = kMaxSplit;
+    int ch = ceil_div(ceil_div(ctx, ns), kAttnTile) * kAttnTile;
+    *chunk = ch;
+    *n_split = ceil_div(ctx, ch);
+}
+
+template <typename T>
+int launch_attn(cudaStream_t st, const AttnArgs &a, int B, int M) {
+    dim3 grid(a.n_split, B * a.H);
+    auto k8 = attn_partial_kernel<T, 8>;
+    auto k16 = attn_partial_kernel<T, 16>;
+    auto k32 = attn_partial_kernel<T, 32>;
+    if (M <= 8) {
+        LAUNCH(k8, grid, kAttnThreads, (attn_smem<T, 8>(a.Dh)), st, a);
+    } else if (M <= 16) {
+        LAUNCH(k16, grid, kAttnThreads, (attn_smem<T, 16>(a.Dh)), st, a);
+    } else {
+        LAUNCH(k32, grid, kAttnThreads, (attn_smem<T, 32>(a.Dh)), st, a);
+    }
+    return SSD_OK;
+}
+
+int run_setup(const ssd_model *m, ssd_kv *kv, int M, const int32_t *n_rows, const Workspace &w, cudaStream_t st) {
+    SetupArgs s;
+    s.B = kv->B; s.M = M; s.n_rows = n_rows; s.len = kv->len; s.s_max = kv->S;
+    s.pos_limit = m->a.pos == 0 ? m->a.max_pos : 0;
+    s.rotary_dim = m->a.pos == 1 ? m->a.rotary_dim : 0;
+    s.rotary_base = m->a.rotary_base;
+    s.ri = w.ri;
+    s.status = kv->status;
+    LAUNCH(setup_rows_kernel, kv->B * M, 64, 0, st, s);
+    return SSD_OK;
+}
+
+int run_attention(const ssd_model *m, ssd_kv *kv, int layer, const float *q, int M, const Workspace &w,
+                  const CombineArgs &comb_in, cudaStream_t st) {
+    const ssd_arch &a = m->a;
+    AttnArgs at;
+    at.q = q;
+    at.cache = kv->cache + (size_t)layer * kv->layer_bytes;
+    at.len = kv->len;
+    at.M = M; at.H = a.n_heads; at.Dh = a.head_dim; at.S = kv->S; at.d = a.d_model;
+    int ctx = kv->len_ub + M;
+    if (ctx > kv->S) ctx = kv->S;
+    plan_split(kv->B, a.n_heads, ctx, &at.chunk, &at.n_split);
+    at.scale = 1.0f / sqrtf((float)a.head_dim);
+    at.ri = w.ri;
+    at.part_m = w.part_m; at.part_l = w.part_l; at.part_o = w.part_o;
+    int rc = a.dtype ? launch_attn<__nv_bfloat16>(st, at, kv->B, M) : launch_attn<float>(st, at, kv->B, M);
+    if (rc) return rc;
+    CombineArgs cb = comb_in;
+    cb.part_m = w.part_m; cb.part_l = w.part_l; cb.part_o = w.part_o;
+    cb.H = a.n_heads; cb.Dh = a.head_dim; cb.n_split = at.n_split; cb.d = a.d_model;
+    LAUNCH(attn_combine_kernel, dim3(a.n_heads, kv->B * M), 128, 0, st, cb);
+    return SSD_OK;
+}
+
+// One decoder forward over B x M rows against the cache.  Appends (does not commit) the rows'
+// keys/values; leaves logits in w.logits when want_logits.
+int forward(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int M, const int32_t *n_rows,
+            bool want_logits, const Workspace &w, cudaStream_t st) {
+    const ssd_arch &a = m->a;
+    const int B = kv->B, R = B * M, d = a.d_model, F = a.d_ff;
+    GemmCall gc{m, st, R, (R + 7) / 8 * 8};
+    int rc = run_setup(m, kv, M, n_rows, w, st);
+    if (rc) return rc;
+    if (a.dtype) {
+        LAUNCH(embed_kernel<__nv_bfloat16>, R, 256, 0, st, (const __nv_bfloat16 *)m->w[T_TOK],
+               (const __nv_bfloat16 *)m->w[T_POS], tokens, tok_stride, M, a.vocab, d, w.ri, w.x);
+    } else {
+        LAUNCH(embed_kernel<float>, R, 256, 0, st, (const float *)m->w[T_TOK], (const float *)m->w[T_POS], tokens,
+               tok_stride, M, a.vocab, d, w.ri, w.x);
+    }
+    auto norm_args = [&](const float *g1, const float *b1, Operand o1) {
+        NormArgs n;
+        memset(&n, 0, sizeof(n));
+        n.x = w.x; n.d = d; n.kind = a.norm; n.eps = a.norm_eps;
+        n.n_norms = 1; n.g[0] = g1; n.b[0] = b1; n.out[0] = o1;
+        return n;
+    };
+    for (int l = 0; l < a.n_layers; ++l) {
+        const CUtensorMap *tm = a.dtype ? &m->tm[4 * l] : nullptr;
+        const float *b_qkv = (const float *)lw(m, l, L_BQKV), *b_o = (const float *)lw(m, l, L_BO);
+        const float *b_in = (const float *)lw(m, l, L_BIN), *b_out = (const float *)lw(m, l, L_BOUT);
+        // ---- norm(s) + pre-load of the GEMM outputs ----
+        NormArgs n1 = norm_args((const float *)lw(m, l, L_LN1G), (const float *)lw(m, l, L_LN1B), w.xn1);
+        n1.init[n1.n_init++] = InitJob{w.qkv, b_qkv, 3 * d, 3 * d};
+        if (a.parallel_residual) {
+            n1.n_norms = 2;
+            n1.g[1] = (const float *)lw(m, l, L_LN2G);
+            n1.b[1] = (const float *)lw(m, l, L_LN2B);
+            n1.out[1] = w.xn2;
+            n1.init[n1.n_init++] = InitJob{w.t_in, b_in, m->d_in, m->d_in};
+        }
+        LAUNCH(norm_kernel, R, 256, 0, st, n1);
+        if ((rc = gemm(gc, lw(m, l, L_WQKV), tm ? tm + 0 : nullptr, w.xn1, d, 3 * d, w.qkv, 3 * d, kv->status))) return rc;
+        if (a.parallel_residual)
+            if ((rc = gemm(gc, lw(m, l, L_WIN), tm ? tm + 2 : nullptr, w.xn2, d, m->d_in, w.t_in, m->d_in, kv->status)))
+                return rc;
+        // ---- rotary + append, attention ----
+        RopeArgs ra;
+        ra.qkv = w.qkv; ra.q_out = w.qrot;
+        ra.cache = kv->cache + (size_t)l * kv->layer_bytes;
+        ra.d = d; ra.H = a.n_heads; ra.Dh = a.head_dim; ra.S = kv->S;
+        ra.rotary_dim = a.pos == 1 ? a.rotary_dim : 0;
+        ra.ri = w.ri;
+        if (a.dtype) {
+            LAUNCH(rope_append_kernel<__nv_bfloat16>, R, 256, 0, st, ra);
+        } else {
+            LAUNCH(rope_append_kernel<float>, R, 256, 0, st, ra);
+        }
+        CombineArgs cb;
+        memset(&cb, 0, sizeof(cb));
+        cb.out = w.ao;
+        cb.x = w.x;
+        cb.bias.b0 = b_o;
+        cb.bias.b1 = a.parallel_residual ? b_out : nullptr;
+        if ((rc = run_attention(m, kv, l, w.qrot, M, w, cb, st))) return rc;
+        BiasJob no_bias{nullptr, nullptr};
+        if (a.parallel_residual) {
+            LAUNCH(act_kernel, dim3(ceil_div(F, 256), R), 256, 0, st, w.t_in, m->d_in, F, a.act == 1, w.act, w.x, d,
+                   no_bias);
+            if ((rc = gemm(gc, lw(m, l, L_WO), tm ? tm + 1 : nullptr, w.ao, d, d, w.x, d, kv->status))) return rc;
+            if ((rc = gemm(gc, lw(m, l, L_WOUT), tm ? tm + 3 : nullptr, w.act, F, d, w.x, d, kv->status))) return rc;
+        } else {
+            if ((rc = gemm(gc, lw(m, l, L_WO), tm ? tm + 1 : nullptr, w.ao, d, d, w.x, d, kv->status))) return rc;
+            NormArgs n2 = norm_args((const float *)lw(m, l, L_LN2G), (const float *)lw(m, l, L_LN2B), w.xn1);
+            n2.init[n2.n_init++] = InitJob{w.t_in, b_in, m->d_in, m->d_in};
+            LAUNCH(norm_kernel, R, 256, 0, st, n2);
+            if ((rc = gemm(gc, lw(m, l, L_WIN), tm ? tm + 2 : nullptr, w.xn1, d, m->d_in, w.t_in, m->d_in, kv->status)))
+                return rc;
+            BiasJob bj{b_out, nullptr};
+            LAUNCH(act_kernel, dim3(ceil_div(F, 256), R), 256, 0, st, w.t_in, m->d_in, F, a.act == 1, w.act, w.x, d, bj);
+            if ((rc = gemm(gc, lw(m, l, L_WOUT), tm ? tm + 3 : nullptr, w.act, F, d, w.x, d, kv->status))) return rc;
+        }
+    }
+    if (want_logits) {
+        NormArgs nf = norm_args((const float *)fw(m, 0), (const float *)fw(m, 1), w.xn1);
+        nf.init[nf.n_init++] = InitJob{w.logits, nullptr, a.vocab, a.vocab};
+        LAUNCH(norm_kernel, R, 256, 0, st, nf);
+        if ((rc = gemm(gc, lm_matrix(m), a.dtype ? &m->tm[(size_t)4 * a.n_layers] : nullptr, w.xn1, d, a.vocab, w.logits,
+                       a.vocab, kv->status)))
+            return rc;
+    }
+    kv->last_rows = M;
+    return SSD_OK;
+}
+
+int check_ws(const ssd_model *m, int B, int M, void *ws, size_t ws_bytes, Workspace *out) {
+    if (!ws) return SSD_E_ARG;
+    if (B * M > kMaxRows || M > kMaxRowsPerSeq || M < 1) return SSD_E_CAPACITY;
+    if (((uintptr_t)ws & 255) != 0) return SSD_E_ARG;
+    *out = carve(m, B, M, (uint8_t *)ws);
+    if (out->bytes > ws_bytes) return SSD_E_CAPACITY;
+    return SSD_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+extern "C" {
+
+int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n_tensors, ssd_model **out) {
+    if (!arch || !dev_weights || !out) return SSD_E_ARG;
+    int rc = check_arch(*arch);
+    if (rc) return rc;
+    if (n_tensors != 2 + PER_LAYER * arch->n_layers + 3) return SSD_E_ARG;
+    // required tensors
+    auto need = [&](int i) { return dev_weights[i] != nullptr; };
+    if (!need(T_TOK) || (arch->pos == 0 && !need(T_POS))) return SSD_E_ARG;
+    for (int l = 0; l < arch->n_layers; ++l) {
+        const int b = T_L0 + PER_LAYER * l;
+        if (!need(b + L_LN1G) || !need(b + L_WQKV) || !need(b + L_WO) || !need(b + L_LN2G) || !need(b + L_WIN) ||
+            !need(b + L_WOUT))
+            return SSD_E_ARG;
+    }
+    const int fb = T_L0 + PER_LAYER * arch->n_layers;
+    if (!need(fb) || (!arch->tie_lm_head && !need(fb + 2))) return SSD_E_ARG;
+    if ((rc = init_device_once())) return rc;
+    ssd_model *m = new (std::nothrow) ssd_model();
+    if (!m) return SSD_E_ARG;
+    m->a = *arch;
+    m->w.assign(dev_weights, dev_weights + n_tensors);
+    m->d_in = arch->act == 1 ? 2 * arch->d_ff : arch->d_ff;
+    if ((rc = build_maps(m))) {
+        delete m;
+        return rc;
+    }
+    *out = m;
+    return SSD_OK;
+}
+
+int ssd_model_share_prefix(const ssd_model *target, int n_layers, ssd_model **draft_out) {
+    if (!target || !draft_out || n_layers < 1 || n_layers > target->a.n_layers) return SSD_E_ARG;
+    ssd_model *m = new (std::nothrow) ssd_model();
+    if (!m) return SSD_E_ARG;
+    m->a = target->a;
+    m->a.n_layers = n_layers;
+    m->d_in = target->d_in;
+    m->w.assign(target->w.begin(), target->w.begin() + T_L0 + PER_LAYER * n_layers);
+    m->w.insert(m->w.end(), target->w.end() - 3, target->w.end());
+    if (!target->tm.empty()) {
+        m->tm.assign(target->tm.begin(), target->tm.begin() + 4 * n_layers);
+        m->tm.push_back(target->tm.back());
+    }
+    *draft_out = m;
+    return SSD_OK;
+}
+
+void ssd_model_destroy(ssd_model *m) { delete m; }
+
+static size_t kv_header_bytes(int batch) { return align_up(sizeof(int32_t) * (kHeaderInts + 2 * (size_t)batch), 1024); }
+
+size_t ssd_kv_bytes(const ssd_model *m, int batch, int max_len) {
+    if (!m || batch < 1 || max_len < 1) return 0;
+    size_t es = m->a.dtype ? 2 : 4;
+    return kv_header_bytes(batch) + (size_t)m->a.n_layers * batch * 2 * m->a.d_model * max_len * es;
+}
+
+size_t ssd_workspace_bytes(const ssd_model *m, int batch, int rows_per_seq, int max_len) {
+    (void)max_len;
+    if (!m || batch < 1 || rows_per_seq < 1 || batch * rows_per_seq > kMaxRows || rows_per_seq > kMaxRowsPerSeq) return 0;
+    return carve(m, batch, rows_per_seq, nullptr).bytes;
+}
+
+int kv_init(const ssd_model *m, int batch, int max_len, void *dev_buf, size_t bytes, void *stream, ssd_kv **out) {
+    if (!m || !dev_buf || !out || batch < 1 || max_len < 1) return SSD_E_ARG;
+    if (batch > kMaxRows) return SSD_E_CAPACITY;
+    if (((uintptr_t)dev_buf & 255) != 0) return SSD_E_ARG;
+    if (bytes < ssd_kv_bytes(m, batch, max_len)) return SSD_E_CAPACITY;
+    ssd_kv *kv = new (std::nothrow) ssd_kv();
+    if (!kv) return SSD_E_ARG;
+    kv->a = m->a;
+    kv->B = batch;
+    kv->S = max_len;
+    kv->buf = (uint8_t *)dev_buf;
+    kv->status = (int32_t *)dev_buf;
+    kv->len = kv->status + kHeaderInts;
+    kv->keep = kv->len + batch;
+    kv->cache = kv->buf + kv_header_bytes(batch);
+    kv->esize = m->a.dtype ? 2 : 4;
+    kv->layer_bytes = (size_t)batch * 2 * m->a.d_model * max_len * kv->esize;
+    kv->len_ub = 0;
+    kv->last_rows = 0;
+    if (cudaMemsetAsync(dev_buf, 0, kv_header_bytes(batch), (cudaStream_t)stream) != cudaSuccess) {
+        delete kv;
+        return SSD_E_CUDA;
+    }
+    *out = kv;
+    return SSD_OK;
+}
+
+void kv_destroy(ssd_kv *kv) { delete kv; }
+
+static bool same_cache_shape(const ssd_model *m, const ssd_kv *kv) {
+    return m->a.n_layers == kv->a.n_layers && m->a.d_model == kv->a.d_model && m->a.n_heads == kv->a.n_heads &&
+           m->a.dtype == kv->a.dtype;
+}
+
+int kv_prefill(ssd_model *m, ssd_kv *kv, const int32_t *dev_tokens, const int32_t *dev_n_tokens, int max_tokens,
+               void *dev_ws, size_t ws_bytes, void *stream) {
+    if (!m || !kv || !dev_tokens || !dev_n_tokens || max_tokens < 0) return SSD_E_ARG;
+    if (!same_cache_shape(m, kv)) return SSD_E_ARG;
+    if (kv->len_ub + max_tokens > kv->S) return SSD_E_CAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    int C = kMaxRows / kv->B;
+    if (C > 8) C = 8;
+    if (C < 1) return SSD_E_CAPACITY;
+    Workspace w;
+    int rc = check_ws(m, kv->B, C, dev_ws, ws_bytes, &w);
+    if (rc) return rc;
+    const int chunks = ceil_div(max_tokens, C);
+    for (int c = 0; c < chunks; ++c) {
+        LAUNCH(prefill_rows_kernel, ceil_div(kv->B, 64), 64, 0, st, dev_n_tokens, c, C, w.n_rows_tmp, kv->B);
+        if ((rc = forward(m, kv, dev_tokens + (size_t)c * C, max_tokens, C, w.n_rows_tmp, false, w, st))) return rc;
+        LAUNCH(kv_commit_rows_kernel, ceil_div(kv->B, 64), 64, 0, st, kv->len, w.ri.n_eff, kv->B);
+        kv->len_ub += C;
+        if (kv->len_ub > kv->S) kv->len_ub = kv->S;
+    }
+    return SSD_OK;
+}
+
+int draft_step(ssd_model *draft, ssd_kv *dkv, const int32_t *dev_tokens_in, int tokens_stride, int rows_in,
+               const int32_t *dev_n_in, float temperature, const float *dev_u, int u_stride, int32_t *dev_token_out,
+               int token_out_stride, float *dev_q_out, size_t q_stride, void *dev_ws, size_t ws_bytes, void *stream) {
+    if (!draft || !dkv || !dev_tokens_in || !dev_u || !dev_token_out || !dev_q_out) return SSD_E_ARG;
+    if (rows_in < 1 || rows_in > 2 || tokens_stride < rows_in || temperature < 0.f) return SSD_E_ARG;
+    if (!same_cache_shape(draft, dkv)) return SSD_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    Workspace w;
+    int rc = check_ws(draft, dkv->B, rows_in, dev_ws, ws_bytes, &w);
+    if (rc) return rc;
+    if ((rc = forward(draft, dkv, dev_tokens_in, tokens_stride, rows_in, dev_n_in, true, w, st))) return rc;
+    DraftTailArgs t;
+    t.logits = w.logits; t.M = rows_in; t.V = draft->a.vocab; t.n_eff = w.ri.n_eff;
+    t.inv_t = temperature > 0.f ? 1.0f / temperature : 0.f;
+    t.u = dev_u; t.u_stride = u_stride;
+    t.token_out = dev_token_out; t.token_stride = token_out_stride;
+    t.q_out = dev_q_out; t.q_stride = q_stride;
+    LAUNCH(draft_tail_kernel, dkv->B, kTailThreads, 0, st, t);
+    LAUNCH(kv_commit_rows_kernel, ceil_div(dkv->B, 64), 64, 0, st, dkv->len, w.ri.n_eff, dkv->B);
+    dkv->len_ub += rows_in;
+    if (dkv->len_ub > dkv->S) dkv->len_ub = dkv->S;
+    return SSD_OK;
+}
+
+size_t verify_scratch_bytes(int batch, int K) {
+    if (batch < 1 || K < 0) return 0;
+    return align_up(sizeof(RowStat) * (size_t)batch * (K + 1), 256);
+}
+
+static int run_verify_tail(const float *logits, int B, int K, int V, const int32_t *rows, const float *q,
+                           const float *u, float temperature, int32_t *n_acc, int32_t *next, int next_stride,
+                           float *p_debug, int32_t *keep, RowStat *stats, cudaStream_t st) {
+    VerifyArgs v;
+    v.logits = logits; v.K = K; v.V = V; v.rows = rows; v.q = q; v.u = u;
+    v.inv_t = temperature > 0.f ? 1.0f / temperature : 0.f;
+    v.n_accepted = n_acc; v.next_token = next; v.next_stride = next_stride;
+    v.p_debug = p_debug; v.keep = keep; v.stats = stats;
+    LAUNCH(row_stats_kernel, dim3(K + 1, B), kTailThreads, 0, st, v);
+    LAUNCH(verify_kernel, B, kTailThreads, 0, st, v);
+    return SSD_OK;
+}
+
+int verify_from_logits(const float *dev_logits, int batch, int K, int vocab, const int32_t *dev_rows,
+                       const float *dev_q, const float *dev_u, float temperature, int32_t *dev_n_accepted,
+                       int32_t *dev_next_token, int next_token_stride, float *dev_p_debug, void *dev_scratch,
+                       size_t scratch_bytes, void *stream) {
+    if (!dev_logits || !dev_rows || !dev_u || !dev_n_accepted || !dev_next_token || !dev_scratch) return SSD_E_ARG;
+    if (batch < 1 || K < 0 || K + 1 > kMaxRowsPerSeq || vocab < 1 || temperature < 0.f || next_token_stride < 1)
+        return SSD_E_ARG;
+    if (K > 0 && !dev_q) return SSD_E_ARG;
+    if (scratch_bytes < verify_scratch_bytes(batch, K)) return SSD_E_CAPACITY;
+    return run_verify_tail(dev_logits, batch, K, vocab, dev_rows, dev_q, dev_u, temperature, dev_n_accepted,
+                           dev_next_token, next_token_stride, dev_p_debug, nullptr, (RowStat *)dev_scratch,
+                           (cudaStream_t)stream);
+}
+
+int target_verify(ssd_model *target, ssd_kv *tkv, const int32_t *dev_rows, int K, const float *dev_q,
+                  const float *dev_u, float temperature, int32_t *dev_n_accepted, int32_t *dev_next_token,
+                  int next_token_stride, float *dev_p_debug, void *dev_ws, size_t ws_bytes, void *stream) {
+    if (!target || !tkv || !dev_rows || !dev_u || !dev_n_accepted || !dev_next_token) return SSD_E_ARG;
+    if (K < 0 || K + 1 > kMaxRowsPerSeq || temperature < 0.f || next_token_stride < 1) return SSD_E_ARG;
+    if (K > 0 && !dev_q) return SSD_E_ARG;
+    if (!same_cache_shape(target, tkv)) return SSD_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    Workspace w;
+    int rc = check_ws(target, tkv->B, K + 1, dev_ws, ws_bytes, &w);
+    if (rc) return rc;
+    if ((rc = forward(target, tkv, dev_rows, K + 1, K + 1, nullptr, true, w, st))) return rc;
+    return run_verify_tail(w.logits, tkv->B, K, target->a.vocab, dev_rows, dev_q, dev_u, temperature, dev_n_accepted,
+                           dev_next_token, next_token_stride, dev_p_debug, tkv->keep, w.stats, st);
+}
+
+int kv_commit(ssd_kv *kv, const int32_t *dev_n_keep, void *stream) {
+    if (!kv) return SSD_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    LAUNCH(kv_commit_kernel, ceil_div(kv->B, 64), 64, 0, st, kv->len, dev_n_keep ? dev_n_keep : kv->keep, kv->B);
+    kv->len_ub += kv->last_rows > 0 ? kv->last_rows : 1;
+    if (kv->len_ub > kv->S) kv->len_ub = kv->S;
+    return SSD_OK;
+}
+
+int kv_rollback(ssd_kv *kv, const int32_t *dev_new_len, void *stream) {
+    if (!kv || !dev_new_len) return SSD_E_ARG;
+    LAUNCH(kv_rollback_kernel, ceil_div(kv->B, 64), 64, 0, (cudaStream_t)stream, kv->len, dev_new_len, kv->B);
+    return SSD_OK;
+}
+
+int spec_advance(ssd_kv *tkv, ssd_kv *dkv, int32_t *dev_rows, int K, const int32_t *dev_n_accepted,
+                 const int32_t *dev_next_token, int next_token_stride, int32_t *dev_out_tokens, int out_cap,
+                 int32_t *dev_out_count, int32_t *dev_draft_in, int32_t *dev_draft_n_in, void *stream) {
+    if (!tkv || !dev_rows || !dev_n_accepted || !dev_next_token || K < 0 || next_token_stride < 1) return SSD_E_ARG;
+    if (dkv && dkv->B != tkv->B) return SSD_E_ARG;
+    AdvanceArgs a;
+    a.tlen = tkv->len; a.dlen = dkv ? dkv->len : nullptr;
+    a.rows = dev_rows; a.K = K; a.B = tkv->B;
+    a.n_accepted = dev_n_accepted; a.next_token = dev_next_token; a.next_stride = next_token_stride;
+    a.out_tokens = dev_out_tokens; a.out_cap = out_cap; a.out_count = dev_out_count;
+    a.draft_in = dev_draft_in; a.draft_n_in = dev_draft_n_in;
+    LAUNCH(spec_advance_kernel, ceil_div(tkv->B, 64), 64, 0, (cudaStream_t)stream, a);
+    tkv->len_ub += K + 1;
+    if (tkv->len_ub > tkv->S) tkv->len_ub = tkv->S;
+    return SSD_OK;
+}
+
+int kv_lengths(ssd_kv *kv, int32_t *host_out, void *stream) {
+    if (!kv || !host_out) return SSD_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_OK(cudaMemcpyAsync(host_out, kv->len, sizeof(int32_t) * kv->B, cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    int mx = 0;
+    for (int b = 0; b < kv->B; ++b) mx = host_out[b] > mx ? host_out[b] : mx;
+    kv->len_ub = mx;  // the bound is exact again
+    return SSD_OK;
+}
+
+int ssd_device_status(ssd_kv *kv, int32_t *host_out, void *stream) {
+    if (!kv || !host_out) return SSD_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_OK(cudaMemcpyAsync(host_out, kv->status, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CUDA_OK(cudaStreamSynchronize(st));
+    return SSD_OK;
+}
+
+int attention_rows(ssd_model *m, ssd_kv *kv, int layer, const float *dev_q, int rows, float *dev_out, void *dev_ws,
+                   size_t ws_bytes, void *stream) {
+    if (!m || !kv || !dev_q || !dev_out || layer < 0 || layer >= m->a.n_layers) return SSD_E_ARG;
+    if (!same_cache_shape(m, kv)) return SSD_E_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    Workspace w;
+    int rc = check_ws(m, kv->B, rows, dev_ws, ws_bytes, &w);
+    if (rc) return rc;
+    // the probe rows are not appended: row j attends whatever the cache holds at 0 .. len + j
+    if ((rc = run_setup(m, kv, rows, nullptr, w, st))) return rc;
+    CombineArgs cb;
+    memset(&cb, 0, sizeof(cb));
+    cb.out_f32 = dev_out;
+    return run_attention(m, kv, layer, dev_q, rows, w, cb, st);
+}
+
+int ssd_last_logits(const ssd_model *m, int batch, int rows_per_seq, const void *dev_ws, size_t ws_bytes,
+                    float *dev_out, void *stream) {
+    if (!m || !dev_out) return SSD_E_ARG;
+    Workspace w;
+    int rc = check_ws(m, batch, rows_per_seq, const_cast<void *>(dev_ws), ws_bytes, &w);
+    if (rc) return rc;
+    CUDA_OK(cudaMemcpyAsync(dev_out, w.logits, sizeof(float) * (size_t)batch * rows_per_seq * m->a.vocab,
+                            cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return SSD_OK;
+}
+
+uint64_t ssd_launch_count(void) { return g_launches.load(); }
+
+int ssd_gemm_profile(int enable) {
+    g_prof = enable != 0;
+    g_prof_used = 0;
+    return SSD_OK;
+}
+
+int ssd_gemm_profile_read(uint64_t *launches, double *total_ms, int reset) {
+    if (!launches || !total_ms) return SSD_E_ARG;
+    CUDA_OK(cudaDeviceSynchronize());
+    double ms = 0.0;
+    for (size_t i = 0; i + 1 < g_prof_used; i += 2) {
+        float t = 0.f;
+        CUDA_OK(cudaEventElapsedTime(&t, g_prof_events[i], g_prof_events[i + 1]));
+        ms += t;
+    }
+    *launches = g_prof_used / 2;
+    *total_ms = ms;
+    if (reset) g_prof_used = 0;
+    return SSD_OK;
+}
+
+const char *ssd_strerror(int status) {
+    switch (status) {
+        case SSD_OK: return "ok";
+        case SSD_E_ARG: return "bad argument";
+        case SSD_E_SHAPE: return "architecture not covered by the kernels";
+        case SSD_E_CAPACITY: return "rows do not fit (cache, workspace or position table)";
+        case SSD_E_CUDA: return "CUDA call failed";
+        case SSD_E_TIMEOUT: return "a bounded device-side wait gave up";
+        case SSD_E_UNIMPL: return "not implemented";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,293 @@
+// Vocabulary-wide tail of a step: temperature softmax statistics, the accept / reject scan,
+// residual renormalise-and-resample or bonus draw, and the draft's "sample from q, export q".
+// (Section "Speculative Sampling", Figure 2: the target "qualifies and accepts (or rejects)" the
+// draft tokens and generates one token itself.)  No host round-trip: everything a decision
+// needs stays on the device; reductions use warp shuffles, prefix sums run in fp64.
+#pragma once
+#include "common.cuh"
+
+namespace ssd {
+
+constexpr int kTailThreads = 1024;
+
+struct RowStat {
+    float mx;      // max logit of the row
+    float z;       // sum exp((l - mx) / T)
+    int32_t amax;  // argmax (lowest index among maxima)
+    int32_t pad;
+};
+
+// p_j of a row from its statistics; the one place this is computed, so the rows exported for
+// inspection are bit-identical to the rows the decisions use.
+__device__ __forceinline__ float prob_of(float logit, const RowStat &st, float inv_t, int j) {
+    if (inv_t == 0.f) return j == st.amax ? 1.f : 0.f;  // greedy: one-hot at the argmax
+    return expf((logit - st.mx) * inv_t) / st.z;
+}
+
+// Block-wide (max, lowest index of max).
+__device__ __forceinline__ void block_argmax(float v, int idx, float *sv, int *si, float &out_v, int &out_i) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, v, o);
+        int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+        if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+    }
+    __syncthreads();
+    if (lane == 0) { sv[w] = v; si[w] = idx; }
+    __syncthreads();
+    if (w == 0) {
+        v = lane < nw ? sv[lane] : -INFINITY;
+        idx = lane < nw ? si[lane] : 0x7fffffff;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            float ov = __shfl_xor_sync(0xffffffffu, v, o);
+            int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+            if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+        }
+        if (lane == 0) { sv[0] = v; si[0] = idx; }
+    }
+    __syncthreads();
+    out_v = sv[0];
+    out_i = si[0];
+}
+
+// Row statistics of logits[row, :]; every thread returns the same RowStat.
+__device__ __forceinline__ RowStat row_stats(const float *logits, int V, float inv_t, float *sv, int *si,
+                                             double *sd) {
+    float mx = -INFINITY;
+    int am = 0x7fffffff;
+    for (int j = threadIdx.x; j < V; j += blockDim.x) {
+        float l = logits[j];
+        if (l > mx) { mx = l; am = j; }  // strided ascending: first maximum per thread
+    }
+    RowStat st;
+    block_argmax(mx, am, sv, si, st.mx, st.amax);
+    double z = 0.0;
+    if (inv_t != 0.f) {
+        float part = 0.f;
+        for (int j = threadIdx.x; j < V; j += blockDim.x) part += expf((logits[j] - st.mx) * inv_t);
+        z = block_sum((double)part, sd);
+    }
+    st.z = (float)z;
+    st.pad = 0;
+    return st;
+}
+
+// Inverse-CDF draw over V weights w(j) >= 0: the smallest j whose inclusive prefix sum exceeds
+// u * S; prefix sums in index order, fp64.  If rounding leaves none: the largest j with w > 0.
+// Each thread owns a contiguous segment so the prefix order is the index order.  Returns S via
+// *total (all threads); the drawn index is valid in all threads.  S <= 0 returns -1.
+template <typename WeightFn>
+__device__ __forceinline__ int inv_cdf_block(WeightFn w, int V, float u, double *sd, int *si, double *total) {
+    const int seg = (V + blockDim.x - 1) / blockDim.x;
+    const int j0 = min(V, (int)threadIdx.x * seg), j1 = min(V, j0 + seg);
+    double local = 0.0;
+    int last_pos = -1;
+    for (int j = j0; j < j1; ++j) {
+        float wj = w(j);
+        local += (double)wj;
+        if (wj > 0.f) last_pos = j;
+    }
+    // exclusive scan of the per-thread sums over the block (warp scan + scan of warp totals)
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    double incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        double t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();
+    if (lane == 31) sd[wid] = incl;
+    if (threadIdx.x == 0) { si[0] = 0x7fffffff; si[1] = -1; }
+    __syncthreads();
+    double warp_off = 0.0, S = 0.0;
+    for (int k = 0; k < nw; ++k) {  // nw <= 32: short serial pass keeps the order fixed
+        double t = sd[k];
+        if (k < wid) warp_off += t;
+        S += t;
+    }
+    *total = S;
+    if (!(S > 0.0)) { __syncthreads(); return -1; }
+    const double target = (double)u * S;
+    double run = warp_off + (incl - local);
+    int hit = 0x7fffffff;
+    if (run + local > target || run > target) {
+        for (int j = j0; j < j1; ++j) {
+            const float wj = w(j);
+            run += (double)wj;
+            if (wj > 0.f && run > target) { hit = j; break; }  // a zero-weight index is never drawn
+        }
+    }
+    if (hit != 0x7fffffff) atomicMin(&si[0], hit);
+    if (last_pos >= 0) atomicMax(&si[1], last_pos);
+    __syncthreads();
+    int res = si[0] != 0x7fffffff ? si[0] : si[1];
+    __syncthreads();
+    return res;
+}
+
+struct VerifyArgs {
+    const float *logits;    // [B, K+1, V]
+    int K, V;
+    const int32_t *rows;    // [B, K+1]: pending, x~_1..x~_K
+    const float *q;         // [B, K, V]
+    const float *u;         // [B, K+1]
+    float inv_t;            // 1/T, 0 = greedy
+    int32_t *n_accepted;    // [B]
+    int32_t *next_token;
+    int next_stride;
+    float *p_debug;         // [B, K+1, V] or null
+    int32_t *keep;          // [B] or null: n_accepted + 1 for kv_commit
+    RowStat *stats;         // scratch [B, K+1]
+};
+
+// grid (K+1, B): statistics of every row (+ optional export of the p row)
+__global__ void __launch_bounds__(kTailThreads) row_stats_kernel(VerifyArgs a) {
+    __shared__ float sv[32];
+    __shared__ int si[32];
+    __shared__ double sd[32];
+    const int i = blockIdx.x, b = blockIdx.y;
+    const float *lg = a.logits + ((size_t)b * (a.K + 1) + i) * a.V;
+    RowStat st = row_stats(lg, a.V, a.inv_t, sv, si, sd);
+    if (threadIdx.x == 0) a.stats[b * (a.K + 1) + i] = st;
+    if (a.p_debug) {
+        float *p = a.p_debug + ((size_t)b * (a.K + 1) + i) * a.V;
+        for (int j = threadIdx.x; j < a.V; j += blockDim.x) p[j] = prob_of(lg[j], st, a.inv_t, j);
+    }
+}
+
+// grid (B): accept scan, then residual / bonus draw
+__global__ void __launch_bounds__(kTailThreads) verify_kernel(VerifyArgs a) {
+    __shared__ double sd[32];
+    __shared__ int si[32];
+    __shared__ int s_acc;
+    const int b = blockIdx.x, K = a.K, V = a.V;
+    const RowStat *st = a.stats + b * (K + 1);
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int i = 0; i < K; ++i) {
+            int x = a.rows[b * (K + 1) + 1 + i];
+            x = max(0, min(x, V - 1));
+            const float px = prob_of(a.logits[((size_t)b * (K + 1) + i) * V + x], st[i], a.inv_t, x);
+            const float qx = a.q[((size_t)b * K + i) * V + x];
+            // accept with probability min(1, p/q): u * q < p, one fp32 rounding of the product
+            if (__fmul_rn(a.u[b * (K + 1) + i], qx) < px) ++acc; else break;
+        }
+        s_acc = acc;
+    }
+    __syncthreads();
+    const int acc = s_acc;
+    const float *lg = a.logits + ((size_t)b * (K + 1) + acc) * V;
+    const RowStat rs = st[acc];
+    const float u = a.u[b * (K + 1) + K];
+    const float inv_t = a.inv_t;
+    double S;
+    int y = -1;
+    if (acc < K) {
+        const float *qr = a.q + ((size_t)b * K + acc) * V;
+        y = inv_cdf_block([&](int j) { return fmaxf(0.f, __fsub_rn(prob_of(lg[j], rs, inv_t, j), qr[j])); }, V, u,
+                          sd, si, &S);
+    }
+    if (y < 0)  // all accepted: bonus from p_{K+1}; or an all-zero residual: fall back to p
+        y = inv_cdf_block([&](int j) { return prob_of(lg[j], rs, inv_t, j); }, V, u, sd, si, &S);
+    if (y < 0) y = rs.amax;  // a row whose probabilities all vanished (non-finite logits)
+    if (threadIdx.x == 0) {
+        a.n_accepted[b] = acc;
+        a.next_token[(size_t)b * a.next_stride] = y;
+        if (a.keep) a.keep[b] = acc + 1;
+    }
+}
+
+struct DraftTailArgs {
+    const float *logits;  // [B, M, V] rows of the draft forward
+    int M, V;
+    const int32_t *n_eff; // [B] rows fed per sequence (the last one is sampled)
+    float inv_t;
+    const float *u; int u_stride;
+    int32_t *token_out; int token_stride;
+    float *q_out; size_t q_stride;
+};
+
+// grid (B): q = softmax(last row / T), exported; x~ = inverse-CDF(q, u)
+__global__ void __launch_bounds__(kTailThreads) draft_tail_kernel(DraftTailArgs a) {
+    __shared__ float sv[32];
+    __shared__ int si[32];
+    __shared__ double sd[32];
+    const int b = blockIdx.x;
+    int row = a.n_eff[b] - 1;
+    if (row < 0) row = 0;
+    const float *lg = a.logits + ((size_t)b * a.M + row) * a.V;
+    const RowStat st = row_stats(lg, a.V, a.inv_t, sv, si, sd);
+    float *q = a.q_out + (size_t)b * a.q_stride;
+    for (int j = threadIdx.x; j < a.V; j += blockDim.x) q[j] = prob_of(lg[j], st, a.inv_t, j);
+    __syncthreads();
+    double S;
+    int y = inv_cdf_block([&](int j) { return q[j]; }, a.V, a.u[(size_t)b * a.u_stride], sd, si, &S);
+    if (y < 0) y = st.amax;
+    if (threadIdx.x == 0) a.token_out[(size_t)b * a.token_stride] = y;
+}
+
+// ---------------- cache length bookkeeping ----------------
+__global__ void kv_commit_kernel(int32_t *len, const int32_t *n_keep, int B) {
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) len[b] += max(0, n_keep[b]);
+}
+__global__ void kv_commit_rows_kernel(int32_t *len, const int32_t *n_eff, int B) {
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) len[b] += n_eff[b];
+}
+__global__ void kv_rollback_kernel(int32_t *len, const int32_t *new_len, int B) {
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) len[b] = max(0, min(len[b], new_len[b]));
+}
+// chunk c of a prompt pass: rows fed per sequence = clamp(n_tokens - c*C, 0, C)
+__global__ void prefill_rows_kernel(const int32_t *n_tokens, int chunk, int C, int32_t *n_rows, int B) {
+    int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < B) n_rows[b] = max(0, min(C, n_tokens[b] - chunk * C));
+}
+
+struct AdvanceArgs {
+    int32_t *tlen, *dlen;  // target / draft committed lengths (dlen may be null)
+    int32_t *rows;         // [B, K+1]
+    int K, B;
+    const int32_t *n_accepted, *next_token;
+    int next_stride;
+    int32_t *out_tokens; int out_cap; int32_t *out_count;
+    int32_t *draft_in, *draft_n_in;
+};
+
+__global__ void spec_advance_kernel(AdvanceArgs a) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= a.B) return;
+    const int K = a.K;
+    int acc = max(0, min(a.n_accepted[b], K));
+    const int y = a.next_token[(size_t)b * a.next_stride];
+    int32_t *row = a.rows + (size_t)b * (K + 1);
+    const int n = a.tlen[b] + 1;  // committed tokens before this iteration
+    if (a.out_tokens && a.out_count) {
+        int c = a.out_count[b];
+        for (int i = 0; i < acc; ++i, ++c)
+            if (c < a.out_cap) a.out_tokens[(size_t)b * a.out_cap + c] = row[1 + i];
+        if (c < a.out_cap) a.out_tokens[(size_t)b * a.out_cap + c] = y;
+        a.out_count[b] = c + 1;
+    } else if (a.out_count) {
+        a.out_count[b] += acc + 1;
+    }
+    if (a.draft_in && a.draft_n_in) {
+        if (acc == K && K > 0) {
+            a.draft_in[2 * b] = row[K];
+            a.draft_in[2 * b + 1] = y;
+            a.draft_n_in[b] = 2;
+        } else {
+            a.draft_in[2 * b] = y;
+            a.draft_in[2 * b + 1] = y;
+            a.draft_n_in[b] = 1;
+        }
+    }
+    a.tlen[b] += acc + 1;
+    if (a.dlen) a.dlen[b] = min(a.dlen[b], K > 0 ? min(n + acc, n + K - 1) : n + acc);
+    row[0] = y;
+}
+
+}  // namespace ssd

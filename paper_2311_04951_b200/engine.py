@@ -1,0 +1,119 @@
+"""Generation loops on top of the C ABI: orchestration only (which call comes next, where its
+buffers live).  No arithmetic of the method happens here; every number is produced by the
+library's kernels.
+
+One speculative iteration (Section "Speculative Sampling", Figure 2; cache handling of Section
+"So, what's the problem?") is:  K x draft_step  ->  target_verify  ->  spec_advance,
+all queued on one stream, wired through device buffers so that nothing returns to the host:
+draft_step writes its token straight into the verification row block and its q row straight
+into the q block; spec_advance writes the next pending token and the draft's catch-up rows.
+"""
+from __future__ import annotations
+
+from typing import Callable, Dict, List, Optional
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+class Engine:
+    def __init__(self, target: B.Model, draft: Optional[B.Model], batch: int, max_len: int, K: int,
+                 temperature: float, out_cap: int):
+        self.target, self.draft = target, draft
+        self.batch, self.max_len, self.K, self.T = batch, max_len, K, float(temperature)
+        V = target.arch.vocab
+        dev = "cuda"
+        self.tkv = B.KV(target, batch, max_len)
+        self.ws_t = target.new_workspace(batch, K + 1, max_len)
+        self.rows = torch.zeros(batch, K + 1, dtype=torch.int32, device=dev)
+        self.n_acc = torch.zeros(batch, dtype=torch.int32, device=dev)
+        self.next_tok = torch.zeros(batch, dtype=torch.int32, device=dev)
+        self.out_cap = out_cap
+        self.out_tokens = torch.zeros(batch, out_cap, dtype=torch.int32, device=dev)
+        self.out_count = torch.zeros(batch, dtype=torch.int32, device=dev)
+        self.chunk = min(8, B.MAX_ROWS // batch)
+        self.ws_pre_t = target.new_workspace(batch, self.chunk, max_len)
+        if draft is not None and K > 0:
+            self.dkv = B.KV(draft, batch, max_len)
+            self.ws_d = draft.new_workspace(batch, 2, max_len)
+            self.ws_pre_d = draft.new_workspace(batch, self.chunk, max_len)
+            self.q = torch.zeros(batch, K, V, dtype=torch.float32, device=dev)
+            self.draft_in = torch.zeros(batch, 2, dtype=torch.int32, device=dev)
+            self.draft_n_in = torch.ones(batch, dtype=torch.int32, device=dev)
+        else:
+            self.dkv = None
+            self.q = None
+
+    # ---- prompt pass (functional, untimed) ----
+    def prefill(self, prompts: torch.Tensor) -> None:
+        """prompts int32 [batch, P] on the device: all but the last token are fed to both caches; the
+        last one becomes the pending token."""
+        P = prompts.shape[1]
+        if P > 1:
+            body = prompts[:, :P - 1].contiguous()
+            n = torch.full((self.batch,), P - 1, dtype=torch.int32, device=prompts.device)
+            B.kv_prefill(self.target, self.tkv, body, n, self.ws_pre_t)
+            if self.dkv is not None:
+                B.kv_prefill(self.draft, self.dkv, body, n, self.ws_pre_d)
+        self.rows[:, 0] = prompts[:, P - 1]
+        if self.dkv is not None:
+            self.draft_in[:, 0] = prompts[:, P - 1]
+            self.draft_n_in.fill_(1)
+        self.out_count.zero_()
+
+    # ---- one iteration; u_draft [batch, K], u_verify [batch, K+1] fp32 on the device ----
+    def spec_iteration(self, u_draft: torch.Tensor, u_verify: torch.Tensor, p_debug: Optional[torch.Tensor] = None):
+        K, V = self.K, self.target.arch.vocab
+        for i in range(K):
+            if i == 0:
+                tok_in, stride, rows_in, n_in = self.draft_in, 2, 2, self.draft_n_in
+            else:
+                tok_in, stride, rows_in, n_in = self.rows[:, i:], K + 1, 1, None
+            B.draft_step(self.draft, self.dkv, tok_in, stride, rows_in, n_in, self.T, u_draft[:, i:], K,
+                         self.rows[:, i + 1:], K + 1, self.q[:, i], K * V, self.ws_d)
+        B.target_verify(self.target, self.tkv, self.rows, K, self.q, u_verify, self.T, self.n_acc, self.next_tok, 1,
+                        p_debug, self.ws_t)
+
+    def advance(self) -> None:
+        B.spec_advance(self.tkv, self.dkv, self.rows, self.K, self.n_acc, self.next_tok, 1, self.out_tokens,
+                       self.out_cap, self.out_count, self.draft_in if self.dkv is not None else None,
+                       self.draft_n_in if self.dkv is not None else None)
+
+    def ar_step(self, u: torch.Tensor, p_debug: Optional[torch.Tensor] = None) -> None:
+        """Plain autoregressive decode step (Eq. 1): one row per sequence, token drawn with u [batch, 1]."""
+        assert self.K == 0
+        B.target_verify(self.target, self.tkv, self.rows, 0, None, u, self.T, self.n_acc, self.next_tok, 1, p_debug,
+                        self.ws_t)
+        self.advance()
+
+    # ---- whole generations ----
+    def generate(self, prompts: np.ndarray, n_new: int, uniforms: Callable[[int, int], np.ndarray],
+                 check_every: int = 4, max_iters: Optional[int] = None) -> Dict:
+        """uniforms(seq, iteration) -> fp32 [2K+1] (speculative) or [>=1] (autoregressive, K == 0).
+        Runs until every sequence has >= n_new tokens; the host only polls the counters."""
+        dev = "cuda"
+        K = self.K
+        self.prefill(torch.from_numpy(np.ascontiguousarray(prompts, np.int32)).to(dev))
+        iters = 0
+        limit = max_iters if max_iters is not None else n_new
+        while iters < limit:
+            for _ in range(check_every):
+                if iters >= limit:
+                    break
+                u = np.stack([uniforms(s, iters) for s in range(self.batch)]).astype(np.float32)
+                if K == 0:
+                    self.ar_step(torch.from_numpy(u[:, :1].copy()).to(dev))
+                else:
+                    ud = torch.from_numpy(u[:, :K].copy()).to(dev)
+                    uv = torch.from_numpy(u[:, K:2 * K + 1].copy()).to(dev)
+                    self.spec_iteration(ud, uv)
+                    self.advance()
+                iters += 1
+            if int(self.out_count.min().item()) >= n_new:
+                break
+        counts = self.out_count.cpu().numpy()
+        toks = self.out_tokens.cpu().numpy()
+        return {"tokens": [toks[b, :min(n_new, counts[b])].tolist() for b in range(self.batch)],
+                "counts": counts, "iterations": iters, "status": self.tkv.status()}
