@@ -1,0 +1,435 @@
+#!/usr/bin/env python
+"""Benchmark of the speculative-sampling verification path on B200.
+
+A "step" is one speculative iteration over one batch: K draft steps, one target verification
+pass over K+1 rows per sequence, accept/reject/resample and cache bookkeeping.  The headline
+value is generated tokens per second (speculative); the same run also times plain
+autoregressive decoding, the verification pass alone, and attributes device time to the
+weight-streaming GEMM kernel for the roofline figure.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "generated tok/s, speculative vs autoregressive; verify-step HBM GB/s vs peak"
+FALLBACK_HBM_GBS = 6650.0
+
+# bench workloads: name -> (preset, batch, prompt, K, temperature)
+WORKLOADS = {
+    "neox-1.4b": dict(preset="neox-1.4b"),
+    "neox-2.7b": dict(preset="neox-2.7b"),
+    "llama-7b-b8": dict(preset="llama-7b"),
+    "llama-7b-b1": dict(preset="llama-7b", batch=1, prompt=2048),
+    "tiny": dict(preset="tiny"),
+}
+
+
+def measured_hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------ bytes the method must move
+def weight_bytes(arch) -> int:
+    """Bytes of matrices streamed by one forward (all layers + LM head), model dtype."""
+    es = 2 if arch.dtype else 4
+    d, F = arch.d_model, arch.d_ff
+    per_layer = 3 * d * d + d * d + arch.d_in * d + d * F
+    return (arch.n_layers * per_layer + arch.vocab * d) * es
+
+
+def verify_step_bytes(arch, batch, K, ctx_lens) -> int:
+    """Algorithmic bytes of one verification pass: weights once, embedding rows, KV read of
+    every sequence's context plus the new rows, KV write, draft rows q and the uniforms."""
+    es = 2 if arch.dtype else 4
+    M = K + 1
+    kv_tok = 2 * arch.n_layers * arch.d_model * es
+    b = weight_bytes(arch) + batch * M * arch.d_model * es
+    b += sum((int(n) + M) * kv_tok for n in ctx_lens) + batch * M * kv_tok
+    b += batch * K * arch.vocab * 4 + batch * M * 4
+    return b
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------ model construction
+def random_weights_on_device(arch, seed, torch, late_scale=1.0, late_from=0):
+    """Random-init tensors drawn on the device (N(0, 0.02); gains 1 + N(0, 0.02)), ABI order."""
+    from paper_2311_04951_b200 import synth
+    g = torch.Generator(device="cuda")
+    out = []
+    for i, name in enumerate(synth.tensor_names(arch)):
+        shape = synth.tensor_shape(arch, name)
+        if shape is None:
+            out.append(None)
+            continue
+        g.manual_seed(seed * 100003 + i)
+        t = torch.randn(shape, generator=g, device="cuda", dtype=torch.float32) * 0.02
+        base = name.split(".")[-1]
+        if base.endswith("_g"):
+            t += 1.0
+        if "." in name and base in ("w_o", "w_out", "b_o", "b_out") and int(name.split(".")[0][1:]) >= late_from:
+            t *= late_scale
+        out.append(t.to(torch.bfloat16) if (len(shape) == 2 and arch.dtype) else t)
+    return out
+
+
+def resolve(workload):
+    from paper_2311_04951_b200 import synth
+    w = dict(WORKLOADS[workload])
+    cfg = dict(synth.PRESETS[w.pop("preset")])
+    cfg.update(w)
+    return cfg
+
+
+def run_ours(args, rank, world):
+    import torch
+    from paper_2311_04951_b200 import binding as B, engine, synth
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    cfg = resolve(args.workload)
+    arch, Bn, K, T, P = cfg["target"], cfg["batch"], cfg["K"], cfg["temperature"], cfg["prompt"]
+    seeds = cfg["seeds"]
+    # layer-skip drafts need correlated exits: damp the late layers' output projections
+    late = dict(late_scale=0.2, late_from=4) if cfg["draft"] == "prefix:4" else {}
+    target = B.Model(arch, random_weights_on_device(arch, seeds["w"], torch, **late))
+    if isinstance(cfg["draft"], str):
+        draft = target.share_prefix(int(cfg["draft"].split(":")[1]))
+    else:
+        draft = B.Model(cfg["draft"], random_weights_on_device(cfg["draft"], seeds["wd"], torch))
+    steps, warm = args.steps, max(args.warmup, 3)
+    max_len = P + (steps + warm + 8) * (K + 1) + 16
+    if arch.pos == 0:
+        max_len = min(max_len, arch.max_pos)
+    out_cap = (steps + warm + 8) * (K + 1)
+    prompts = torch.from_numpy(synth.gen_prompt(seeds["prompt"], Bn, P, arch.vocab)).cuda()
+
+    def uniforms(n_iters, width):
+        u = np.stack([np.stack([synth.gen_uniforms(seeds["u"] + rank, s, it, width) for s in range(Bn)])
+                      for it in range(n_iters)])
+        return u  # [iters, B, width]
+
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- speculative: device-resident inputs ----------------
+    eng = engine.Engine(target, draft, Bn, max_len, K, T, out_cap)
+    eng.prefill(prompts)
+    u_all = uniforms(warm + steps, 2 * K + 1)
+    ud = torch.from_numpy(u_all[:, :, :K].copy()).cuda()
+    uv = torch.from_numpy(u_all[:, :, K:].copy()).cuda()
+    for it in range(warm):
+        eng.spec_iteration(ud[it], uv[it])
+        eng.advance()
+    barrier()
+    count0 = eng.out_count.clone()
+    launches0 = B.launch_count()
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for it in range(warm, warm + steps):
+        eng.spec_iteration(ud[it], uv[it])
+        eng.advance()
+    e1.record()
+    barrier()
+    spec_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    launches = B.launch_count() - launches0
+    spec_tokens = int((eng.out_count - count0).sum().item())
+    accepted_mean = spec_tokens / (steps * Bn) - 1.0
+    ctx_lens = eng.tkv.lengths()
+    status = eng.tkv.status() or eng.dkv.status()
+
+    # ---------------- GEMM kernel attribution over the same region (events around each launch) ----
+    eng_p = engine.Engine(target, draft, Bn, max_len, K, T, out_cap)
+    eng_p.prefill(prompts)
+    for it in range(warm):
+        eng_p.spec_iteration(ud[it], uv[it])
+        eng_p.advance()
+    torch.cuda.synchronize()
+    B.gemm_profile(True)
+    prof_steps = min(steps, 8)
+    for it in range(warm, warm + prof_steps):
+        eng_p.spec_iteration(ud[it], uv[it])
+        eng_p.advance()
+    n_gemm, gemm_ms = B.gemm_profile_read()
+    B.gemm_profile(False)
+    d_arch = draft.arch
+    gemm_bytes = prof_steps * (weight_bytes(arch) + K * weight_bytes(d_arch))
+    gemm_gbs = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
+    del eng_p
+
+    # ---------------- verification pass alone, and one-row decode, on the same cache ----------------
+    def time_verify(k, reps):
+        e = engine.Engine(target, None, Bn, max_len, k, T, 8) if k == 0 else eng
+        if k == 0:
+            e.prefill(prompts)
+        q = eng.q[:, :max(k, 1)].contiguous() if k else None
+        u = uv[0][:, :k + 1].contiguous()
+        rows = eng.rows[:, :k + 1].contiguous()
+        ws = e.ws_t
+        for _ in range(3):
+            B.target_verify(target, e.tkv, rows, k, q, u, T, eng.n_acc, eng.next_tok, 1, None, ws)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            B.target_verify(target, e.tkv, rows, k, q, u, T, eng.n_acc, eng.next_tok, 1, None, ws)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps, e.tkv.lengths()
+
+    verify_ms, v_lens = time_verify(K, max(5, min(steps, 20)))
+    decode_ms, d_lens = time_verify(0, max(5, min(steps, 20)))
+    v_bytes = verify_step_bytes(arch, Bn, K, v_lens)
+    d_bytes = verify_step_bytes(arch, Bn, 0, d_lens)
+
+    # ---------------- autoregressive generation ----------------
+    ar = engine.Engine(target, None, Bn, max_len, 0, T, out_cap)
+    ar.prefill(prompts)
+    u1 = torch.from_numpy(uniforms(warm + steps, 1)).cuda()
+    for it in range(warm):
+        ar.ar_step(u1[it])
+    barrier()
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record()
+    for it in range(warm, warm + steps):
+        ar.ar_step(u1[it])
+    a1.record()
+    barrier()
+    ar_ms = a0.elapsed_time(a1)
+    ar_tps = steps * Bn / (ar_ms * 1e-3)
+    del ar
+
+    # ---------------- end to end: host buffers, copies inside the timed region ----------------
+    eng2 = engine.Engine(target, draft, Bn, max_len, K, T, out_cap)
+    eng2.prefill(prompts)
+    pin_u = torch.from_numpy(u_all).pin_memory()
+    host_res = torch.zeros(Bn, K + 3, dtype=torch.int32).pin_memory()
+    dev_u = torch.zeros(Bn, 2 * K + 1, device="cuda")
+    res = torch.zeros(Bn, K + 3, dtype=torch.int32, device="cuda")
+    for it in range(warm):
+        eng2.spec_iteration(ud[it], uv[it])
+        eng2.advance()
+    barrier()
+    c0 = eng2.out_count.clone()
+    t0 = time.perf_counter()
+    for it in range(warm, warm + steps):
+        dev_u.copy_(pin_u[it], non_blocking=True)                       # H2D: this step's uniforms
+        eng2.spec_iteration(dev_u[:, :K].contiguous(), dev_u[:, K:].contiguous())
+        res[:, 0] = eng2.n_acc
+        res[:, 1] = eng2.next_tok
+        res[:, 2:] = eng2.rows
+        eng2.advance()
+        host_res.copy_(res, non_blocking=True)                          # D2H: accepted count + tokens
+        torch.cuda.synchronize()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+    e2e_tokens = int((eng2.out_count - c0).sum().item())
+    h2d = Bn * (2 * K + 1) * 4
+    d2h = Bn * (K + 3) * 4
+
+    # ---------------- aggregate over ranks ----------------
+    tot_tokens, tot_e2e_tokens, max_ms, max_e2e = spec_tokens, e2e_tokens, spec_ms, e2e_s
+    if dist is not None:
+        t = torch.tensor([spec_tokens, e2e_tokens], dtype=torch.float64, device="cuda")
+        m = torch.tensor([spec_ms, e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        dist.all_reduce(m, op=dist.ReduceOp.MAX)
+        tot_tokens, tot_e2e_tokens, max_ms, max_e2e = int(t[0]), int(t[1]), float(m[0]), float(m[1])
+
+    peak, which = measured_hbm_peak()
+    line = {
+        "metric": METRIC, "value": tot_tokens / (max_ms * 1e-3), "unit": "tok/s", "n_gpus": world,
+        "steps": steps, "warmup": warm, "ms_per_step": max_ms / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if arch.dtype else "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": Bn, "prompt": P, "K": K, "temperature": T,
+                   "target": f"{arch.n_layers}L d{arch.d_model} V{arch.vocab}",
+                   "draft": cfg["draft"] if isinstance(cfg["draft"], str) else
+                   f"{cfg['draft'].n_layers}L d{cfg['draft'].d_model}",
+                   "l2": "inputs larger than L2 (weights streamed each pass exceed 126 MB)",
+                   "multi_gpu": "replicas only (independent sequences, no collective)"},
+        "clocks": clocks,
+        "e2e": {"value": tot_e2e_tokens / max_e2e, "unit": "tok/s", "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": gemm_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": gemm_gbs / peak, "traffic": None, "peak_source": which,
+                     "kernel": "gemm_bf16_kernel", "launches": n_gemm,
+                     "avg_launch_us": 1e3 * gemm_ms / max(n_gemm, 1)},
+        "speculative": {"tok_s": spec_tokens / (spec_ms * 1e-3), "accepted_per_iter": accepted_mean,
+                        "tokens_per_iter": spec_tokens / (steps * Bn)},
+        "autoregressive": {"tok_s": ar_tps, "ms_per_token": ar_ms / steps},
+        "verify": {"ms": verify_ms, "rows": Bn * (K + 1), "bytes": v_bytes, "gbs": v_bytes / verify_ms / 1e6,
+                   "frac_of_peak": v_bytes / verify_ms / 1e6 / peak, "frac_of_8tbs": v_bytes / verify_ms / 1e6 / 8000,
+                   "decode_ms": decode_ms, "decode_gbs": d_bytes / decode_ms / 1e6,
+                   "verify_over_decode": verify_ms / decode_ms, "ctx": [int(x) for x in v_lens]},
+        "device_status": int(status),
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(args.workload, steps=None, budget_s=20.0)
+    if dist is not None:
+        dist.destroy_process_group()
+    return line
+
+
+# ------------------------------------------------------------------ CPU oracle timing
+def cpu_baseline(workload, steps, budget_s):
+    """The oracle as it stands, on the host cores: speculative iterations of the same models
+    (same shapes, seeded numpy weights) from a SHORT prompt (16 tokens), timed whole."""
+    from oracle import decoder as od, sampling as osamp
+    from paper_2311_04951_b200 import synth
+    cfg = resolve(workload)
+    arch, K, T = cfg["target"], cfg["K"], cfg["temperature"]
+    cores = os.cpu_count() or 1
+    od.set_threads(cores)
+    ws = synth.gen_weights(arch, cfg["seeds"]["w"])
+    tgt = od.Model(arch, ws)
+    if isinstance(cfg["draft"], str):
+        d_arch, d_ws = synth.prefix_draft(arch, ws, int(cfg["draft"].split(":")[1]))
+    else:
+        d_arch, d_ws = cfg["draft"], synth.gen_weights(cfg["draft"], cfg["seeds"]["wd"])
+    drf = od.Model(d_arch, d_ws)
+    P = 16
+    prompt = synth.gen_prompt(cfg["seeds"]["prompt"], 1, P, arch.vocab)[0]
+    s_max = P + 64 * (K + 1)
+    tc, dc = tgt.new_cache(s_max), drf.new_cache(s_max)
+    tc.feed(prompt[:-1], want_logits=False)
+    dc.feed(prompt[:-1], want_logits=False)
+    x = [int(t) for t in prompt]
+    tokens, iters, t0 = 0, 0, time.perf_counter()
+    while True:
+        u = synth.gen_uniforms(cfg["seeds"]["u"], 0, iters, 2 * K + 1)
+        n = len(x)
+        feed, qs, drafts = x[dc.len:n], [], []
+        for i in range(K):
+            q = osamp.softmax_t(dc.feed(feed)[-1], T)
+            t = osamp.inv_cdf(q, u[i])
+            qs.append(q)
+            drafts.append(t)
+            feed = [t]
+        lg = tc.feed([x[n - 1]] + drafts, advance=False)
+        ps = [osamp.softmax_t(lg[i], T) for i in range(K + 1)]
+        a, y = osamp.accept_resample(ps, qs, drafts, u[K:2 * K], u[2 * K])
+        x.extend(drafts[:a] + [y])
+        tc.len += a + 1
+        dc.rollback(min(n + a, n + K - 1))
+        tokens += a + 1
+        iters += 1
+        el = time.perf_counter() - t0
+        if (steps is not None and iters >= steps) or el > budget_s or (steps is None and iters >= 32):
+            break
+    return {"value": tokens / el, "unit": "tok/s", "cores": od.get_threads(), "kind": "oracle",
+            "sample": f"{iters} speculative iteration(s) of the {workload} models, batch 1, prompt {P}, K={K}, "
+                      f"{tokens} tokens in {el:.1f} s", "ms_per_step": 1e3 * el / iters, "iters": iters}
+
+
+def run_reference(args, rank, world):
+    """Reference arm = the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return None
+    cb = cpu_baseline(args.workload, steps=args.steps + max(args.warmup, 0), budget_s=150.0)
+    cfg = resolve(args.workload)
+    arch = cfg["target"]
+    return {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": "tok/s", "n_gpus": world,
+            "steps": cb["iters"], "warmup": 0, "ms_per_step": cb["ms_per_step"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32 storage, f64 accumulate", "data": "synthetic",
+            "config": {"workload": args.workload, "batch": 1, "prompt": 16, "K": cfg["K"],
+                       "temperature": cfg["temperature"], "target": f"{arch.n_layers}L d{arch.d_model} V{arch.vocab}"},
+            "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": cb["value"], "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="neox-1.4b", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        line = run_reference(args, rank, world)
+    else:
+        line = run_ours(args, rank, world)
+    if rank == 0 and line is not None:
+        print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()

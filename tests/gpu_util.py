@@ -18,6 +18,17 @@ from oracle import sampling as osamp
 
 LOGIT_ATOL, LOGIT_RTOL = 2e-2, 1e-2
 P_ATOL = 1e-4
+# A logit error d moves a probability by a factor e^(+-2d) at most (numerator and normaliser).  On
+# models whose weights are scaled up to make the rows peaky, a bf16-weight logit error well inside
+# LOGIT_ATOL therefore exceeds 1e-4 absolute on a large p; those comparisons add this relative term.
+P_RTOL_PEAKY = 5e-2
+
+
+def assert_probs_close(got, ref, peaky, what=""):
+    err = np.abs(got.astype(np.float64) - ref.astype(np.float64))
+    bound = P_ATOL + (P_RTOL_PEAKY * ref if peaky else 0.0)
+    worst = int(np.argmax(err - bound))
+    assert (err <= bound).all(), f"{what}: |dp| {err.flat[worst]:.3e} at p = {ref.flat[worst]:.3e}"
 
 
 def scaled_weights(synth, arch, seed, scale):
@@ -72,7 +83,7 @@ def check_draw_on_own_row(q_row, u, tok_got):
     return False
 
 
-def lockstep(engine, synth, prompt, n_iters, K, seed_u, oracle_trace, seq=0):
+def lockstep(engine, synth, prompt, n_iters, K, seed_u, oracle_trace, seq=0, peaky=False):
     """Run n_iters speculative iterations on the GPU engine (batch 1), checking layers A-C against
     the oracle's per-iteration records.  Returns (#iterations in sync, #iterations run)."""
     V = engine.target.arch.vocab
@@ -101,13 +112,13 @@ def lockstep(engine, synth, prompt, n_iters, K, seed_u, oracle_trace, seq=0):
             t = oracle_trace[it]
             same_drafts = 0
             for i in range(K):
-                assert np.abs(q[i] - t["q"][i]).max() <= P_ATOL, f"q row {i} of iteration {it}"
+                assert_probs_close(q[i], t["q"][i], peaky, f"q row {i} of iteration {it}")
                 if drafts[i] != t["drafts"][i]:
                     break
                 same_drafts += 1
             # p row i is conditioned on drafts[:i]: comparable while those coincide
             for i in range(same_drafts + 1):
-                assert np.abs(p[i] - t["p"][i]).max() <= P_ATOL, f"p row {i} of iteration {it}"
+                assert_probs_close(p[i], t["p"][i], peaky, f"p row {i} of iteration {it}")
             if same_drafts == K and a == t["a"] and y == t["y"]:
                 synced += 1
             else:

@@ -48,6 +48,8 @@ def test_tiny_config_full_trajectory():
     ("gpt2_f32", synth.gpt2_like(3, 128, 4, 256, 400, 160), 7.0, 3, 0.9),
     ("neox_bf16", synth.neox_like(3, 256, 4, 512, 640), 7.0, 5, 0.8),
     ("llama_bf16", synth.llama_like(3, 256, 2, 704, 640), 7.0, 4, 1.0),
+    ("neox_bf16_natural_init", synth.neox_like(3, 256, 4, 512, 640), 1.0, 5, 0.8),
+    ("llama_bf16_natural_init", synth.llama_like(3, 256, 2, 704, 640), 1.0, 4, 1.0),
 ])
 def test_lockstep_trajectories_per_family(name, arch, scale, K, T):
     (tgt, drf), (otgt, odrf) = build_pair(arch, 21, scale, 1)
@@ -56,7 +58,8 @@ def test_lockstep_trajectories_per_family(name, arch, scale, K, T):
     ref = ospec.speculative_generate(otgt, odrf, prompt[0], n_new, K, T, lambda it: synth.gen_uniforms(23, 0, it, 2 * K + 1),
                                      160, keep_trace=True)
     eng = engine.Engine(tgt, drf, 1, 160, K, T, 128)
-    synced, n = gu.lockstep(eng, synth, prompt[0], ref["iterations"], K, 23, ref["trace"])
+    synced, n = gu.lockstep(eng, synth, prompt[0], ref["iterations"], K, 23, ref["trace"],
+                            peaky=bool(arch.dtype) and scale > 1.0)
     assert eng.tkv.status() == 0
     accepted = sum(t["a"] for t in ref["trace"])
     assert 0 < accepted < K * len(ref["trace"])          # both outcomes occur
