@@ -195,6 +195,33 @@ int verify_from_logits(const float *dev_logits, int batch, int K, int vocab, con
                        size_t scratch_bytes, void *stream);
 size_t verify_scratch_bytes(int batch, int K);
 
+/*
+ * verify_from_logits without any scratch argument, for callers that must not allocate device
+ * memory: code that runs inside someone else's memory plan (a serving runtime that hands out a
+ * fixed arena and forbids cudaMalloc after start-up), inside a region where an allocation would
+ * synchronise the device or fail (a latency-critical decode loop, a process whose memory is fully
+ * committed to weights and KV cache), or from a language binding that can pass pointers through
+ * but cannot own CUDA buffers.  The paper has no counterpart of this call; it is a packaging of the
+ * same tail for such callers.
+ *
+ * The statistics that the two tail kernels pass to each other are kept in a fixed array inside
+ * the library (SSD_NOALLOC_MAX_ROWS entries of 16 bytes = 64 KB, present on every GPU that loads
+ * the library, for the life of the process).  Inputs and outputs are still the caller's.
+ *   - batch * (K + 1) > SSD_NOALLOC_MAX_ROWS is refused with SSD_E_CAPACITY; nothing is launched.
+ *   - The call never calls cudaMalloc / cudaFree or any allocating routine.
+ *   - The first call on each device looks up the array's device address (a host-side query with
+ *     that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.  Each
+ *     call overwrites every entry it later reads, so stale contents are harmless; but two calls
+ *     whose kernels overlap on the GPU (different streams, no ordering) race on it.  Order them.
+ * Results are identical to verify_from_logits.
+ */
+enum { SSD_NOALLOC_MAX_ROWS = 4096 };
+int verify_from_logits_noalloc(const float *dev_logits, int batch, int K, int vocab, const int32_t *dev_rows,
+                               const float *dev_q, const float *dev_u, float temperature,
+                               int32_t *dev_n_accepted, int32_t *dev_next_token, int next_token_stride,
+                               float *dev_p_debug, void *stream);
+
 /* Attention of one layer alone, for long-context checks: q fp32 [batch, rows, d] (already
  * position-encoded) against the cache of `layer`; row j of sequence b sees positions
  * 0 .. len[b] + j.  Output fp32 [batch, rows, d]. */

@@ -37,7 +37,7 @@ class SsdArch(ctypes.Structure):
 EXPORTS = ["ssd_model_create", "ssd_model_share_prefix", "ssd_model_destroy", "ssd_kv_bytes",
            "ssd_workspace_bytes", "kv_init", "kv_destroy", "kv_prefill", "draft_step", "target_verify",
            "kv_commit", "kv_rollback", "spec_advance", "kv_lengths", "ssd_device_status",
-           "verify_from_logits", "verify_scratch_bytes", "attention_rows", "ssd_last_logits", "ssd_launch_count",
+           "verify_from_logits", "verify_from_logits_noalloc", "verify_scratch_bytes", "attention_rows", "ssd_last_logits", "ssd_launch_count",
            "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror"]
 
 
@@ -77,6 +77,7 @@ def load():
     L.kv_lengths.argtypes = [vp, vp, vp]
     L.ssd_device_status.argtypes = [vp, vp, vp]
     L.verify_from_logits.argtypes = [vp, i32, i32, i32, vp, vp, vp, f32, vp, vp, i32, vp, vp, sz, vp]
+    L.verify_from_logits_noalloc.argtypes = [vp, i32, i32, i32, vp, vp, vp, f32, vp, vp, i32, vp, vp]
     L.verify_scratch_bytes.argtypes = [i32, i32]
     L.verify_scratch_bytes.restype = sz
     L.attention_rows.argtypes = [vp, vp, i32, vp, i32, vp, vp, sz, vp]
@@ -259,6 +260,24 @@ def verify_from_logits(logits: torch.Tensor, K: int, rows: torch.Tensor, q: Opti
     _check(load().verify_from_logits(_p(logits), B, K, V, _p(rows), _p(q), _p(u), temperature, _p(n_accepted),
                                      _p(next_token), next_token_stride, _p(p_debug), _p(scratch), scratch.numel(),
                                      _stream()), "verify_from_logits")
+
+
+NOALLOC_MAX_ROWS = 4096
+
+
+def verify_from_logits_noalloc(logits: torch.Tensor, K: int, rows: torch.Tensor, q: Optional[torch.Tensor],
+                               u: torch.Tensor, temperature: float, n_accepted: torch.Tensor,
+                               next_token: torch.Tensor, next_token_stride: int,
+                               p_debug: Optional[torch.Tensor]) -> None:
+    """The tail of a verification on supplied logits, for callers that may not allocate on the device:
+    same arguments as verify_from_logits minus the scratch buffer (the library keeps a fixed 64 KB
+    array for it, shared by all calls on a device; at most NOALLOC_MAX_ROWS logits rows per call;
+    calls that overlap on the GPU must be ordered by the caller)."""
+    Bn, M, V = logits.shape
+    assert M == K + 1 and logits.is_contiguous() and logits.dtype == torch.float32
+    _check(load().verify_from_logits_noalloc(_p(logits), Bn, K, V, _p(rows), _p(q), _p(u), temperature,
+                                             _p(n_accepted), _p(next_token), next_token_stride, _p(p_debug),
+                                             _stream()), "verify_from_logits_noalloc")
 
 
 def attention_rows(model: Model, kv: KV, layer: int, q: torch.Tensor, rows: int, out: torch.Tensor,

@@ -754,6 +754,54 @@ int ssd_last_logits(const ssd_model *m, int batch, int rows_per_seq, const void 
     return SSD_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// verify_from_logits for callers that cannot allocate device memory.
+//
+// The row statistics (max, normaliser, argmax of every logits row) that the two tail kernels hand
+// to each other live in a fixed array inside the library image instead of a caller buffer.  The
+// array is part of every context that loads the library (64 KB per GPU, held until exit).
+static __device__ __align__(256) RowStat g_noalloc_stats[SSD_NOALLOC_MAX_ROWS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+RowStat *g_noalloc_ptr[kMaxDevices] = {nullptr};
+std::mutex g_noalloc_mu;
+
+// In host code `g_noalloc_stats` is only a handle for the runtime, not a device address: the real
+// address differs per device and has to be asked for with that device current.
+int noalloc_scratch(RowStat **out) {
+    int dev = -1;
+    CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SSD_E_CAPACITY;
+    std::lock_guard<std::mutex> lk(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_stats) != cudaSuccess || !p) return SSD_E_CUDA;
+        g_noalloc_ptr[dev] = (RowStat *)p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return SSD_OK;
+}
+}  // namespace
+
+int verify_from_logits_noalloc(const float *dev_logits, int batch, int K, int vocab, const int32_t *dev_rows,
+                               const float *dev_q, const float *dev_u, float temperature,
+                               int32_t *dev_n_accepted, int32_t *dev_next_token, int next_token_stride,
+                               float *dev_p_debug, void *stream) {
+    if (!dev_logits || !dev_rows || !dev_u || !dev_n_accepted || !dev_next_token) return SSD_E_ARG;
+    if (batch < 1 || K < 0 || K + 1 > kMaxRowsPerSeq || vocab < 1 || temperature < 0.f || next_token_stride < 1)
+        return SSD_E_ARG;
+    if (K > 0 && !dev_q) return SSD_E_ARG;
+    if ((long long)batch * (K + 1) > SSD_NOALLOC_MAX_ROWS) return SSD_E_CAPACITY;
+    RowStat *stats = nullptr;
+    int rc = noalloc_scratch(&stats);
+    if (rc) return rc;
+    // every entry a call reads is written earlier in the same call (row_stats_kernel fills
+    // stats[0 .. batch*(K+1)) before verify_kernel looks at them): nothing has to start at zero
+    return run_verify_tail(dev_logits, batch, K, vocab, dev_rows, dev_q, dev_u, temperature, dev_n_accepted,
+                           dev_next_token, next_token_stride, dev_p_debug, nullptr, stats, (cudaStream_t)stream);
+}
+
 uint64_t ssd_launch_count(void) { return g_launches.load(); }
 
 int ssd_gemm_profile(int enable) {
