@@ -75,14 +75,26 @@ enum { SSD_MAX_ROWS = 64,        /* rows (sequences x rows per sequence) of one 
 
 /*
  * Bind an architecture to caller-owned device tensors (order above, n_tensors = 2 + 12 L + 3).
- * Borrows the pointers, copies nothing.  Covered: head_dim <= 128 and a multiple of 8,
+ * Borrows the pointers; copies only the descriptor table into dev_desc (bf16 models; see
+ * ssd_model_desc_bytes; NULL / 0 for fp32 models).  Covered: head_dim <= 128 and a multiple of 8,
  * n_heads * head_dim == d_model, rotary_dim even and <= head_dim; bf16 models additionally need
  * d_model, d_ff >= 128 and multiples of 8, vocab >= 128 (rows are fetched by tensor-map copies
  * of 128 x 64 elements).  Anything else: SSD_E_SHAPE.
  * (The decoder the target and draft models run: Eq. 1; block families named in Section
  * "Solution" / "Experiments": GPT-2, Dolly V2 = GPT-NeoX, Llama-2.)
  */
-int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n_tensors, ssd_model **out);
+int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n_tensors, void *dev_desc,
+                     size_t desc_bytes, ssd_model **out);
+
+/* Bytes of the caller-owned device block a bf16 model needs for its descriptor table (tensor maps
+ * of the matrices and pointers to the vectors, which the forward kernel walks on the device); 0 for
+ * fp32 models.  Pass a 256-byte aligned block of at least this size to ssd_model_create, which
+ * fills it once with a synchronous copy; it must outlive the model and its layer-skip drafts. */
+size_t ssd_model_desc_bytes(const ssd_arch *arch);
+
+/* bf16 models run the whole forward as one cooperative kernel by default; 0 selects one launch per
+ * step instead (same results up to fp32 summation order; kept for comparison). */
+int ssd_set_persistent(int enable);
 
 /* A layer-skip draft: the first n_layers layers of `target` plus its final norm and LM head
  * (an early-exit style draft, cf. Section "Speculative Sampling").  Shares the target's tensors. */
@@ -233,6 +245,17 @@ int attention_rows(ssd_model *m, ssd_kv *kv, int layer, const float *dev_q, int 
  * must be those of that forward. */
 int ssd_last_logits(const ssd_model *m, int batch, int rows_per_seq, const void *dev_ws, size_t ws_bytes,
                     float *dev_out, void *stream);
+
+/* Profiling aid for the single-kernel forward, whose phases no external profiler can separate:
+ * when enabled, one CTA stamps the GPU's nanosecond timer at kernel start, after every grid
+ * barrier and at its end.  ssd_read_trace copies the stamps of the last forward that used this
+ * workspace (same batch / rows_per_seq) to the host; consecutive differences are phase durations
+ * in the order: set-up, embedding, then per layer [qkv(+MLP-in), attention, out-proj(+MLP-out),
+ * statistics] (parallel residual) or [qkv, attention, out-proj, statistics, MLP-in, MLP-out,
+ * statistics] (sequential), then the LM head.  Synchronises the stream.  Off by default. */
+int ssd_set_trace(int enable);
+int ssd_read_trace(const ssd_model *m, int batch, int rows_per_seq, const void *dev_ws, size_t ws_bytes,
+                   uint64_t *host_out, int max_entries, int *n_out, void *stream);
 
 /* Number of kernels this library has launched in this process so far. */
 uint64_t ssd_launch_count(void);

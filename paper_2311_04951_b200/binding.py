@@ -34,10 +34,10 @@ class SsdArch(ctypes.Structure):
         ("rotary_base", ctypes.c_float), ("norm_eps", ctypes.c_float)]
 
 
-EXPORTS = ["ssd_model_create", "ssd_model_share_prefix", "ssd_model_destroy", "ssd_kv_bytes",
+EXPORTS = ["ssd_model_create", "ssd_model_desc_bytes", "ssd_set_persistent", "ssd_model_share_prefix", "ssd_model_destroy", "ssd_kv_bytes",
            "ssd_workspace_bytes", "kv_init", "kv_destroy", "kv_prefill", "draft_step", "target_verify",
            "kv_commit", "kv_rollback", "spec_advance", "kv_lengths", "ssd_device_status",
-           "verify_from_logits", "verify_from_logits_noalloc", "verify_scratch_bytes", "attention_rows", "ssd_last_logits", "ssd_launch_count",
+           "verify_from_logits", "verify_from_logits_noalloc", "verify_scratch_bytes", "attention_rows", "ssd_last_logits", "ssd_set_trace", "ssd_read_trace", "ssd_launch_count",
            "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror"]
 
 
@@ -57,7 +57,10 @@ def load():
     L = ctypes.CDLL(path)
     vp, i32, sz, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t, ctypes.c_float
     pp = ctypes.POINTER(ctypes.c_void_p)
-    L.ssd_model_create.argtypes = [ctypes.POINTER(SsdArch), pp, i32, pp]
+    L.ssd_model_create.argtypes = [ctypes.POINTER(SsdArch), pp, i32, vp, sz, pp]
+    L.ssd_model_desc_bytes.argtypes = [ctypes.POINTER(SsdArch)]
+    L.ssd_model_desc_bytes.restype = sz
+    L.ssd_set_persistent.argtypes = [i32]
     L.ssd_model_share_prefix.argtypes = [vp, i32, pp]
     L.ssd_model_destroy.argtypes = [vp]
     L.ssd_model_destroy.restype = None
@@ -82,6 +85,8 @@ def load():
     L.verify_scratch_bytes.restype = sz
     L.attention_rows.argtypes = [vp, vp, i32, vp, i32, vp, vp, sz, vp]
     L.ssd_last_logits.argtypes = [vp, i32, i32, vp, sz, vp, vp]
+    L.ssd_set_trace.argtypes = [i32]
+    L.ssd_read_trace.argtypes = [vp, i32, i32, vp, sz, vp, i32, ctypes.POINTER(ctypes.c_int), vp]
     L.ssd_launch_count.restype = ctypes.c_uint64
     L.ssd_gemm_profile.argtypes = [i32]
     L.ssd_gemm_profile_read.argtypes = [ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_double), i32]
@@ -140,7 +145,9 @@ class Model:
         ptrs = (ctypes.c_void_p * n)(*[None if t is None else t.data_ptr() for t in self.tensors])
         h = ctypes.c_void_p()
         a = arch_struct(arch)
-        _check(L.ssd_model_create(ctypes.byref(a), ptrs, n, ctypes.byref(h)), "ssd_model_create")
+        nd = int(L.ssd_model_desc_bytes(ctypes.byref(a)))
+        self.desc = torch.empty(max(nd, 1), dtype=torch.uint8, device="cuda") if nd else None
+        _check(L.ssd_model_create(ctypes.byref(a), ptrs, n, _p(self.desc), nd, ctypes.byref(h)), "ssd_model_create")
         self.h = h
 
     def share_prefix(self, n_layers: int) -> "Model":
@@ -291,6 +298,24 @@ def last_logits(model: Model, batch: int, rows_per_seq: int, ws: torch.Tensor) -
     _check(load().ssd_last_logits(model.h, batch, rows_per_seq, _p(ws), ws.numel(), _p(out), _stream()),
            "ssd_last_logits")
     return out
+
+
+def set_persistent(enable: bool) -> None:
+    _check(load().ssd_set_persistent(1 if enable else 0), "ssd_set_persistent")
+
+
+def set_trace(enable: bool) -> None:
+    _check(load().ssd_set_trace(1 if enable else 0), "ssd_set_trace")
+
+
+def read_trace(model: Model, batch: int, rows_per_seq: int, ws: torch.Tensor) -> np.ndarray:
+    """Nanosecond stamps of the last single-kernel forward on this workspace (start, after every
+    grid barrier, end)."""
+    out = np.zeros(1024, np.uint64)
+    n = ctypes.c_int()
+    _check(load().ssd_read_trace(model.h, batch, rows_per_seq, _p(ws), ws.numel(), out.ctypes.data_as(ctypes.c_void_p),
+                                 1024, ctypes.byref(n), _stream()), "ssd_read_trace")
+    return out[:n.value]
 
 
 def launch_count() -> int:

@@ -15,6 +15,7 @@
 #include "attention.cuh"
 #include "common.cuh"
 #include "gemm.cuh"
+#include "persistent.cuh"
 #include "rowops.cuh"
 #include "tail.cuh"
 
@@ -28,6 +29,8 @@ bool g_attr_done = false;
 std::mutex g_mu;
 
 // ---- optional per-launch timing of the weight-streaming GEMM ----
+bool g_persistent = true;  // bf16 models: whole forward in one cooperative kernel
+bool g_trace = false;       // stamp the global timer after every grid barrier of the forward kernel
 bool g_prof = false;
 std::vector<cudaEvent_t> g_prof_events;  // pairs
 size_t g_prof_used = 0;
@@ -134,6 +137,7 @@ struct ssd_model {
     std::vector<const void *> w;  // 2 + 12 L + 3 tensors
     std::vector<CUtensorMap> tm;  // bf16 models: per layer {qkv, o, in, out}, then lm head
     int d_in;
+    const ModelDesc *dev_desc;    // bf16 models: the same maps + vector pointers in device memory (caller-owned)
 };
 
 struct ssd_kv {
@@ -195,15 +199,24 @@ struct Workspace {
     Operand xn1, xn2, ao, act;
     float *part_m, *part_l, *part_o;
     int max_split;
+    // persistent kernel
+    float *ao_f32;
+    float2 *row_stats;  // [2L+1][R] (mean, rstd)
+    unsigned *sync;  // [0] grid barrier counter, [16..] attention tickets
+    size_t sync_bytes;
+    unsigned long long *trace;  // [kTraceSlots] phase time stamps (debug)
+    int rows_k;      // rows the persistent kernel's tiles span (padded)
     size_t bytes;
 };
 
 constexpr int kMaxSplit = 32;
+constexpr int kTraceSlots = 1024;
 
 // Carve (or just size, base == nullptr) the workspace for B sequences x M rows.
 Workspace carve(const ssd_model *m, int B, int M, uint8_t *base) {
     const ssd_arch &a = m->a;
     const int R = B * M, Rp = (R + 7) / 8 * 8, d = a.d_model, F = a.d_ff;
+    const int Rk = Rp <= 40 ? Rp : 64;  // kernel instantiations exist for 8..40 and 64 rows
     size_t off = 0;
     auto take = [&](size_t bytes) -> uint8_t * {
         uint8_t *p = base ? base + off : nullptr;
@@ -220,10 +233,16 @@ Workspace carve(const ssd_model *m, int B, int M, uint8_t *base) {
     w.ri.rope_cos = (float *)take(sizeof(float) * (size_t)R * (half ? half : 1));
     w.ri.rope_sin = (float *)take(sizeof(float) * (size_t)R * (half ? half : 1));
     w.n_rows_tmp = (int32_t *)take(sizeof(int32_t) * B);
-    w.x = (float *)take(sizeof(float) * (size_t)R * d);
+    w.rows_k = Rk;
+    w.x = (float *)take(sizeof(float) * (size_t)Rk * d);
     w.qkv = (float *)take(sizeof(float) * (size_t)R * 3 * d);
     w.qrot = (float *)take(sizeof(float) * (size_t)R * d);
-    w.t_in = (float *)take(sizeof(float) * (size_t)R * m->d_in);
+    w.t_in = (float *)take(sizeof(float) * (size_t)Rk * m->d_in);
+    w.ao_f32 = (float *)take(sizeof(float) * (size_t)Rk * d);
+    w.row_stats = (float2 *)take(sizeof(float2) * (size_t)(2 * a.n_layers + 1) * R);
+    w.sync_bytes = sizeof(unsigned) * (16 + (size_t)B * a.n_heads);
+    w.sync = (unsigned *)take(w.sync_bytes);
+    w.trace = (unsigned long long *)take(sizeof(unsigned long long) * kTraceSlots);
     w.logits = (float *)take(sizeof(float) * (size_t)R * a.vocab);
     w.stats = (RowStat *)take(sizeof(RowStat) * R);
     auto operand = [&](int ld, bool needed) {
@@ -379,11 +398,92 @@ int run_attention(const ssd_model *m, ssd_kv *kv, int layer, const float *q, int
     return SSD_OK;
 }
 
+inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 4 : 7) * a.n_layers; }
+
+template <int NT, int MR>
+int launch_forward_nt(FwdParams p, cudaStream_t st) {
+    const int stage = kWTileBytes + (p.swiglu ? 2 : 1) * NT * 8 * kTileK * 4;
+    const size_t attn = align_up((size_t)MR * (p.Dh + kAttnTile + 3) * 4 + 2 * (size_t)kAttnTile * (p.Dh + 8) * 2, 128);
+    const size_t tail_fixed = 24 * 12 + 16 + sizeof(Shared) + 16 * sizeof(double) + 256;
+    int S = (int)(((size_t)kSmemBudget - 1024 - attn - tail_fixed) / stage);
+    if (S > 12) S = 12;
+    if (S < 2) return SSD_E_CAPACITY;
+    p.stages = S;
+    p.attn_smem_off = (int)align_up((size_t)S * stage + 24 * (size_t)S + 16 + sizeof(Shared) + 16 * sizeof(double), 128);
+    const size_t smem = 1024 + (size_t)p.attn_smem_off + attn;
+    static bool attr = false;
+    if (!attr) {
+        if (cudaFuncSetAttribute(forward_kernel<NT, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) !=
+            cudaSuccess)
+            return SSD_E_CUDA;
+        attr = true;
+    }
+    void *args[] = {&p};
+    if (cudaLaunchCooperativeKernel((void *)forward_kernel<NT, MR>, dim3(g_num_sms), dim3(kPersistThreads), args, smem,
+                                    st) != cudaSuccess)
+        return SSD_E_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return SSD_OK;
+}
+
+template <int MR>
+int launch_forward_mr(const FwdParams &p, int rows_k, cudaStream_t st) {
+    switch (rows_k / 8) {
+        case 1: if (MR == 8) return launch_forward_nt<1, 8>(p, st); break;
+        case 2: if (MR <= 16) return launch_forward_nt<2, MR <= 16 ? MR : 8>(p, st); break;
+        case 3: return launch_forward_nt<3, MR>(p, st);
+        case 4: return launch_forward_nt<4, MR>(p, st);
+        case 5: return launch_forward_nt<5, MR>(p, st);
+        case 8: return launch_forward_nt<8, MR>(p, st);
+        default: break;
+    }
+    return SSD_E_CAPACITY;
+}
+
+// The whole forward as one cooperative launch (bf16 models).
+int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int M, const int32_t *n_rows,
+                       bool want_logits, const Workspace &w, cudaStream_t st) {
+    const ssd_arch &a = m->a;
+    FwdParams p;
+    memset(&p, 0, sizeof(p));
+    const int R = kv->B * M, Rk = w.rows_k;
+    p.md = m->dev_desc;
+    p.n_layers = a.n_layers; p.d = a.d_model; p.H = a.n_heads; p.Dh = a.head_dim; p.F = a.d_ff; p.d_in = m->d_in;
+    p.V = a.vocab; p.norm_kind = a.norm; p.swiglu = a.act == 1; p.parallel = a.parallel_residual;
+    p.rotary_dim = a.pos == 1 ? a.rotary_dim : 0; p.learned_pos = a.pos == 0; p.is_bf16_emb = 1;
+    p.eps = a.norm_eps; p.rotary_base = a.rotary_base; p.attn_scale = 1.0f / sqrtf((float)a.head_dim);
+    p.B = kv->B; p.M = M; p.R = R;
+    p.tokens = tokens; p.tok_stride = tok_stride; p.n_rows = n_rows;
+    p.tok_emb = m->w[T_TOK]; p.pos_emb = m->w[T_POS];
+    p.pos_limit = a.pos == 0 ? a.max_pos : 0;
+    p.cache = kv->cache; p.layer_bytes = kv->layer_bytes; p.len = kv->len; p.S = kv->S; p.status = kv->status;
+    p.ri = w.ri;
+    p.x = w.x; p.qkv = w.qkv; p.t_in = w.t_in; p.ao = w.ao_f32; p.logits = w.logits;
+    p.stats = w.row_stats;
+    p.part_m = w.part_m; p.part_l = w.part_l; p.part_o = w.part_o;
+    p.gbar = w.sync; p.tickets = w.sync + 16;
+    int ctx = kv->len_ub + M;
+    if (ctx > kv->S) ctx = kv->S;
+    plan_split(kv->B, a.n_heads, ctx, &p.chunk, &p.n_split);
+    p.want_logits = want_logits ? 1 : 0;
+    p.trace = (g_trace && 2 + barriers_needed(a) + 3 < kTraceSlots) ? w.trace : nullptr;
+    CUDA_OK(cudaMemsetAsync(w.sync, 0, w.sync_bytes, st));
+    int rc;
+    if (M <= 8) rc = launch_forward_mr<8>(p, Rk, st);
+    else if (M <= 16) rc = launch_forward_mr<16>(p, Rk, st);
+    else rc = launch_forward_mr<32>(p, Rk, st);
+    if (rc) return rc;
+    kv->last_rows = M;
+    return SSD_OK;
+}
+
 // One decoder forward over B x M rows against the cache.  Appends (does not commit) the rows'
 // keys/values; leaves logits in w.logits when want_logits.
 int forward(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int M, const int32_t *n_rows,
             bool want_logits, const Workspace &w, cudaStream_t st) {
     const ssd_arch &a = m->a;
+    if (a.dtype == 1 && g_persistent && m->dev_desc)
+        return forward_persistent(m, kv, tokens, tok_stride, M, n_rows, want_logits, w, st);
     const int B = kv->B, R = B * M, d = a.d_model, F = a.d_ff;
     GemmCall gc{m, st, R, (R + 7) / 8 * 8};
     int rc = run_setup(m, kv, M, n_rows, w, st);
@@ -484,8 +584,16 @@ int check_ws(const ssd_model *m, int B, int M, void *ws, size_t ws_bytes, Worksp
 // ------------------------------------------------------------------------------------------
 extern "C" {
 
-int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n_tensors, ssd_model **out) {
+size_t ssd_model_desc_bytes(const ssd_arch *arch) {
+    if (!arch || arch->n_layers < 1 || arch->dtype != 1) return 0;
+    return sizeof(ModelDesc) + sizeof(LayerDesc) * (size_t)arch->n_layers;
+}
+
+int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n_tensors, void *dev_desc,
+                     size_t desc_bytes, ssd_model **out) {
     if (!arch || !dev_weights || !out) return SSD_E_ARG;
+    if (arch->dtype == 1 && (!dev_desc || desc_bytes < ssd_model_desc_bytes(arch) || ((uintptr_t)dev_desc & 255)))
+        return SSD_E_ARG;
     int rc = check_arch(*arch);
     if (rc) return rc;
     if (n_tensors != 2 + PER_LAYER * arch->n_layers + 3) return SSD_E_ARG;
@@ -510,7 +618,34 @@ int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n
         delete m;
         return rc;
     }
+    m->dev_desc = nullptr;
+    if (arch->dtype == 1) {
+        // the tensor maps and vector pointers the persistent kernel walks, copied once to the caller's block
+        std::vector<uint8_t> host(ssd_model_desc_bytes(arch), 0);
+        ModelDesc *md = reinterpret_cast<ModelDesc *>(host.data());
+        md->tm_lm = m->tm[(size_t)4 * arch->n_layers];
+        md->lnf_g = (const float *)fw(m, 0);
+        md->lnf_b = (const float *)fw(m, 1);
+        LayerDesc *ld = reinterpret_cast<LayerDesc *>(md + 1);
+        for (int l = 0; l < arch->n_layers; ++l) {
+            for (int k = 0; k < 4; ++k) ld[l].tm[k] = m->tm[4 * l + k];
+            ld[l].ln1_g = (const float *)lw(m, l, L_LN1G); ld[l].ln1_b = (const float *)lw(m, l, L_LN1B);
+            ld[l].b_qkv = (const float *)lw(m, l, L_BQKV); ld[l].b_o = (const float *)lw(m, l, L_BO);
+            ld[l].ln2_g = (const float *)lw(m, l, L_LN2G); ld[l].ln2_b = (const float *)lw(m, l, L_LN2B);
+            ld[l].b_in = (const float *)lw(m, l, L_BIN); ld[l].b_out = (const float *)lw(m, l, L_BOUT);
+        }
+        if (cudaMemcpy(dev_desc, host.data(), host.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+            delete m;
+            return SSD_E_CUDA;
+        }
+        m->dev_desc = reinterpret_cast<const ModelDesc *>(dev_desc);
+    }
     *out = m;
+    return SSD_OK;
+}
+
+int ssd_set_persistent(int enable) {
+    g_persistent = enable != 0;
     return SSD_OK;
 }
 
@@ -521,6 +656,7 @@ int ssd_model_share_prefix(const ssd_model *target, int n_layers, ssd_model **dr
     m->a = target->a;
     m->a.n_layers = n_layers;
     m->d_in = target->d_in;
+    m->dev_desc = target->dev_desc;  // LM head first, then the layers: a prefix of the layers is a prefix of the block
     m->w.assign(target->w.begin(), target->w.begin() + T_L0 + PER_LAYER * n_layers);
     m->w.insert(m->w.end(), target->w.end() - 3, target->w.end());
     if (!target->tm.empty()) {
@@ -803,6 +939,27 @@ int verify_from_logits_noalloc(const float *dev_logits, int batch, int K, int vo
 }
 
 uint64_t ssd_launch_count(void) { return g_launches.load(); }
+
+int ssd_set_trace(int enable) {
+    g_trace = enable != 0;
+    return SSD_OK;
+}
+
+int ssd_read_trace(const ssd_model *m, int batch, int rows_per_seq, const void *dev_ws, size_t ws_bytes,
+                   uint64_t *host_out, int max_entries, int *n_out, void *stream) {
+    if (!m || !host_out || !n_out || max_entries < 1) return SSD_E_ARG;
+    Workspace w;
+    int rc = check_ws(m, batch, rows_per_seq, const_cast<void *>(dev_ws), ws_bytes, &w);
+    if (rc) return rc;
+    std::vector<unsigned long long> tmp(kTraceSlots);
+    CUDA_OK(cudaMemcpyAsync(tmp.data(), w.trace, sizeof(unsigned long long) * kTraceSlots, cudaMemcpyDeviceToHost,
+                            (cudaStream_t)stream));
+    CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+    int n = 0;
+    while (n < kTraceSlots && n < max_entries && tmp[n] != 0) { host_out[n] = tmp[n]; ++n; }
+    *n_out = n;
+    return SSD_OK;
+}
 
 int ssd_gemm_profile(int enable) {
     g_prof = enable != 0;

@@ -131,3 +131,32 @@ def test_capacity_and_argument_errors():
     with pytest.raises(B.SsdError) as e:
         B.Model(bad, B.upload_weights(arch, synth.gen_weights(arch, 1)))
     assert e.value.code == -2
+
+
+@pytest.mark.parametrize("name", ["neox_bf16", "llama_bf16", "gpt2_bf16", "neox_bf16_h80"])
+def test_single_kernel_forward_equals_stepwise_forward(name):
+    """The whole-forward cooperative kernel and the one-launch-per-step path compute the same
+    logits and cache rows (same arithmetic; only the fp32 reduction order differs)."""
+    arch = ARCHS[name]
+    ws_np = gu.scaled_weights(synth, arch, 3, 6.0)
+    model = B.Model(arch, B.upload_weights(arch, ws_np))
+    Bn, S, K = 2, 64, 4
+    prompts = synth.gen_prompt(4, Bn, 20, arch.vocab)
+    rows = synth.gen_prompt(5, Bn, K + 1, arch.vocab)
+    res = []
+    for persistent in (True, False):
+        B.set_persistent(persistent)
+        try:
+            kv = B.KV(model, Bn, S)
+            ws = model.new_workspace(Bn, 8, S)
+            B.kv_prefill(model, kv, torch.from_numpy(prompts).to("cuda"),
+                         torch.tensor([20, 13], dtype=torch.int32, device="cuda"), ws)
+            lg = gpu_logits(model, kv, ws, rows, K)
+            assert kv.status() == 0
+            res.append((lg, kv.cache_view().float().cpu().numpy()))
+        finally:
+            B.set_persistent(True)
+    assert np.abs(res[0][0] - res[1][0]).max() < 1e-2
+    for b, n in enumerate((20 + K + 1, 13 + K + 1)):
+        a, c = res[0][1][:, b, :, :, :n], res[1][1][:, b, :, :, :n]
+        assert (np.abs(a - c) <= gu.LOGIT_RTOL * np.abs(c) + gu.LOGIT_ATOL).all()
