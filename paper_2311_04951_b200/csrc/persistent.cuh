@@ -1,7 +1,7 @@
 // The whole decoder forward of a verification pass (or a draft step) as ONE persistent
 // cooperative kernel, one CTA per SM.
 //
-// Why: a pass is a chain of ~7 small dependent steps per layer; as separate launches the HBM
+// Why: a pass is a chain of ~8 small dependent steps per layer; as separate launches the HBM
 // stream stops at every boundary (the paper's point in Section "Autoregressive vs Speculative
 // Sampling" is that the pass is memory-bound, so idle HBM time is the cost).  Here the weight
 // stream never stops: a producer thread per CTA walks the static schedule of every weight tile
@@ -9,17 +9,15 @@
 // copies, running ahead across phase boundaries; only the small activation tiles wait for the
 // grid barrier of the phase that produces them.
 //
-// Roles in a CTA (384 threads):
+// Roles in a CTA (288 threads):
 //   warps 0-7   consumers: bf16 tensor-core MMAs on (weight tile, activation tile) stages,
 //               fp32 reductions of partial tiles into the output (bias added by the unit that
-//               holds k-chunk 0)
-//   warps 8-10  transform: fetch the fp32 activation slice of a stage from L2 (cp.async, a few
-//               stages ahead) and turn it, in place in shared memory, into the bf16 hi/lo pair
-//               the MMAs read -- applying LayerNorm/RMSNorm (row statistics from the previous
-//               phase), GELU / SwiGLU, or nothing
-//   warp 11     producer: TMA issue for the weight tiles, free-running across phases
-// Warps 0-10 also execute the non-GEMM phases (row set-up, embedding, row statistics,
-// attention with rotary + KV append + split merge) and the grid barriers.
+//               holds k-chunk 0); between GEMM phases the same warps run the small phases
+//               (row set-up, embedding, norm, activation, attention with rotary + KV append +
+//               split merge), which leave every GEMM operand in global memory already split
+//               into bf16 hi + lo, and the grid barriers
+//   warp 8      producer: TMA issue for weight tiles (free-running) and operand tiles (gated
+//               by the grid barrier of the phase that wrote them)
 // Every wait (mbarrier, grid barrier) is bounded; on time-out SSD_E_TIMEOUT is recorded, the CTA
 // stops taking work, waits (bounded) for its copies in flight and returns.
 #pragma once
@@ -33,10 +31,7 @@
 namespace ssd {
 
 constexpr int kConsumerWarps = 8;
-constexpr int kTransformWarps = 3;  // 8 + 3 + 1 = 12 warps: three per SM partition, 168 registers each
-constexpr int kXThreads = kTransformWarps * 32;
-constexpr int kXAheadMax = 8;  // activation slices in flight per CTA (bounded by the ring depth)
-constexpr int kWorkThreads = (kConsumerWarps + kTransformWarps) * 32;  // 352: everyone but the producer
+constexpr int kWorkThreads = kConsumerWarps * 32;  // 256: everyone but the producer
 constexpr int kPersistThreads = kWorkThreads + 32;
 constexpr int kAttnThreadsP = 256;
 
@@ -54,9 +49,15 @@ __device__ __forceinline__ const LayerDesc *layer_desc(const ModelDesc *md, int 
     return reinterpret_cast<const LayerDesc *>(md + 1) + l;
 }
 
-enum { XF_IDENT = 0, XF_NORM = 1, XF_GELU = 2, XF_SWIGLU = 3 };
+enum { OP_XN1 = 0, OP_XN2 = 1, OP_AO = 2, OP_ACT = 3 };
 
 struct alignas(64) FwdParams {
+    // GEMM operands in global memory, bf16 hi rows [0, rk) then lo rows [rk, 2 rk), row pitch = K:
+    // normalised rows (two sets for parallel-residual blocks), attention output, MLP activation.
+    CUtensorMap tm_op[4];  // box 64 x (2 rk), 128-byte swizzle
+    __nv_bfloat16 *op[4];
+    int op_ld[4];
+    int rk;
     const ModelDesc *md;
     // architecture
     int n_layers, d, H, Dh, F, d_in, V, norm_kind, swiglu, parallel, rotary_dim, learned_pos, is_bf16_emb;
@@ -76,8 +77,7 @@ struct alignas(64) FwdParams {
     int32_t *status;
     // workspace
     RowInfo ri;
-    float *x, *qkv, *t_in, *ao, *logits;
-    float2 *stats;  // [slot][R] (mean, rstd)
+    float *x, *qkv, *t_in, *logits;
     float *part_m, *part_l, *part_o;
     unsigned *tickets;  // [B*H]
     unsigned *gbar;     // grid barrier counter (zeroed before launch)
@@ -88,48 +88,45 @@ struct alignas(64) FwdParams {
 };
 
 struct GemmDesc {
-    const CUtensorMap *tmW;
-    const float *srcA;  // fp32 activations [R, lda]; SwiGLU reads a second slice at column colB
-    int lda, colB;
+    const CUtensorMap *tmW, *tmX;
     int N, Kd, n_tiles, kchunks;
-    int xf, need;    // transform kind; grid barriers that must have completed before its activations exist
+    int need;  // grid barriers that must have completed before its operand exists
     float *out;
     int ldo;
-    const float *bias, *g, *b;
-    int stat_slot;
+    const float *bias;
 };
 
 __device__ __forceinline__ int n_gemms(const FwdParams &p) { return 4 * p.n_layers + (p.want_logits ? 1 : 0); }
-__device__ __forceinline__ int barriers_per_layer(const FwdParams &p) { return p.parallel ? 4 : 7; }
+__device__ __forceinline__ int barriers_per_layer(const FwdParams &p) { return p.parallel ? 4 : 8; }
 
 // GEMM number gi in execution order.  sequential: qkv, o, in, out; parallel: qkv, in, o, out.
+// Barrier count before layer l: 2 (set-up; embedding + first norm) + barriers_per_layer * l.
+//   sequential layer: qkv | attention | o | norm2 | in | act | out | next norm   (8 barriers)
+//   parallel layer:   qkv, in | attention + act | o, out | next norms            (4 barriers)
 __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi) {
     GemmDesc g;
     const int l = gi >> 2, e = gi & 3;
     const int base = 2 + barriers_per_layer(p) * l;
     if (l >= p.n_layers) {  // LM head
-        g.tmW = &p.md->tm_lm; g.srcA = p.x; g.lda = p.d; g.colB = 0;
-        g.N = p.V; g.Kd = p.d; g.xf = XF_NORM; g.need = base; g.out = p.logits; g.ldo = p.V;
-        g.bias = nullptr; g.g = p.md->lnf_g; g.b = p.md->lnf_b; g.stat_slot = 2 * p.n_layers;
+        g.tmW = &p.md->tm_lm; g.tmX = &p.tm_op[OP_XN1];
+        g.N = p.V; g.Kd = p.d; g.need = base; g.out = p.logits; g.ldo = p.V; g.bias = nullptr;
     } else {
         const LayerDesc *ld = layer_desc(p.md, l);
         int kind;  // 0 qkv, 1 o, 2 in, 3 out
         if (p.parallel) kind = (e == 0) ? 0 : (e == 1) ? 2 : (e == 2) ? 1 : 3;
         else kind = e;
-        g.tmW = &ld->tm[kind]; g.colB = 0; g.g = nullptr; g.b = nullptr; g.stat_slot = 0;
+        g.tmW = &ld->tm[kind];
         if (kind == 0) {
-            g.srcA = p.x; g.lda = p.d; g.N = 3 * p.d; g.Kd = p.d; g.xf = XF_NORM; g.need = base;
-            g.out = p.qkv; g.ldo = 3 * p.d; g.bias = ld->b_qkv; g.g = ld->ln1_g; g.b = ld->ln1_b; g.stat_slot = 2 * l;
+            g.tmX = &p.tm_op[OP_XN1]; g.N = 3 * p.d; g.Kd = p.d; g.need = base;
+            g.out = p.qkv; g.ldo = 3 * p.d; g.bias = ld->b_qkv;
         } else if (kind == 1) {
-            g.srcA = p.ao; g.lda = p.d; g.N = p.d; g.Kd = p.d; g.xf = XF_IDENT; g.need = base + 2;
+            g.tmX = &p.tm_op[OP_AO]; g.N = p.d; g.Kd = p.d; g.need = base + 2;
             g.out = p.x; g.ldo = p.d; g.bias = ld->b_o;
         } else if (kind == 2) {
-            g.srcA = p.x; g.lda = p.d; g.N = p.d_in; g.Kd = p.d; g.xf = XF_NORM; g.need = p.parallel ? base : base + 4;
-            g.out = p.t_in; g.ldo = p.d_in; g.bias = ld->b_in; g.g = ld->ln2_g; g.b = ld->ln2_b;
-            g.stat_slot = p.parallel ? 2 * l : 2 * l + 1;
+            g.tmX = &p.tm_op[p.parallel ? OP_XN2 : OP_XN1]; g.N = p.d_in; g.Kd = p.d; g.need = p.parallel ? base : base + 4;
+            g.out = p.t_in; g.ldo = p.d_in; g.bias = ld->b_in;
         } else {
-            g.srcA = p.t_in; g.lda = p.d_in; g.N = p.d; g.Kd = p.F; g.xf = p.swiglu ? XF_SWIGLU : XF_GELU; g.colB = p.F;
-            g.need = p.parallel ? base + 2 : base + 5;
+            g.tmX = &p.tm_op[OP_ACT]; g.N = p.d; g.Kd = p.F; g.need = p.parallel ? base + 2 : base + 6;
             g.out = p.x; g.ldo = p.d; g.bias = ld->b_out;
         }
     }
@@ -156,40 +153,26 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned *p) {
 __device__ __forceinline__ void red_release_add(unsigned *p, unsigned v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void cp_async16(void *dst, const void *src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-// wait until at most n (0..8) of this thread's most recent cp.async groups are pending
-__device__ __forceinline__ void cp_async_wait_dyn(int n) {
-    switch (n) {
-        case 0: cp_async_wait<0>(); break;
-        case 1: cp_async_wait<1>(); break;
-        case 2: cp_async_wait<2>(); break;
-        case 3: cp_async_wait<3>(); break;
-        case 4: cp_async_wait<4>(); break;
-        case 5: cp_async_wait<5>(); break;
-        case 6: cp_async_wait<6>(); break;
-        case 7: cp_async_wait<7>(); break;
-        default: cp_async_wait<8>(); break;
-    }
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// operand element (r, i) of a hi/lo buffer
+__device__ __forceinline__ void store_hilo(__nv_bfloat16 *buf, int rk, int ld, int r, int i, float v) {
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    buf[(size_t)r * ld + i] = h;
+    buf[(size_t)(rk + r) * ld + i] = __float2bfloat16_rn(v - __bfloat162float(h));
 }
 
 struct alignas(16) Shared {
     volatile int released;  // grid barriers completed so far
     volatile int abort;     // some wait in this CTA gave up
     volatile int go;        // snapshot of !abort taken inside the grid barrier: uniform for all work threads
-    volatile int abort_x;   // set by a transform warp only, read by both after their own barrier
-    float mean[kMaxRows], rstd[kMaxRows];
     int flag;
-    int pad[3];
 };
 
 // Grid barrier for the 320 work threads of every CTA.  Returns false (the same value in every work
 // thread of the CTA) once a wait has timed out anywhere in this CTA; the caller then stops.
 __device__ __forceinline__ bool grid_sync(const FwdParams &p, Shared *sh, int &epoch) {
+    fence_async_proxy();  // this thread's operand writes must be seen by other CTAs' TMA reads
     __threadfence();
     named_bar(1, kWorkThreads);
     ++epoch;
@@ -222,7 +205,7 @@ __device__ __forceinline__ bool grid_sync(const FwdParams &p, Shared *sh, int &e
     return sh->go != 0;
 }
 
-// ---- non-GEMM phases (320 work threads) -------------------------------------------------------
+// ---- non-GEMM phases (256 work threads) -------------------------------------------------------
 
 __device__ __forceinline__ float block_sum_work(float v, float *red) {
     v = warp_sum(v);
@@ -232,7 +215,7 @@ __device__ __forceinline__ float block_sum_work(float v, float *red) {
     named_bar(2, kWorkThreads);
     float t = 0.f;
 #pragma unroll
-    for (int i = 0; i < kConsumerWarps + kTransformWarps; ++i) t += red[i];
+    for (int i = 0; i < kConsumerWarps; ++i) t += red[i];
     return t;
 }
 __device__ __forceinline__ double block_sum_work(double v, double *red) {
@@ -243,7 +226,7 @@ __device__ __forceinline__ double block_sum_work(double v, double *red) {
     named_bar(2, kWorkThreads);
     double t = 0.0;
 #pragma unroll
-    for (int i = 0; i < kConsumerWarps + kTransformWarps; ++i) t += red[i];
+    for (int i = 0; i < kConsumerWarps; ++i) t += red[i];
     return t;
 }
 
@@ -257,8 +240,10 @@ __device__ __forceinline__ void grid_zero(float *dst, int R, int n, int ld) {
     }
 }
 
-// (mean, rstd) of row r of x -> stats[slot][r]; one CTA per row
-__device__ __forceinline__ void row_stats_phase(const FwdParams &p, int slot, double *red) {
+// Norm of every row of x into hi/lo operand buffers (one or two gain/bias sets from the same
+// statistics); one CTA per row.
+__device__ __forceinline__ void norm_phase(const FwdParams &p, const float *g1, const float *b1, int op1,
+                                           const float *g2, const float *b2, int op2, double *red) {
     for (int r = blockIdx.x; r < p.R; r += gridDim.x) {
         const float *x = p.x + (size_t)r * p.d;
         double s1 = 0.0, s2 = 0.0;
@@ -277,7 +262,24 @@ __device__ __forceinline__ void row_stats_phase(const FwdParams &p, int slot, do
         } else {
             var = s2 / p.d;
         }
-        if (threadIdx.x == 0) p.stats[(size_t)slot * p.R + r] = make_float2((float)mean, (float)rsqrt(var + (double)p.eps));
+        const float mu = (float)mean, rs = (float)rsqrt(var + (double)p.eps);
+        for (int i = threadIdx.x; i < p.d; i += kWorkThreads) {
+            const float c = (__ldcg(x + i) - mu) * rs;
+            store_hilo(p.op[op1], p.rk, p.op_ld[op1], r, i, c * g1[i] + (b1 ? b1[i] : 0.f));
+            if (g2) store_hilo(p.op[op2], p.rk, p.op_ld[op2], r, i, c * g2[i] + (b2 ? b2[i] : 0.f));
+        }
+    }
+}
+
+// MLP activation of t_in into the hi/lo operand of the down projection, spread over the grid
+__device__ __forceinline__ void act_phase(const FwdParams &p) {
+    const long long total = (long long)p.R * p.F;
+    for (long long i = (long long)blockIdx.x * kWorkThreads + threadIdx.x; i < total;
+         i += (long long)gridDim.x * kWorkThreads) {
+        const int r = (int)(i / p.F), c = (int)(i % p.F);
+        const float *t = p.t_in + (size_t)r * p.d_in;
+        const float v = p.swiglu ? silu(__ldcg(t + c)) * __ldcg(t + p.F + c) : gelu_erf(__ldcg(t + c));
+        store_hilo(p.op[OP_ACT], p.rk, p.op_ld[OP_ACT], r, c, v);
     }
 }
 
@@ -519,7 +521,7 @@ __device__ void attention_item(const FwdParams &p, int layer, int item, uint8_t 
                         acc = fmaf(__ldcg(p.part_o + (base + s) * Dh + e), w, acc);
                     }
                 }
-                p.ao[(size_t)(r0 + m) * d + h * Dh + e] = L > 0.f ? acc / L : 0.f;
+                store_hilo(p.op[OP_AO], p.rk, p.op_ld[OP_AO], r0 + m, h * Dh + e, L > 0.f ? acc / L : 0.f);
             }
             if (tid == 0) p.tickets[bh] = 0;  // ready for the next layer (a grid barrier lies between)
         }
@@ -540,13 +542,13 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int kRp = NT * 8;
-    constexpr int kRawBytes = kRp * kTileK * 4;  // one fp32 activation slice == one hi/lo bf16 pair
-    const int kStageBytes = kWTileBytes + (p.swiglu ? 2 : 1) * kRawBytes;
+    constexpr int kXBytes = 2 * kRp * kTileK * 2;  // hi tile followed by lo tile
+    constexpr int kStageBytes = kWTileBytes + kXBytes;
     const int S = p.stages;
     uint8_t *ring = smem;
     uint8_t *attn_scratch = smem + p.attn_smem_off;
     uint64_t *fullW = (uint64_t *)(smem + (size_t)S * kStageBytes);
-    uint64_t *xrdy = fullW + S, *empty = xrdy + S;
+    uint64_t *fullX = fullW + S, *empty = fullX + S;
     Shared *sh = (Shared *)(((uintptr_t)(empty + S) + 15) & ~(uintptr_t)15);
     double *red = (double *)(sh + 1);
 
@@ -554,219 +556,160 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(&fullW[s], 1);
-            mbar_init(&xrdy[s], kTransformWarps);
+            mbar_init(&fullX[s], 1);
             mbar_init(&empty[s], kConsumerWarps);
         }
         sh->released = 0;
         sh->abort = 0;
         sh->go = 1;
-        sh->abort_x = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     const int NG = n_gemms(p);
 
-    if (warp == kConsumerWarps + kTransformWarps) {
-        // =============================== producer: weight tiles only ===============================
-        // Weights never change, so this stream does not wait for any phase: it runs as far ahead
-        // of the consumers as the ring allows, across grid barriers.
+    if (warp == kConsumerWarps) {
+        // =============================== producer ===============================
+        // Two cursors over the same unit sequence.  Weights never change, so their cursor runs as far
+        // ahead as the ring allows, across grid barriers; an operand tile is fetched once the phase
+        // that wrote it has been released.
         if (lane == 0) {
-            int issued = 0;
-            bool ok = true;
-            for (int gi = 0; gi < NG && ok; ++gi) {
-                const GemmDesc g = gemm_desc(p, gi);
-                int c0, c1;
-                unit_range(g, c0, c1);
-                int tile = c0 / g.kchunks, kc = c0 % g.kchunks;
-                for (int c = c0; c < c1; ++c, ++issued) {
-                    const int s = issued % S;
-                    if (sh->abort || (issued >= S && !mbar_wait(&empty[s], ((issued / S) - 1) & 1))) {
-                        set_status(p.status, kTimeoutCode);
-                        sh->abort = 1;
-                        ok = false;
-                        break;
+            int issuedW = 0, issuedX = 0;
+            int gw = 0, cw = 0, cw1 = 0, tw = 0, kw = 0;
+            int gx = 0, cx = 0, cx1 = 0, kx = 0;
+            GemmDesc dw, dx;
+            bool have_w = false, have_x = false;
+            auto next_w = [&]() {
+                for (; gw < NG; ++gw) {
+                    dw = gemm_desc(p, gw);
+                    unit_range(dw, cw, cw1);
+                    if (cw < cw1) { tw = cw / dw.kchunks; kw = cw % dw.kchunks; have_w = true; return; }
+                }
+                have_w = false;
+            };
+            auto next_x = [&]() {
+                for (; gx < NG; ++gx) {
+                    dx = gemm_desc(p, gx);
+                    unit_range(dx, cx, cx1);
+                    if (cx < cx1) { kx = cx % dx.kchunks; have_x = true; return; }
+                }
+                have_x = false;
+            };
+            next_w();
+            next_x();
+            int seen_release = 0;
+            long long idle_since = clock64();
+            while ((have_w || have_x) && !sh->abort) {
+                bool progressed = false;
+                if (have_w) {
+                    const int s = issuedW % S;
+                    if (issuedW < S || mbar_test_wait(&empty[s], ((issuedW / S) - 1) & 1)) {
+                        mbar_expect_tx(&fullW[s], kWTileBytes);
+                        tma_load_2d(ring + (size_t)s * kStageBytes, dw.tmW, kw * kTileK, tw * kTileN, &fullW[s]);
+                        ++issuedW;
+                        progressed = true;
+                        if (++kw == dw.kchunks) { kw = 0; ++tw; }
+                        if (++cw == cw1) { ++gw; next_w(); }
                     }
-                    mbar_expect_tx(&fullW[s], kWTileBytes);
-                    tma_load_2d(ring + (size_t)s * kStageBytes, g.tmW, kc * kTileK, tile * kTileN, &fullW[s]);
-                    if (++kc == g.kchunks) { kc = 0; ++tile; }
+                }
+                if (have_x && issuedX < issuedW) {
+                    if (dx.need > seen_release) {
+                        seen_release = sh->released;
+                        if (dx.need <= seen_release) fence_async_proxy();  // that phase's writes -> visible to TMA
+                    }
+                    if (dx.need <= seen_release) {
+                        const int s = issuedX % S;
+                        mbar_expect_tx(&fullX[s], kXBytes);
+                        tma_load_2d(ring + (size_t)s * kStageBytes + kWTileBytes, dx.tmX, kx * kTileK, 0, &fullX[s]);
+                        ++issuedX;
+                        progressed = true;
+                        if (++kx == dx.kchunks) kx = 0;
+                        if (++cx == cx1) { ++gx; next_x(); }
+                    }
+                }
+                if (progressed) {
+                    idle_since = clock64();
+                } else if (clock64() - idle_since > kWaitCycles) {
+                    set_status(p.status, kTimeoutCode);
+                    sh->abort = 1;
                 }
             }
             // error path only: wait (bounded) for copies still in flight before the CTA may exit
-            if (!ok)
-                for (int i = (issued > S ? issued - S : 0); i < issued; ++i) mbar_wait(&fullW[i % S], (i / S) & 1);
+            if (sh->abort) {
+                for (int i = (issuedW > S ? issuedW - S : 0); i < issuedW; ++i) mbar_wait(&fullW[i % S], (i / S) & 1);
+                for (int i = (issuedX > S ? issuedX - S : 0); i < issuedX; ++i) mbar_wait(&fullX[i % S], (i / S) & 1);
+            }
         }
     } else {
         // =============================== work warps ===============================
         int epoch = 0, it = 0;  // grid barriers passed; ring stages consumed
-        bool alive = true;
+        bool alive = true;      // per warp: false once one of its waits gave up
         float acc[NT][4];
 #pragma unroll
         for (int j = 0; j < NT; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
 
-        // run this CTA's units of GEMM gi (consumers: MMA; transform warps: operand preparation)
+        // run this CTA's units of GEMM gi
         auto run_gemm = [&](int gi) {
             const GemmDesc g = gemm_desc(p, gi);
             int c0, c1;
             unit_range(g, c0, c1);
             if (c0 >= c1) return;
-            const int n_units = c1 - c0;
-            if (warp >= kConsumerWarps) {
-                // ---------------- transform warps ----------------
-                const int tt = threadIdx.x - kConsumerWarps * 32;  // 0..95
-                const int kp = tt & 31, rw = tt >> 5;              // k pair; row = kTransformWarps * i + rw
-                constexpr int kRowsPer = (kRp + kTransformWarps - 1) / kTransformWarps;
-                constexpr int kChunksPer = (kRp * 16 + kXThreads - 1) / kXThreads;
-                const bool two = g.xf == XF_SWIGLU;
-                if (g.xf == XF_NORM) {
-                    for (int r = tt; r < p.R; r += kXThreads) {
-                        const float2 st = __ldcg(p.stats + (size_t)g.stat_slot * p.R + r);
-                        sh->mean[r] = st.x;
-                        sh->rstd[r] = st.y;
-                    }
+            int tile = c0 / g.kchunks, kc = c0 % g.kchunks;
+            auto flush = [&](int t, bool with_bias) {
+                const int n = t * kTileN + warp * 16 + (lane >> 2);
+                float b0 = 0.f, b1 = 0.f;
+                if (with_bias && g.bias) {
+                    if (n < g.N) b0 = __ldg(g.bias + n);
+                    if (n + 8 < g.N) b1 = __ldg(g.bias + n + 8);
                 }
-                // fetch of unit j's activation slice(s) into its ring slot (16-byte cp.async chunks)
-                const int it0 = it;  // ring stage of this GEMM's first unit
-                auto issue = [&](int j) {
-                    const int its = it0 + j, s = its % S;
-                    if (its >= S && !mbar_wait(&empty[s], ((its / S) - 1) & 1)) {
-                        set_status(p.status, kTimeoutCode);
-                        sh->abort = 1;
-                        sh->abort_x = 1;
-                    } else {
-                        uint8_t *xa = ring + (size_t)s * kStageBytes + kWTileBytes;
-                        const int k0 = ((c0 + j) % g.kchunks) * kTileK;
 #pragma unroll
-                        for (int q = 0; q < kChunksPer; ++q) {
-                            const int ch = tt + kXThreads * q, r = ch >> 4, c16 = ch & 15, k = k0 + c16 * 4;
-                            if (r < p.R && k < g.Kd) {
-                                const float *src = g.srcA + (size_t)r * g.lda + k;
-                                cp_async16(xa + r * 256 + c16 * 16, src);
-                                if (two) cp_async16(xa + kRawBytes + r * 256 + c16 * 16, src + g.colB);
-                            }
-                        }
+                for (int j = 0; j < NT; ++j) {
+                    const int m0 = 8 * j + (lane & 3) * 2;
+                    if (n < g.N) {
+                        if (m0 < p.R) atomicAdd(g.out + (size_t)m0 * g.ldo + n, acc[j][0] + b0);
+                        if (m0 + 1 < p.R) atomicAdd(g.out + (size_t)(m0 + 1) * g.ldo + n, acc[j][1] + b0);
                     }
-                    cp_async_commit();
-                };
-                // exactly `ahead` groups are committed before the loop and one per iteration, so that
-                // "at most `ahead` groups pending" means "slice j has landed" whatever n_units is
-                const int ahead = min(kXAheadMax, S - 2);
-                for (int j = 0; j < ahead; ++j) {
-                    if (j < n_units) issue(j); else cp_async_commit();
+                    if (n + 8 < g.N) {
+                        if (m0 < p.R) atomicAdd(g.out + (size_t)m0 * g.ldo + n + 8, acc[j][2] + b1);
+                        if (m0 + 1 < p.R) atomicAdd(g.out + (size_t)(m0 + 1) * g.ldo + n + 8, acc[j][3] + b1);
+                    }
+                    acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
                 }
-                int kc = c0 % g.kchunks;
-                for (int j = 0; j < n_units; ++j, ++it) {
-                    if (j + ahead < n_units) issue(j + ahead); else cp_async_commit();
-                    cp_async_wait_dyn(ahead);
-                    named_bar(4, kXThreads);  // every thread's chunks of slice j have landed
-                    if (sh->abort_x) { alive = false; break; }  // the same value in all transform warps here
-                    const int s = it % S;
-                    uint8_t *xa = ring + (size_t)s * kStageBytes + kWTileBytes;
-                    const float *ra = reinterpret_cast<const float *>(xa);
-                    const float *rb = reinterpret_cast<const float *>(xa + kRawBytes);
-                    float2 v[kRowsPer];
-                    const int k = kc * kTileK + 2 * kp;
-                    float2 gg = make_float2(1.f, 1.f), bb = make_float2(0.f, 0.f);
-                    if (g.xf == XF_NORM && k < g.Kd) {
-                        gg = __ldg(reinterpret_cast<const float2 *>(g.g + k));
-                        if (g.b) bb = __ldg(reinterpret_cast<const float2 *>(g.b + k));
-                    }
-#pragma unroll
-                    for (int i = 0; i < kRowsPer; ++i) {
-                        const int r = kTransformWarps * i + rw;
-                        float2 a = make_float2(0.f, 0.f);
-                        if (r < p.R && k < g.Kd) {  // rows / columns beyond the data were not fetched
-                            a = *reinterpret_cast<const float2 *>(ra + r * kTileK + 2 * kp);
-                            if (g.xf == XF_NORM) {
-                                const float mu = sh->mean[r], rs = sh->rstd[r];
-                                a.x = (a.x - mu) * rs * gg.x + bb.x;
-                                a.y = (a.y - mu) * rs * gg.y + bb.y;
-                            } else if (g.xf == XF_GELU) {
-                                a.x = gelu_erf(a.x);
-                                a.y = gelu_erf(a.y);
-                            } else if (g.xf == XF_SWIGLU) {
-                                const float2 u = *reinterpret_cast<const float2 *>(rb + r * kTileK + 2 * kp);
-                                a.x = silu(a.x) * u.x;
-                                a.y = silu(a.y) * u.y;
-                            }
-                        }
-                        v[i] = a;
-                    }
-                    named_bar(4, kXThreads);  // all raw values are in registers: overwrite in place
-#pragma unroll
-                    for (int i = 0; i < kRowsPer; ++i) {
-                        const int r = kTransformWarps * i + rw;
-                        if (r >= kRp) break;
-                        const __nv_bfloat162 hi = __floats2bfloat162_rn(v[i].x, v[i].y);
-                        const __nv_bfloat162 lo = __floats2bfloat162_rn(v[i].x - __low2float(hi), v[i].y - __high2float(hi));
-                        const uint32_t off = (uint32_t)r * 128u + ((uint32_t)((kp >> 2) ^ (r & 7)) << 4) + (uint32_t)(kp & 3) * 4u;
-                        *reinterpret_cast<__nv_bfloat162 *>(xa + off) = hi;
-                        *reinterpret_cast<__nv_bfloat162 *>(xa + kRp * 128 + off) = lo;
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&xrdy[s]);
-                    if (++kc == g.kchunks) kc = 0;
+            };
+            const int arow = lane & 15, achunk = lane >> 4, brow = lane & 7, bsel = lane >> 3;
+            bool has_k0 = (kc == 0);  // does the running tile segment include k-chunk 0 (it adds the bias)
+            for (int c = c0; c < c1 && alive; ++c, ++it) {
+                const int s = it % S;
+                if (!mbar_wait(&fullW[s], (it / S) & 1) || !mbar_wait(&fullX[s], (it / S) & 1)) {
+                    set_status(p.status, kTimeoutCode);
+                    sh->abort = 1;
+                    alive = false;
+                    break;
                 }
-                cp_async_wait<0>();
-            } else {
-                // ---------------- consumers ----------------
-                int tile = c0 / g.kchunks, kc = c0 % g.kchunks;
-                auto flush = [&](int t, bool with_bias) {
-                    const int n = t * kTileN + warp * 16 + (lane >> 2);
-                    float b0 = 0.f, b1 = 0.f;
-                    if (with_bias && g.bias) {
-                        if (n < g.N) b0 = __ldg(g.bias + n);
-                        if (n + 8 < g.N) b1 = __ldg(g.bias + n + 8);
-                    }
+                const uint32_t st = smem_u32(ring + (size_t)s * kStageBytes);
+                const uint32_t wbase = st + (uint32_t)(warp * 16 + arow) * 128u;
+                const uint32_t xbase = st + kWTileBytes + (bsel >= 2 ? kRp * 128 : 0) + (uint32_t)brow * 128u;
+#pragma unroll
+                for (int ks = 0; ks < kTileK / 16; ++ks) {
+                    uint32_t a0, a1, a2, a3;
+                    ldmatrix_x4(wbase + ((uint32_t)((2 * ks + achunk) ^ (arow & 7)) << 4), a0, a1, a2, a3);
 #pragma unroll
                     for (int j = 0; j < NT; ++j) {
-                        const int m0 = 8 * j + (lane & 3) * 2;
-                        if (n < g.N) {
-                            if (m0 < p.R) atomicAdd(g.out + (size_t)m0 * g.ldo + n, acc[j][0] + b0);
-                            if (m0 + 1 < p.R) atomicAdd(g.out + (size_t)(m0 + 1) * g.ldo + n, acc[j][1] + b0);
-                        }
-                        if (n + 8 < g.N) {
-                            if (m0 < p.R) atomicAdd(g.out + (size_t)m0 * g.ldo + n + 8, acc[j][2] + b1);
-                            if (m0 + 1 < p.R) atomicAdd(g.out + (size_t)(m0 + 1) * g.ldo + n + 8, acc[j][3] + b1);
-                        }
-                        acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
-                    }
-                };
-                const int arow = lane & 15, achunk = lane >> 4, brow = lane & 7, bsel = lane >> 3;
-                bool has_k0 = (kc == 0);  // does the running tile segment include k-chunk 0 (it adds the bias)
-                for (int c = c0; c < c1 && alive; ++c, ++it) {
-                    const int s = it % S;
-                    if (!mbar_wait(&fullW[s], (it / S) & 1) || !mbar_wait(&xrdy[s], (it / S) & 1)) {
-                        set_status(p.status, kTimeoutCode);
-                        sh->abort = 1;
-                        alive = false;
-                        break;
-                    }
-                    const uint32_t st = smem_u32(ring + (size_t)s * kStageBytes);
-                    const uint32_t wbase = st + (uint32_t)(warp * 16 + arow) * 128u;
-                    const uint32_t xbase = st + kWTileBytes + (bsel >= 2 ? kRp * 128 : 0) + (uint32_t)brow * 128u;
-#pragma unroll
-                    for (int ks = 0; ks < kTileK / 16; ++ks) {
-                        uint32_t a0, a1, a2, a3;
-                        ldmatrix_x4(wbase + ((uint32_t)((2 * ks + achunk) ^ (arow & 7)) << 4), a0, a1, a2, a3);
-#pragma unroll
-                        for (int j = 0; j < NT; ++j) {
-                            uint32_t h0, h1, l0, l1;
-                            ldmatrix_x4(xbase + (uint32_t)j * 1024u + ((uint32_t)((2 * ks + (bsel & 1)) ^ brow) << 4), h0, h1, l0, l1);
-                            mma_bf16(acc[j], a0, a1, a2, a3, h0, h1);
-                            mma_bf16(acc[j], a0, a1, a2, a3, l0, l1);
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&empty[s]);
-                    if (++kc == g.kchunks) {
-                        flush(tile, has_k0);
-                        kc = 0;
-                        ++tile;
-                        has_k0 = true;
+                        uint32_t h0, h1, l0, l1;
+                        ldmatrix_x4(xbase + (uint32_t)j * 1024u + ((uint32_t)((2 * ks + (bsel & 1)) ^ brow) << 4), h0, h1, l0, l1);
+                        mma_bf16(acc[j], a0, a1, a2, a3, h0, h1);
+                        mma_bf16(acc[j], a0, a1, a2, a3, l0, l1);
                     }
                 }
-                if (alive && kc != 0) flush(tile, has_k0);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty[s]);
+                if (++kc == g.kchunks) {
+                    flush(tile, has_k0);
+                    kc = 0;
+                    ++tile;
+                    has_k0 = true;
+                }
             }
+            if (alive && kc != 0) flush(tile, has_k0);
         };
 
         if (p.trace && blockIdx.x == 0 && threadIdx.x == 0) {
@@ -777,21 +720,32 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
         // ---- phase program (the same structure gemm_desc() encodes) ----
         // `go` is uniform over the work threads (taken inside the grid barrier), so every named barrier
         // below is reached by all of them or by none.
+        auto norm_for_layer = [&](int l) {  // operand(s) of layer l's first GEMM(s), or of the LM head
+            if (l < p.n_layers) {
+                const LayerDesc *ld = layer_desc(p.md, l);
+                if (p.parallel) norm_phase(p, ld->ln1_g, ld->ln1_b, OP_XN1, ld->ln2_g, ld->ln2_b, OP_XN2, red);
+                else norm_phase(p, ld->ln1_g, ld->ln1_b, OP_XN1, nullptr, nullptr, 0, red);
+                grid_zero(p.qkv, p.R, 3 * p.d, 3 * p.d);
+                if (p.parallel) grid_zero(p.t_in, p.R, p.d_in, p.d_in);
+            } else if (p.want_logits) {
+                norm_phase(p, p.md->lnf_g, p.md->lnf_b, OP_XN1, nullptr, nullptr, 0, red);
+                grid_zero(p.logits, p.R, p.V, p.V);
+            }
+        };
         setup_phase(p);
         bool go = grid_sync(p, sh, epoch);
         if (go) {
             embed_phase(p);
-            grid_zero(p.qkv, p.R, 3 * p.d, 3 * p.d);
-            if (p.parallel) grid_zero(p.t_in, p.R, p.d_in, p.d_in);
             named_bar(2, kWorkThreads);  // the embedding rows are read back by the CTA that wrote them
-            row_stats_phase(p, 0, red);
+            norm_for_layer(0);
             go = grid_sync(p, sh, epoch);
         }
         for (int l = 0; l < p.n_layers && go; ++l) {
             run_gemm(4 * l + 0);                       // qkv
-            if (p.parallel) run_gemm(4 * l + 1);       // MLP in (same input)
+            if (p.parallel) run_gemm(4 * l + 1);       // MLP in (same block input)
             if (!(go = grid_sync(p, sh, epoch))) break;
             attention_phase<MR>(p, l, attn_scratch, sh);
+            if (p.parallel) act_phase(p);
             if (!(go = grid_sync(p, sh, epoch))) break;
             if (p.parallel) {
                 run_gemm(4 * l + 2);                   // out-proj -> x
@@ -800,18 +754,18 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             } else {
                 run_gemm(4 * l + 1);                   // out-proj -> x
                 if (!(go = grid_sync(p, sh, epoch))) break;
-                row_stats_phase(p, 2 * l + 1, red);
+                const LayerDesc *ld = layer_desc(p.md, l);
+                norm_phase(p, ld->ln2_g, ld->ln2_b, OP_XN1, nullptr, nullptr, 0, red);
                 grid_zero(p.t_in, p.R, p.d_in, p.d_in);
                 if (!(go = grid_sync(p, sh, epoch))) break;
                 run_gemm(4 * l + 2);                   // MLP in
                 if (!(go = grid_sync(p, sh, epoch))) break;
+                act_phase(p);
+                if (!(go = grid_sync(p, sh, epoch))) break;
                 run_gemm(4 * l + 3);                   // MLP out -> x
                 if (!(go = grid_sync(p, sh, epoch))) break;
             }
-            row_stats_phase(p, 2 * (l + 1), red);
-            if (l + 1 < p.n_layers) grid_zero(p.qkv, p.R, 3 * p.d, 3 * p.d);
-            if (l + 1 < p.n_layers && p.parallel) grid_zero(p.t_in, p.R, p.d_in, p.d_in);
-            if (l + 1 == p.n_layers && p.want_logits) grid_zero(p.logits, p.R, p.V, p.V);
+            norm_for_layer(l + 1);
             if (!(go = grid_sync(p, sh, epoch))) break;
         }
         if (go && p.want_logits) run_gemm(4 * p.n_layers);

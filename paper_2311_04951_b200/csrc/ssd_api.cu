@@ -200,8 +200,6 @@ struct Workspace {
     float *part_m, *part_l, *part_o;
     int max_split;
     // persistent kernel
-    float *ao_f32;
-    float2 *row_stats;  // [2L+1][R] (mean, rstd)
     unsigned *sync;  // [0] grid barrier counter, [16..] attention tickets
     size_t sync_bytes;
     unsigned long long *trace;  // [kTraceSlots] phase time stamps (debug)
@@ -234,17 +232,17 @@ Workspace carve(const ssd_model *m, int B, int M, uint8_t *base) {
     w.ri.rope_sin = (float *)take(sizeof(float) * (size_t)R * (half ? half : 1));
     w.n_rows_tmp = (int32_t *)take(sizeof(int32_t) * B);
     w.rows_k = Rk;
-    w.x = (float *)take(sizeof(float) * (size_t)Rk * d);
+    w.x = (float *)take(sizeof(float) * (size_t)R * d);
     w.qkv = (float *)take(sizeof(float) * (size_t)R * 3 * d);
     w.qrot = (float *)take(sizeof(float) * (size_t)R * d);
-    w.t_in = (float *)take(sizeof(float) * (size_t)Rk * m->d_in);
-    w.ao_f32 = (float *)take(sizeof(float) * (size_t)Rk * d);
-    w.row_stats = (float2 *)take(sizeof(float2) * (size_t)(2 * a.n_layers + 1) * R);
+    w.t_in = (float *)take(sizeof(float) * (size_t)R * m->d_in);
     w.sync_bytes = sizeof(unsigned) * (16 + (size_t)B * a.n_heads);
     w.sync = (unsigned *)take(w.sync_bytes);
     w.trace = (unsigned long long *)take(sizeof(unsigned long long) * kTraceSlots);
     w.logits = (float *)take(sizeof(float) * (size_t)R * a.vocab);
     w.stats = (RowStat *)take(sizeof(RowStat) * R);
+    // GEMM operands: hi rows [0, rows) then lo rows [rows, 2 rows) in one buffer; the stepwise path
+    // pads rows to Rp, the single-kernel path to Rk (one allocation of 2 * Rk rows serves both)
     auto operand = [&](int ld, bool needed) {
         Operand o;
         o.f32 = nullptr; o.hi = nullptr; o.lo = nullptr; o.ld = ld;
@@ -252,8 +250,8 @@ Workspace carve(const ssd_model *m, int B, int M, uint8_t *base) {
         if (a.dtype == 0) {
             o.f32 = (float *)take(sizeof(float) * (size_t)Rp * ld);
         } else {
-            o.hi = (__nv_bfloat16 *)take(2 * (size_t)Rp * ld);
-            o.lo = (__nv_bfloat16 *)take(2 * (size_t)Rp * ld);
+            o.hi = (__nv_bfloat16 *)take(2 * (size_t)2 * Rk * ld);
+            o.lo = o.hi + (size_t)Rk * ld;
         }
         return o;
     };
@@ -398,11 +396,11 @@ int run_attention(const ssd_model *m, ssd_kv *kv, int layer, const float *q, int
     return SSD_OK;
 }
 
-inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 4 : 7) * a.n_layers; }
+inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 4 : 8) * a.n_layers; }
 
 template <int NT, int MR>
 int launch_forward_nt(FwdParams p, cudaStream_t st) {
-    const int stage = kWTileBytes + (p.swiglu ? 2 : 1) * NT * 8 * kTileK * 4;
+    constexpr int stage = kWTileBytes + 2 * NT * 8 * kTileK * 2;
     const size_t attn = align_up((size_t)MR * (p.Dh + kAttnTile + 3) * 4 + 2 * (size_t)kAttnTile * (p.Dh + 8) * 2, 128);
     const size_t tail_fixed = 24 * 12 + 16 + sizeof(Shared) + 16 * sizeof(double) + 256;
     int S = (int)(((size_t)kSmemBudget - 1024 - attn - tail_fixed) / stage);
@@ -447,6 +445,13 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     FwdParams p;
     memset(&p, 0, sizeof(p));
     const int R = kv->B * M, Rk = w.rows_k;
+    const Operand *ops[4] = {&w.xn1, &w.xn2, &w.ao, &w.act};
+    for (int i = 0; i < 4; ++i) {
+        p.op[i] = ops[i]->hi;
+        p.op_ld[i] = ops[i]->ld;
+        if (ops[i]->hi && make_map(&p.tm_op[i], ops[i]->hi, 2 * Rk, ops[i]->ld, 2 * Rk)) return SSD_E_CUDA;
+    }
+    p.rk = Rk;
     p.md = m->dev_desc;
     p.n_layers = a.n_layers; p.d = a.d_model; p.H = a.n_heads; p.Dh = a.head_dim; p.F = a.d_ff; p.d_in = m->d_in;
     p.V = a.vocab; p.norm_kind = a.norm; p.swiglu = a.act == 1; p.parallel = a.parallel_residual;
@@ -458,8 +463,7 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     p.pos_limit = a.pos == 0 ? a.max_pos : 0;
     p.cache = kv->cache; p.layer_bytes = kv->layer_bytes; p.len = kv->len; p.S = kv->S; p.status = kv->status;
     p.ri = w.ri;
-    p.x = w.x; p.qkv = w.qkv; p.t_in = w.t_in; p.ao = w.ao_f32; p.logits = w.logits;
-    p.stats = w.row_stats;
+    p.x = w.x; p.qkv = w.qkv; p.t_in = w.t_in; p.logits = w.logits;
     p.part_m = w.part_m; p.part_l = w.part_l; p.part_o = w.part_o;
     p.gbar = w.sync; p.tickets = w.sync + 16;
     int ctx = kv->len_ub + M;
