@@ -232,6 +232,14 @@ __device__ __forceinline__ double block_sum_work(double v, double *red) {
 
 // zero a [R, n] fp32 buffer (row pitch ld), spread over the whole grid
 __device__ __forceinline__ void grid_zero(float *dst, int R, int n, int ld) {
+    if (n == ld && ((R * (long long)n) & 3) == 0) {  // contiguous: 16-byte stores
+        const long long total4 = (long long)R * n / 4;
+        float4 *d4 = reinterpret_cast<float4 *>(dst);
+        for (long long i = (long long)blockIdx.x * kWorkThreads + threadIdx.x; i < total4;
+             i += (long long)gridDim.x * kWorkThreads)
+            d4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
     const long long total = (long long)R * n;
     for (long long i = (long long)blockIdx.x * kWorkThreads + threadIdx.x; i < total;
          i += (long long)gridDim.x * kWorkThreads) {
@@ -241,16 +249,31 @@ __device__ __forceinline__ void grid_zero(float *dst, int R, int n, int ld) {
 }
 
 // Norm of every row of x into hi/lo operand buffers (one or two gain/bias sets from the same
-// statistics); one CTA per row.
-__device__ __forceinline__ void norm_phase(const FwdParams &p, const float *g1, const float *b1, int op1,
+// statistics); one CTA per row.  The row (up to kNormRegs * 256 floats) stays in registers between
+// the statistics and the write pass, and all loads of a pass are issued before the first use, so
+// the phase costs about two L2 round trips instead of one per element.
+constexpr int kNormRegs = 8;  // float4 per thread: rows up to 8192 wide; wider rows are re-read
+__device__ __noinline__ void norm_phase(const FwdParams &p, const float *g1, const float *b1, int op1,
                                            const float *g2, const float *b2, int op2, double *red) {
+    const int n4 = p.d >> 2;  // d is a multiple of 8
     for (int r = blockIdx.x; r < p.R; r += gridDim.x) {
-        const float *x = p.x + (size_t)r * p.d;
+        const float4 *x4 = reinterpret_cast<const float4 *>(p.x + (size_t)r * p.d);
+        float4 xv[kNormRegs];
+#pragma unroll
+        for (int q = 0; q < kNormRegs; ++q) {
+            const int i = threadIdx.x + q * kWorkThreads;
+            xv[q] = i < n4 ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
         double s1 = 0.0, s2 = 0.0;
-        for (int i = threadIdx.x; i < p.d; i += kWorkThreads) {
-            const double v = __ldcg(x + i);
-            s1 += v;
-            s2 += v * v;
+#pragma unroll
+        for (int q = 0; q < kNormRegs; ++q) {
+            s1 += (double)xv[q].x + (double)xv[q].y + (double)xv[q].z + (double)xv[q].w;
+            s2 += (double)xv[q].x * xv[q].x + (double)xv[q].y * xv[q].y + (double)xv[q].z * xv[q].z + (double)xv[q].w * xv[q].w;
+        }
+        for (int i = threadIdx.x + kNormRegs * kWorkThreads; i < n4; i += kWorkThreads) {
+            const float4 v = __ldcg(x4 + i);
+            s1 += (double)v.x + (double)v.y + (double)v.z + (double)v.w;
+            s2 += (double)v.x * v.x + (double)v.y * v.y + (double)v.z * v.z + (double)v.w * v.w;
         }
         s1 = block_sum_work(s1, red);
         s2 = block_sum_work(s2, red);
@@ -263,27 +286,68 @@ __device__ __forceinline__ void norm_phase(const FwdParams &p, const float *g1, 
             var = s2 / p.d;
         }
         const float mu = (float)mean, rs = (float)rsqrt(var + (double)p.eps);
-        for (int i = threadIdx.x; i < p.d; i += kWorkThreads) {
-            const float c = (__ldcg(x + i) - mu) * rs;
-            store_hilo(p.op[op1], p.rk, p.op_ld[op1], r, i, c * g1[i] + (b1 ? b1[i] : 0.f));
-            if (g2) store_hilo(p.op[op2], p.rk, p.op_ld[op2], r, i, c * g2[i] + (b2 ? b2[i] : 0.f));
+        auto emit = [&](int i, const float4 v, const float *g, const float *b, int op) {
+            const float4 gg = __ldg(reinterpret_cast<const float4 *>(g) + i);
+            float4 bb = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (b) bb = __ldg(reinterpret_cast<const float4 *>(b) + i);
+            const float y0 = (v.x - mu) * rs * gg.x + bb.x, y1 = (v.y - mu) * rs * gg.y + bb.y;
+            const float y2 = (v.z - mu) * rs * gg.z + bb.z, y3 = (v.w - mu) * rs * gg.w + bb.w;
+            const __nv_bfloat162 h01 = __floats2bfloat162_rn(y0, y1), h23 = __floats2bfloat162_rn(y2, y3);
+            const __nv_bfloat162 l01 = __floats2bfloat162_rn(y0 - __low2float(h01), y1 - __high2float(h01));
+            const __nv_bfloat162 l23 = __floats2bfloat162_rn(y2 - __low2float(h23), y3 - __high2float(h23));
+            __nv_bfloat16 *hi = p.op[op] + (size_t)r * p.op_ld[op] + 4 * i;
+            __nv_bfloat16 *lo = p.op[op] + (size_t)(p.rk + r) * p.op_ld[op] + 4 * i;
+            uint2 hv, lv;
+            hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
+            lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
+            *reinterpret_cast<uint2 *>(hi) = hv;
+            *reinterpret_cast<uint2 *>(lo) = lv;
+        };
+#pragma unroll
+        for (int q = 0; q < kNormRegs; ++q) {
+            const int i = threadIdx.x + q * kWorkThreads;
+            if (i < n4) {
+                emit(i, xv[q], g1, b1, op1);
+                if (g2) emit(i, xv[q], g2, b2, op2);
+            }
+        }
+        for (int i = threadIdx.x + kNormRegs * kWorkThreads; i < n4; i += kWorkThreads) {
+            const float4 v = __ldcg(x4 + i);
+            emit(i, v, g1, b1, op1);
+            if (g2) emit(i, v, g2, b2, op2);
         }
     }
 }
 
 // MLP activation of t_in into the hi/lo operand of the down projection, spread over the grid
-__device__ __forceinline__ void act_phase(const FwdParams &p) {
-    const long long total = (long long)p.R * p.F;
+__device__ __noinline__ void act_phase(const FwdParams &p) {
+    const int f4 = p.F >> 2;
+    const long long total = (long long)p.R * f4;
     for (long long i = (long long)blockIdx.x * kWorkThreads + threadIdx.x; i < total;
          i += (long long)gridDim.x * kWorkThreads) {
-        const int r = (int)(i / p.F), c = (int)(i % p.F);
-        const float *t = p.t_in + (size_t)r * p.d_in;
-        const float v = p.swiglu ? silu(__ldcg(t + c)) * __ldcg(t + p.F + c) : gelu_erf(__ldcg(t + c));
-        store_hilo(p.op[OP_ACT], p.rk, p.op_ld[OP_ACT], r, c, v);
+        const int r = (int)(i / f4), c = (int)(i % f4);
+        const float4 *t = reinterpret_cast<const float4 *>(p.t_in + (size_t)r * p.d_in);
+        const float4 a = __ldcg(t + c);
+        float y0, y1, y2, y3;
+        if (p.swiglu) {
+            const float4 u = __ldcg(t + f4 + c);
+            y0 = silu(a.x) * u.x; y1 = silu(a.y) * u.y; y2 = silu(a.z) * u.z; y3 = silu(a.w) * u.w;
+        } else {
+            y0 = gelu_erf(a.x); y1 = gelu_erf(a.y); y2 = gelu_erf(a.z); y3 = gelu_erf(a.w);
+        }
+        const __nv_bfloat162 h01 = __floats2bfloat162_rn(y0, y1), h23 = __floats2bfloat162_rn(y2, y3);
+        const __nv_bfloat162 l01 = __floats2bfloat162_rn(y0 - __low2float(h01), y1 - __high2float(h01));
+        const __nv_bfloat162 l23 = __floats2bfloat162_rn(y2 - __low2float(h23), y3 - __high2float(h23));
+        uint2 hv, lv;
+        hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
+        lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
+        __nv_bfloat16 *base = p.op[OP_ACT];
+        *reinterpret_cast<uint2 *>(base + (size_t)r * p.op_ld[OP_ACT] + 4 * c) = hv;
+        *reinterpret_cast<uint2 *>(base + (size_t)(p.rk + r) * p.op_ld[OP_ACT] + 4 * c) = lv;
     }
 }
 
-__device__ __forceinline__ void setup_phase(const FwdParams &p) {
+__device__ __noinline__ void setup_phase(const FwdParams &p) {
     const int half = p.rotary_dim / 2;
     for (int r = blockIdx.x; r < p.R; r += gridDim.x) {
         const int b = r / p.M, j = r % p.M;
@@ -314,7 +378,7 @@ __device__ __forceinline__ void setup_phase(const FwdParams &p) {
     }
 }
 
-__device__ __forceinline__ void embed_phase(const FwdParams &p) {
+__device__ __noinline__ void embed_phase(const FwdParams &p) {
     for (int r = blockIdx.x; r < p.R; r += gridDim.x) {
         const int b = r / p.M, j = r % p.M;
         int tok = __ldcg(p.ri.valid + r) ? p.tokens[(size_t)b * p.tok_stride + j] : 0;
@@ -334,175 +398,291 @@ __device__ __forceinline__ void embed_phase(const FwdParams &p) {
     }
 }
 
-// Attention of one (sequence, head, split) item by 256 threads: rotary on q, the new rows' keys /
-// values taken from qkv (rotary, cache rounding) and appended to the cache by the split that owns
-// their positions, running softmax, P.V; the last split to finish merges all splits into ao.
-template <int MR>
-__device__ void attention_item(const FwdParams &p, int layer, int item, uint8_t *scratch, Shared *sh) {
-    const int split = item % p.n_split, bh = item / p.n_split, b = bh / p.H, h = bh % p.H;
-    const int Dh = p.Dh, pitch = Dh + 8, d = p.d;
-    float *Qs = reinterpret_cast<float *>(scratch);
-    float *Ps = Qs + MR * Dh;
-    float *fac = Ps + MR * kAttnTile;
-    float *run_m = fac + MR, *run_l = run_m + MR;
-    __nv_bfloat16 *Ks = reinterpret_cast<__nv_bfloat16 *>(run_l + MR);
-    __nv_bfloat16 *Vs = Ks + kAttnTile * pitch;
+// ---- attention ---------------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async16(void *dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t addr, uint32_t &r0, uint32_t &r1) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
+constexpr int kAttnRows = 16;  // query rows per item (one MMA row tile)
+__host__ __device__ inline size_t attn_scratch_bytes(int Dh) {
+    // Q hi/lo [16][Dh+8] bf16, two K/V chunk buffers [2][64][Dh+8] bf16 each, per-warp (m, l) [8][16] fp32 x 2
+    return (size_t)2 * kAttnRows * (Dh + 8) * 2 + (size_t)2 * 2 * kAttnTile * (Dh + 8) * 2 + 2 * 8 * kAttnRows * 4;
+}
+
+// Attention of up to 16 query rows of one (sequence, head) over one split of the position axis, by
+// 256 threads, on tensor cores.  K/V chunks of 64 positions are fetched with cp.async into two
+// buffers (the next chunk loads while this one is used).  Warp w owns positions 16 (w & 3) .. +15
+// of each chunk and the output columns of half (w >> 2) of the head: it computes its 16 x 16 score
+// block S = Q K^T (Q as bf16 hi + lo), keeps its own running max / sum, and adds P V (P as bf16
+// hi + lo) to its 16 x Dh/2 accumulators -- no exchange between warps until the end, where the
+// four position groups are merged in shared memory.  Rows of this pass (positions >= len) take
+// their keys / values from qkv (rotary, cache rounding) and the split that owns them appends them
+// to the cache.  With one split the result goes straight to the out-projection operand; otherwise
+// partials are written and the split that finishes last merges them.  All exponentials are base 2.
+__device__ __noinline__ void attention_item(const FwdParams &p, int layer, int item, uint8_t *scratch, Shared *sh) {
+    const int MT = (p.M + kAttnRows - 1) / kAttnRows;
+    const int mt = item % MT, rest = item / MT;
+    const int split = rest % p.n_split, bh = rest / p.n_split, b = bh / p.H, h = bh % p.H;
+    const int Dh = p.Dh, d = p.d, pitch = Dh + 8;
+    const uint32_t pitchB = (uint32_t)pitch * 2u;
+    __nv_bfloat16 *Qhi = reinterpret_cast<__nv_bfloat16 *>(scratch);
+    __nv_bfloat16 *Qlo = Qhi + kAttnRows * pitch;
+    __nv_bfloat16 *KV = Qlo + kAttnRows * pitch;  // buffer i: K at KV + i * 2 * 64 * pitch, V 64 * pitch later
+    float *mw = reinterpret_cast<float *>(KV + 2 * 2 * kAttnTile * pitch);
+    float *lw = mw + 8 * kAttnRows;
+    float *o_acc = reinterpret_cast<float *>(KV);  // [16][Dh] fp32, reuses the chunk buffers after the loop
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int pg = warp & 3, dhh = warp >> 2;
+    const int nk = Dh >> 4;          // k-steps of Q K^T; also 8-column output tiles per head half
+    const int dh0 = dhh * (Dh >> 1);
     const int n_rows = __ldcg(p.ri.n_eff + b);
     const int len = p.len[b];
-    const int r0 = b * p.M;
+    const int r0 = b * p.M, m_base = mt * kAttnRows;
     const int p_begin = split * p.chunk;
     const int p_end = min(p_begin + p.chunk, len + n_rows);
     const int half = p.rotary_dim / 2;
-    constexpr int MH = (MR + 1) / 2;
-    float o[MH];
-#pragma unroll
-    for (int m = 0; m < MH; ++m) o[m] = 0.f;
-    const int e_col = tid & 127, m_par = tid >> 7;  // P.V: column e, rows of parity m_par
+    const float sc = p.attn_scale * 1.4426950408889634f;  // scores in log2 units
 
-    if (tid < kAttnThreadsP) {
-        if (tid < MR) { run_m[tid] = -INFINITY; run_l[tid] = 0.f; }
-        if (p_begin < p_end) {
-            for (int i = tid; i < n_rows * Dh; i += kAttnThreadsP) {
-                const int m = i / Dh, e = i % Dh, r = r0 + m;
-                const float *row = p.qkv + (size_t)r * 3 * d + h * Dh;
-                float q = __ldcg(row + e);
-                if (e < p.rotary_dim) {
-                    const int j = e < half ? e : e - half;
-                    const float c = __ldcg(p.ri.rope_cos + (size_t)r * half + j), s = __ldcg(p.ri.rope_sin + (size_t)r * half + j);
-                    q = e < half ? q * c - __ldcg(row + e + half) * s : __ldcg(row + e - half) * s + q * c;
-                }
-                Qs[m * Dh + e] = q;
+    // ---- Q rows (rotary applied) as bf16 hi / lo ----
+    for (int i = tid; i < kAttnRows * Dh; i += kAttnThreadsP) {
+        const int ml = i / Dh, e = i % Dh, m = m_base + ml;
+        float q = 0.f;
+        if (m < n_rows) {
+            const int r = r0 + m;
+            const float *row = p.qkv + (size_t)r * 3 * d + h * Dh;
+            q = __ldcg(row + e);
+            if (e < p.rotary_dim) {
+                const int j = e < half ? e : e - half;
+                const float c = __ldcg(p.ri.rope_cos + (size_t)r * half + j), s = __ldcg(p.ri.rope_sin + (size_t)r * half + j);
+                q = e < half ? q * c - __ldcg(row + e + half) * s : __ldcg(row + e - half) * s + q * c;
             }
-            __nv_bfloat16 *kc = (__nv_bfloat16 *)(p.cache + (size_t)layer * p.layer_bytes) + ((size_t)(b * 2) * p.H + h) * p.S * Dh;
-            __nv_bfloat16 *vc = kc + (size_t)p.H * p.S * Dh;
-            const int vec_per_row = Dh / 8;
-            for (int t0 = p_begin; t0 < p_end; t0 += kAttnTile) {
-                const int np = min(kAttnTile, p_end - t0);
-                named_bar(3, kAttnThreadsP);
-                for (int i = tid; i < np * vec_per_row; i += kAttnThreadsP) {
-                    const int pp = i / vec_per_row, v8 = i % vec_per_row, pos = t0 + pp;
-                    uint4 kq, vq;
-                    if (pos < len) {
-                        const size_t g = (size_t)pos * Dh + v8 * 8;
-                        kq = __ldcs(reinterpret_cast<const uint4 *>(kc + g));
-                        vq = __ldcs(reinterpret_cast<const uint4 *>(vc + g));
-                    } else {  // a row of this pass: from qkv, position-encoded and rounded as the cache stores it
-                        const int r = r0 + (pos - len);
-                        const float *krow = p.qkv + (size_t)r * 3 * d + d + h * Dh;
-                        const float *vrow = krow + d;
-                        __nv_bfloat16 kb[8], vb[8];
+        }
+        const __nv_bfloat16 hq = __float2bfloat16_rn(q);
+        Qhi[ml * pitch + e] = hq;
+        Qlo[ml * pitch + e] = __float2bfloat16_rn(q - __bfloat162float(hq));
+    }
+
+    __nv_bfloat16 *kc = (__nv_bfloat16 *)(p.cache + (size_t)layer * p.layer_bytes) + ((size_t)(b * 2) * p.H + h) * p.S * Dh;
+    __nv_bfloat16 *vc = kc + (size_t)p.H * p.S * Dh;
+    const int vpr = Dh >> 3;  // 16-byte vectors per row
+    auto load_chunk = [&](int c) {
+        __nv_bfloat16 *Kb = KV + (size_t)(c & 1) * 2 * kAttnTile * pitch, *Vb = Kb + kAttnTile * pitch;
+        const int t0 = p_begin + c * kAttnTile, np = min(kAttnTile, p_end - t0);
+        for (int i = tid; i < kAttnTile * vpr; i += kAttnThreadsP) {
+            const int pp = i / vpr, v8 = i % vpr, pos = t0 + pp;
+            __nv_bfloat16 *dk = Kb + pp * pitch + v8 * 8, *dv = Vb + pp * pitch + v8 * 8;
+            if (pp >= np) {  // beyond the split: zeros (P is 0 there, but 0 * garbage must not be NaN)
+                *reinterpret_cast<uint4 *>(dk) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4 *>(dv) = make_uint4(0, 0, 0, 0);
+            } else if (pos < len) {
+                const size_t go = (size_t)pos * Dh + v8 * 8;
+                cp_async16(dk, kc + go);
+                cp_async16(dv, vc + go);
+            } else {  // a row of this pass: from qkv, position-encoded and rounded as the cache stores it
+                const int r = r0 + (pos - len);
+                const float *krow = p.qkv + (size_t)r * 3 * d + d + h * Dh;
+                const float *vrow = krow + d;
+                __nv_bfloat16 kb[8], vb[8];
 #pragma unroll
-                        for (int t = 0; t < 8; ++t) {
-                            const int e = v8 * 8 + t;
-                            float k = __ldcg(krow + e);
-                            if (e < p.rotary_dim) {
-                                const int j = e < half ? e : e - half;
-                                const float c = __ldcg(p.ri.rope_cos + (size_t)r * half + j), s = __ldcg(p.ri.rope_sin + (size_t)r * half + j);
-                                k = e < half ? k * c - __ldcg(krow + e + half) * s : __ldcg(krow + e - half) * s + k * c;
-                            }
-                            kb[t] = __float2bfloat16_rn(k);
-                            vb[t] = __float2bfloat16_rn(__ldcg(vrow + e));
-                        }
-                        kq = *reinterpret_cast<uint4 *>(kb);
-                        vq = *reinterpret_cast<uint4 *>(vb);
-                        const size_t g = (size_t)pos * Dh + v8 * 8;  // append: exactly one split owns this position
-                        *reinterpret_cast<uint4 *>(kc + g) = kq;
-                        *reinterpret_cast<uint4 *>(vc + g) = vq;
+                for (int u = 0; u < 8; ++u) {
+                    const int e = v8 * 8 + u;
+                    float k = __ldcg(krow + e);
+                    if (e < p.rotary_dim) {
+                        const int j = e < half ? e : e - half;
+                        const float c2 = __ldcg(p.ri.rope_cos + (size_t)r * half + j), s2 = __ldcg(p.ri.rope_sin + (size_t)r * half + j);
+                        k = e < half ? k * c2 - __ldcg(krow + e + half) * s2 : __ldcg(krow + e - half) * s2 + k * c2;
                     }
-                    *reinterpret_cast<uint4 *>(Ks + pp * pitch + v8 * 8) = kq;
-                    *reinterpret_cast<uint4 *>(Vs + pp * pitch + v8 * 8) = vq;
+                    kb[u] = __float2bfloat16_rn(k);
+                    vb[u] = __float2bfloat16_rn(__ldcg(vrow + e));
                 }
-                named_bar(3, kAttnThreadsP);
-                {   // scores: thread = (position, row group of 4)
-                    const int pp = tid % kAttnTile, mg = tid / kAttnTile;
-                    constexpr int MQ = (MR + 3) / 4;
-                    float s[MQ];
-#pragma unroll
-                    for (int i = 0; i < MQ; ++i) s[i] = 0.f;
-                    if (pp < np) {
-                        for (int v8 = 0; v8 < vec_per_row; ++v8) {
-                            float kv[8];
-                            load8<__nv_bfloat16>(Ks + pp * pitch + v8 * 8, kv);
-#pragma unroll
-                            for (int i = 0; i < MQ; ++i) {
-                                const int m = mg + 4 * i;
-                                if (m < n_rows) {
-                                    const float *qv = Qs + m * Dh + v8 * 8;
-#pragma unroll
-                                    for (int e = 0; e < 8; ++e) s[i] = fmaf(qv[e], kv[e], s[i]);
-                                }
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int i = 0; i < MQ; ++i) {
-                        const int m = mg + 4 * i;
-                        if (m < MR && m < n_rows) {
-                            const bool vis = pp < np && (t0 + pp) <= len + m;
-                            Ps[m * kAttnTile + pp] = vis ? s[i] * p.attn_scale : -INFINITY;
-                        }
-                    }
-                }
-                named_bar(3, kAttnThreadsP);
-                for (int m = warp; m < n_rows; m += kAttnThreadsP / 32) {
-                    float s0 = Ps[m * kAttnTile + lane], s1 = Ps[m * kAttnTile + lane + 32];
-                    float tmax = warp_max(fmaxf(s0, s1));
-                    float m_old = run_m[m], m_new = fmaxf(m_old, tmax);
-                    float f = 1.f, e0 = 0.f, e1 = 0.f;
-                    if (m_new > -INFINITY) {
-                        f = __expf(m_old - m_new);
-                        e0 = __expf(s0 - m_new);
-                        e1 = __expf(s1 - m_new);
-                    }
-                    Ps[m * kAttnTile + lane] = e0;
-                    Ps[m * kAttnTile + lane + 32] = e1;
-                    float sum = warp_sum(e0 + e1);
-                    if (lane == 0) {
-                        fac[m] = f;
-                        run_m[m] = m_new;
-                        run_l[m] = run_l[m] * f + sum;
-                    }
-                }
-                named_bar(3, kAttnThreadsP);
-                if (e_col < Dh) {
-#pragma unroll
-                    for (int i = 0; i < MH; ++i) {
-                        const int m = 2 * i + m_par;
-                        if (m < n_rows) o[i] *= fac[m];
-                    }
-                    for (int pp = 0; pp < np; ++pp) {
-                        const float v = __bfloat162float(Vs[pp * pitch + e_col]);
-#pragma unroll
-                        for (int i = 0; i < MH; ++i) {
-                            const int m = 2 * i + m_par;
-                            if (m < n_rows) o[i] = fmaf(Ps[m * kAttnTile + pp], v, o[i]);
-                        }
-                    }
+                const uint4 kq = *reinterpret_cast<uint4 *>(kb), vq = *reinterpret_cast<uint4 *>(vb);
+                *reinterpret_cast<uint4 *>(dk) = kq;
+                *reinterpret_cast<uint4 *>(dv) = vq;
+                if (mt == 0) {  // append: exactly one split owns this position
+                    const size_t go = (size_t)pos * Dh + v8 * 8;
+                    *reinterpret_cast<uint4 *>(kc + go) = kq;
+                    *reinterpret_cast<uint4 *>(vc + go) = vq;
                 }
             }
         }
-        named_bar(3, kAttnThreadsP);
-        for (int m = 0; m < p.M; ++m) {
+        cp_async_commit();
+    };
+
+    float o[8][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    const int n_chunks = p_begin < p_end ? (p_end - p_begin + kAttnTile - 1) / kAttnTile : 0;
+
+    if (n_chunks > 0) load_chunk(0);
+    for (int c = 0; c < n_chunks; ++c) {
+        if (c + 1 < n_chunks) load_chunk(c + 1); else cp_async_commit();
+        cp_async_wait<1>();
+        named_bar(3, kAttnThreadsP);  // chunk c (and, first time, Q) is in shared memory
+        const __nv_bfloat16 *Kb = KV + (size_t)(c & 1) * 2 * kAttnTile * pitch, *Vb = Kb + kAttnTile * pitch;
+        const int pos0 = p_begin + c * kAttnTile + 16 * pg;  // this warp's 16 positions
+        // ---- S = Q K^T for 16 rows x 16 positions ----
+        float s[2][4];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+        {
+            const uint32_t qa = smem_u32(Qhi) + (uint32_t)(lane & 15) * pitchB + (uint32_t)(lane >> 4) * 16u;
+            const uint32_t ql = qa + (uint32_t)kAttnRows * pitchB;
+            const uint32_t ka = smem_u32(Kb) + (uint32_t)(16 * pg + (lane & 7) + 8 * (lane >> 4)) * pitchB + (uint32_t)((lane >> 3) & 1) * 16u;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                if (ks < nk) {
+                    uint32_t a0, a1, a2, a3, c0, c1, c2, c3, k0, k1, k2, k3;
+                    ldmatrix_x4(qa + ks * 32, a0, a1, a2, a3);
+                    ldmatrix_x4(ql + ks * 32, c0, c1, c2, c3);
+                    ldmatrix_x4(ka + ks * 32, k0, k1, k2, k3);  // (pos 0-7: k lo, k hi), (pos 8-15: k lo, k hi)
+                    mma_bf16(s[0], a0, a1, a2, a3, k0, k1);
+                    mma_bf16(s[0], c0, c1, c2, c3, k0, k1);
+                    mma_bf16(s[1], a0, a1, a2, a3, k2, k3);
+                    mma_bf16(s[1], c0, c1, c2, c3, k2, k3);
+                }
+            }
+        }
+        // ---- mask, running max / sum (rows g and g + 8) ----
+        float pr[2][4];
+#pragma unroll
+        for (int hrow = 0; hrow < 2; ++hrow) {
+            const int m = m_base + g + 8 * hrow;
+            float mx = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int pos = pos0 + 8 * j + 2 * t + e;
+                    const bool vis = pos < p_end && pos <= len + m;
+                    const float v = vis ? s[j][2 * hrow + e] * sc : -INFINITY;
+                    s[j][2 * hrow + e] = v;
+                    mx = fmaxf(mx, v);
+                }
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+            const float m_new = fmaxf(m_run[hrow], mx);
+            float f = 1.f, sum = 0.f;
+            if (m_new > -INFINITY) {
+                f = exp2f(m_run[hrow] - m_new);  // 0 on the first non-empty block
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float pv = exp2f(s[j][2 * hrow + e] - m_new);
+                        pr[j][2 * hrow + e] = pv;
+                        sum += pv;
+                    }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 2; ++j) pr[j][2 * hrow] = pr[j][2 * hrow + 1] = 0.f;
+            }
+            m_run[hrow] = m_new;
+            l_run[hrow] = l_run[hrow] * f + sum;  // this thread's share; lanes are summed at the end
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { o[j][2 * hrow] *= f; o[j][2 * hrow + 1] *= f; }
+        }
+        // ---- O += P V  (P as hi + lo; k = the 16 positions; n = this warp's Dh/2 columns) ----
+        {
+            uint32_t ph[4], pl[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {  // a0: (row g, k 2t..) a1: (row g+8, ..) a2: (row g, k 8+2t..) a3: (row g+8, ..)
+                const int j = q >> 1, hrow = q & 1;
+                const float x0 = pr[j][2 * hrow], x1 = pr[j][2 * hrow + 1];
+                const __nv_bfloat162 hv = __floats2bfloat162_rn(x0, x1);
+                ph[q] = *reinterpret_cast<const uint32_t *>(&hv);
+                pl[q] = pack_bf16x2(x0 - __low2float(hv), x1 - __high2float(hv));
+            }
+            const uint32_t va = smem_u32(Vb) + (uint32_t)(16 * pg + (lane & 15)) * pitchB + (uint32_t)dh0 * 2u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (j < nk) {
+                    uint32_t b0, b1;
+                    ldmatrix_x2_trans(va + j * 16, b0, b1);
+                    mma_bf16(o[j], ph[0], ph[1], ph[2], ph[3], b0, b1);
+                    mma_bf16(o[j], pl[0], pl[1], pl[2], pl[3], b0, b1);
+                }
+            }
+        }
+        named_bar(3, kAttnThreadsP);  // everyone is done with this buffer before it is refilled
+    }
+    if (n_chunks == 0) named_bar(3, kAttnThreadsP);  // Q stores vs. later reuse of the scratch
+
+    // ---- merge the four position groups ----
+#pragma unroll
+    for (int hrow = 0; hrow < 2; ++hrow) {
+        l_run[hrow] += __shfl_xor_sync(0xffffffffu, l_run[hrow], 1);
+        l_run[hrow] += __shfl_xor_sync(0xffffffffu, l_run[hrow], 2);
+    }
+    if (t == 0) {
+        mw[warp * kAttnRows + g] = m_run[0];
+        mw[warp * kAttnRows + g + 8] = m_run[1];
+        lw[warp * kAttnRows + g] = l_run[0];
+        lw[warp * kAttnRows + g + 8] = l_run[1];
+    }
+    for (int i = tid; i < kAttnRows * Dh; i += kAttnThreadsP) o_acc[i] = 0.f;
+    named_bar(3, kAttnThreadsP);
+#pragma unroll
+    for (int hrow = 0; hrow < 2; ++hrow) {
+        const int row = g + 8 * hrow;
+        float mx = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) mx = fmaxf(mx, mw[q * kAttnRows + row]);
+        const float f = (m_run[hrow] > -INFINITY) ? exp2f(m_run[hrow] - mx) : 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (j < nk && f != 0.f) {
+                float *dst = o_acc + row * Dh + dh0 + 8 * j + 2 * t;
+                atomicAdd(dst, o[j][2 * hrow] * f);
+                atomicAdd(dst + 1, o[j][2 * hrow + 1] * f);
+            }
+        }
+    }
+    named_bar(3, kAttnThreadsP);
+    const bool direct = p.n_split == 1;
+    for (int i = tid; i < kAttnRows * Dh; i += kAttnThreadsP) {
+        const int ml = i / Dh, e = i % Dh, m = m_base + ml;
+        if (m >= p.M) continue;
+        float mx = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) mx = fmaxf(mx, mw[q * kAttnRows + ml]);
+        float L = 0.f;
+        if (mx > -INFINITY) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float mq = mw[q * kAttnRows + ml];
+                if (mq > -INFINITY) L += lw[q * kAttnRows + ml] * exp2f(mq - mx);
+            }
+        }
+        const bool live = m < n_rows && L > 0.f;
+        if (direct) {
+            store_hilo(p.op[OP_AO], p.rk, p.op_ld[OP_AO], r0 + m, h * Dh + e, live ? o_acc[i] / L : 0.f);
+        } else {
             const size_t slot = ((size_t)(r0 + m) * p.H + h) * p.n_split + split;
-            const bool live = m < n_rows && m < MR;
-            if (tid == 0) {
-                p.part_m[slot] = live ? run_m[m] : -INFINITY;
-                p.part_l[slot] = live ? run_l[m] : 0.f;
+            if (e == 0) {
+                p.part_m[slot] = live ? mx : -INFINITY;
+                p.part_l[slot] = live ? L : 0.f;
             }
-            if (e_col < Dh && (m & 1) == m_par) {
-                float val = 0.f;
-#pragma unroll
-                for (int i = 0; i < MH; ++i)
-                    if (2 * i + m_par == m) val = o[i];
-                p.part_o[slot * Dh + e_col] = live ? val : 0.f;
-            }
+            p.part_o[slot * Dh + e] = live ? o_acc[i] : 0.f;
         }
-        // ticket: the split that finishes last for this (sequence, head) merges them
+    }
+    if (!direct) {
+        // ticket: the item that finishes last for this (sequence, head) merges all partials
         __threadfence();
         named_bar(3, kAttnThreadsP);
-        if (tid == 0) sh->flag = (atomicAdd(p.tickets + bh, 1u) == (unsigned)(p.n_split - 1));
+        if (tid == 0) sh->flag = (atomicAdd(p.tickets + bh, 1u) == (unsigned)(p.n_split * MT - 1));
         named_bar(3, kAttnThreadsP);
         if (sh->flag) {
             __threadfence();
@@ -510,34 +690,34 @@ __device__ void attention_item(const FwdParams &p, int layer, int item, uint8_t 
                 const int m = idx / Dh, e = idx % Dh;
                 const size_t base = ((size_t)(r0 + m) * p.H + h) * p.n_split;
                 float mx = -INFINITY;
-                for (int s = 0; s < p.n_split; ++s) mx = fmaxf(mx, __ldcg(p.part_m + base + s));
+                for (int s2 = 0; s2 < p.n_split; ++s2) mx = fmaxf(mx, __ldcg(p.part_m + base + s2));
                 float L = 0.f, acc = 0.f;
                 if (mx > -INFINITY) {
-                    for (int s = 0; s < p.n_split; ++s) {
-                        const float pm = __ldcg(p.part_m + base + s);
+                    for (int s2 = 0; s2 < p.n_split; ++s2) {
+                        const float pm = __ldcg(p.part_m + base + s2);
                         if (pm == -INFINITY) continue;
-                        const float w = __expf(pm - mx);
-                        L = fmaf(__ldcg(p.part_l + base + s), w, L);
-                        acc = fmaf(__ldcg(p.part_o + (base + s) * Dh + e), w, acc);
+                        const float w = exp2f(pm - mx);
+                        L = fmaf(__ldcg(p.part_l + base + s2), w, L);
+                        acc = fmaf(__ldcg(p.part_o + (base + s2) * Dh + e), w, acc);
                     }
                 }
                 store_hilo(p.op[OP_AO], p.rk, p.op_ld[OP_AO], r0 + m, h * Dh + e, L > 0.f ? acc / L : 0.f);
             }
             if (tid == 0) p.tickets[bh] = 0;  // ready for the next layer (a grid barrier lies between)
         }
-        named_bar(3, kAttnThreadsP);
     }
+    named_bar(3, kAttnThreadsP);  // scratch is free for the next item
 }
 
-template <int MR>
 __device__ __forceinline__ void attention_phase(const FwdParams &p, int layer, uint8_t *scratch, Shared *sh) {
-    const int items = p.B * p.H * p.n_split;
-    for (int item = blockIdx.x; item < items; item += gridDim.x) attention_item<MR>(p, layer, item, scratch, sh);
+    const int MT = (p.M + kAttnRows - 1) / kAttnRows;
+    const int items = p.B * p.H * p.n_split * MT;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) attention_item(p, layer, item, scratch, sh);
 }
 
 // ---- the kernel -----------------------------------------------------------------------------
-// NT = padded rows / 8;  MR = compile-time bound on rows per sequence for attention
-template <int NT, int MR>
+// NT = padded rows / 8
+template <int NT>
 __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __grid_constant__ FwdParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -643,9 +823,6 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
         // =============================== work warps ===============================
         int epoch = 0, it = 0;  // grid barriers passed; ring stages consumed
         bool alive = true;      // per warp: false once one of its waits gave up
-        float acc[NT][4];
-#pragma unroll
-        for (int j = 0; j < NT; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
 
         // run this CTA's units of GEMM gi
         auto run_gemm = [&](int gi) {
@@ -653,6 +830,9 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             int c0, c1;
             unit_range(g, c0, c1);
             if (c0 >= c1) return;
+            float acc[NT][4];  // local to the GEMM: nothing to keep alive across the small phases
+#pragma unroll
+            for (int j = 0; j < NT; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
             int tile = c0 / g.kchunks, kc = c0 % g.kchunks;
             auto flush = [&](int t, bool with_bias) {
                 const int n = t * kTileN + warp * 16 + (lane >> 2);
@@ -744,7 +924,7 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             run_gemm(4 * l + 0);                       // qkv
             if (p.parallel) run_gemm(4 * l + 1);       // MLP in (same block input)
             if (!(go = grid_sync(p, sh, epoch))) break;
-            attention_phase<MR>(p, l, attn_scratch, sh);
+            attention_phase(p, l, attn_scratch, sh);
             if (p.parallel) act_phase(p);
             if (!(go = grid_sync(p, sh, epoch))) break;
             if (p.parallel) {

@@ -335,6 +335,11 @@ int gemm(const GemmCall &c, const void *W, const CUtensorMap *tw, const Operand 
 // Split of the position axis for a context of up to `ctx` positions.
 void plan_split(int B, int H, int ctx, int *chunk, int *n_split) {
     if (ctx < 1) ctx = 1;
+    if (ctx <= 256) {  // short context: one item per (sequence, head) writes its result directly
+        *chunk = ceil_div(ctx, kAttnTile) * kAttnTile;
+        *n_split = 1;
+        return;
+    }
     int want = ceil_div(2 * (g_num_sms > 0 ? g_num_sms : 148), B * H);
     int max_by_len = ceil_div(ctx, kAttnTile);
     int ns = want < 1 ? 1 : want;
@@ -398,10 +403,10 @@ int run_attention(const ssd_model *m, ssd_kv *kv, int layer, const float *q, int
 
 inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 4 : 8) * a.n_layers; }
 
-template <int NT, int MR>
+template <int NT>
 int launch_forward_nt(FwdParams p, cudaStream_t st) {
     constexpr int stage = kWTileBytes + 2 * NT * 8 * kTileK * 2;
-    const size_t attn = align_up((size_t)MR * (p.Dh + kAttnTile + 3) * 4 + 2 * (size_t)kAttnTile * (p.Dh + 8) * 2, 128);
+    const size_t attn = align_up(attn_scratch_bytes(p.Dh), 128);
     const size_t tail_fixed = 24 * 12 + 16 + sizeof(Shared) + 16 * sizeof(double) + 256;
     int S = (int)(((size_t)kSmemBudget - 1024 - attn - tail_fixed) / stage);
     if (S > 12) S = 12;
@@ -411,28 +416,27 @@ int launch_forward_nt(FwdParams p, cudaStream_t st) {
     const size_t smem = 1024 + (size_t)p.attn_smem_off + attn;
     static bool attr = false;
     if (!attr) {
-        if (cudaFuncSetAttribute(forward_kernel<NT, MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) !=
+        if (cudaFuncSetAttribute(forward_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) !=
             cudaSuccess)
             return SSD_E_CUDA;
         attr = true;
     }
     void *args[] = {&p};
-    if (cudaLaunchCooperativeKernel((void *)forward_kernel<NT, MR>, dim3(g_num_sms), dim3(kPersistThreads), args, smem,
+    if (cudaLaunchCooperativeKernel((void *)forward_kernel<NT>, dim3(g_num_sms), dim3(kPersistThreads), args, smem,
                                     st) != cudaSuccess)
         return SSD_E_CUDA;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return SSD_OK;
 }
 
-template <int MR>
-int launch_forward_mr(const FwdParams &p, int rows_k, cudaStream_t st) {
+int launch_forward_rows(const FwdParams &p, int rows_k, cudaStream_t st) {
     switch (rows_k / 8) {
-        case 1: if (MR == 8) return launch_forward_nt<1, 8>(p, st); break;
-        case 2: if (MR <= 16) return launch_forward_nt<2, MR <= 16 ? MR : 8>(p, st); break;
-        case 3: return launch_forward_nt<3, MR>(p, st);
-        case 4: return launch_forward_nt<4, MR>(p, st);
-        case 5: return launch_forward_nt<5, MR>(p, st);
-        case 8: return launch_forward_nt<8, MR>(p, st);
+        case 1: return launch_forward_nt<1>(p, st);
+        case 2: return launch_forward_nt<2>(p, st);
+        case 3: return launch_forward_nt<3>(p, st);
+        case 4: return launch_forward_nt<4>(p, st);
+        case 5: return launch_forward_nt<5>(p, st);
+        case 8: return launch_forward_nt<8>(p, st);
         default: break;
     }
     return SSD_E_CAPACITY;
@@ -472,10 +476,7 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     p.want_logits = want_logits ? 1 : 0;
     p.trace = (g_trace && 2 + barriers_needed(a) + 3 < kTraceSlots) ? w.trace : nullptr;
     CUDA_OK(cudaMemsetAsync(w.sync, 0, w.sync_bytes, st));
-    int rc;
-    if (M <= 8) rc = launch_forward_mr<8>(p, Rk, st);
-    else if (M <= 16) rc = launch_forward_mr<16>(p, Rk, st);
-    else rc = launch_forward_mr<32>(p, Rk, st);
+    int rc = launch_forward_rows(p, Rk, st);
     if (rc) return rc;
     kv->last_rows = M;
     return SSD_OK;
@@ -486,7 +487,7 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
 int forward(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int M, const int32_t *n_rows,
             bool want_logits, const Workspace &w, cudaStream_t st) {
     const ssd_arch &a = m->a;
-    if (a.dtype == 1 && g_persistent && m->dev_desc)
+    if (a.dtype == 1 && g_persistent && m->dev_desc && a.head_dim % 16 == 0)  // the MMA attention tiles by 16
         return forward_persistent(m, kv, tokens, tok_stride, M, n_rows, want_logits, w, st);
     const int B = kv->B, R = B * M, d = a.d_model, F = a.d_ff;
     GemmCall gc{m, st, R, (R + 7) / 8 * 8};
