@@ -413,15 +413,39 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<const uint32_t *>(&v);
 }
 
+// Columns e0 .. e0+7 of one head's q or k row (fp32, `row` points at the head's first column) with
+// the rotary turn of row r applied; rotary_dim and its half are multiples of 8, so the eight
+// columns fall on one side of the split.  All loads are issued before the first use.
+__device__ __forceinline__ void rope_vec8(const FwdParams &p, const float *row, int r, int e0, float (&out)[8]) {
+    const float4 a0 = __ldcg(reinterpret_cast<const float4 *>(row + e0)), a1 = __ldcg(reinterpret_cast<const float4 *>(row + e0 + 4));
+    out[0] = a0.x; out[1] = a0.y; out[2] = a0.z; out[3] = a0.w; out[4] = a1.x; out[5] = a1.y; out[6] = a1.z; out[7] = a1.w;
+    if (e0 < p.rotary_dim) {
+        const int half = p.rotary_dim >> 1;
+        const bool low = e0 < half;
+        const int j0 = low ? e0 : e0 - half;
+        const float *pr_ = row + (low ? e0 + half : e0 - half);
+        const float4 b0 = __ldcg(reinterpret_cast<const float4 *>(pr_)), b1 = __ldcg(reinterpret_cast<const float4 *>(pr_ + 4));
+        const float *cp = p.ri.rope_cos + (size_t)r * half + j0, *sp = p.ri.rope_sin + (size_t)r * half + j0;
+        const float4 c0 = __ldcg(reinterpret_cast<const float4 *>(cp)), c1 = __ldcg(reinterpret_cast<const float4 *>(cp + 4));
+        const float4 s0 = __ldcg(reinterpret_cast<const float4 *>(sp)), s1 = __ldcg(reinterpret_cast<const float4 *>(sp + 4));
+        const float pb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+        const float cc[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        const float ss[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+        for (int u = 0; u < 8; ++u) out[u] = low ? out[u] * cc[u] - pb[u] * ss[u] : pb[u] * ss[u] + out[u] * cc[u];
+    }
+}
+
 constexpr int kAttnRows = 16;  // query rows per item (one MMA row tile)
+constexpr int kAttnBufs = 3;   // K/V chunk buffers: two chunks (64 KB at head 128) in flight per SM
 __host__ __device__ inline size_t attn_scratch_bytes(int Dh) {
-    // Q hi/lo [16][Dh+8] bf16, two K/V chunk buffers [2][64][Dh+8] bf16 each, per-warp (m, l) [8][16] fp32 x 2
-    return (size_t)2 * kAttnRows * (Dh + 8) * 2 + (size_t)2 * 2 * kAttnTile * (Dh + 8) * 2 + 2 * 8 * kAttnRows * 4;
+    // Q hi/lo [16][Dh+8] bf16, kAttnBufs K/V chunk buffers [2][64][Dh+8] bf16 each, per-warp (m, l) [8][16] fp32 x 2
+    return (size_t)2 * kAttnRows * (Dh + 8) * 2 + (size_t)kAttnBufs * 2 * kAttnTile * (Dh + 8) * 2 + 2 * 8 * kAttnRows * 4;
 }
 
 // Attention of up to 16 query rows of one (sequence, head) over one split of the position axis, by
-// 256 threads, on tensor cores.  K/V chunks of 64 positions are fetched with cp.async into two
-// buffers (the next chunk loads while this one is used).  Warp w owns positions 16 (w & 3) .. +15
+// 256 threads, on tensor cores.  K/V chunks of 64 positions are fetched with cp.async into three
+// buffers (the next two chunks load while this one is used).  Warp w owns positions 16 (w & 3) .. +15
 // of each chunk and the output columns of half (w >> 2) of the head: it computes its 16 x 16 score
 // block S = Q K^T (Q as bf16 hi + lo), keeps its own running max / sum, and adds P V (P as bf16
 // hi + lo) to its 16 x Dh/2 accumulators -- no exchange between warps until the end, where the
@@ -438,9 +462,9 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
     __nv_bfloat16 *Qhi = reinterpret_cast<__nv_bfloat16 *>(scratch);
     __nv_bfloat16 *Qlo = Qhi + kAttnRows * pitch;
     __nv_bfloat16 *KV = Qlo + kAttnRows * pitch;  // buffer i: K at KV + i * 2 * 64 * pitch, V 64 * pitch later
-    float *mw = reinterpret_cast<float *>(KV + 2 * 2 * kAttnTile * pitch);
+    float *mw = reinterpret_cast<float *>(KV + kAttnBufs * 2 * kAttnTile * pitch);
     float *lw = mw + 8 * kAttnRows;
-    float *o_acc = reinterpret_cast<float *>(KV);  // [16][Dh] fp32, reuses the chunk buffers after the loop
+    float *o_acc = reinterpret_cast<float *>(KV);  // [4][16][Dh] fp32, reuses the chunk buffers after the loop
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -452,68 +476,59 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
     const int r0 = b * p.M, m_base = mt * kAttnRows;
     const int p_begin = split * p.chunk;
     const int p_end = min(p_begin + p.chunk, len + n_rows);
-    const int half = p.rotary_dim / 2;
     const float sc = p.attn_scale * 1.4426950408889634f;  // scores in log2 units
-
-    // ---- Q rows (rotary applied) as bf16 hi / lo ----
-    for (int i = tid; i < kAttnRows * Dh; i += kAttnThreadsP) {
-        const int ml = i / Dh, e = i % Dh, m = m_base + ml;
-        float q = 0.f;
-        if (m < n_rows) {
-            const int r = r0 + m;
-            const float *row = p.qkv + (size_t)r * 3 * d + h * Dh;
-            q = __ldcg(row + e);
-            if (e < p.rotary_dim) {
-                const int j = e < half ? e : e - half;
-                const float c = __ldcg(p.ri.rope_cos + (size_t)r * half + j), s = __ldcg(p.ri.rope_sin + (size_t)r * half + j);
-                q = e < half ? q * c - __ldcg(row + e + half) * s : __ldcg(row + e - half) * s + q * c;
-            }
-        }
-        const __nv_bfloat16 hq = __float2bfloat16_rn(q);
-        Qhi[ml * pitch + e] = hq;
-        Qlo[ml * pitch + e] = __float2bfloat16_rn(q - __bfloat162float(hq));
-    }
 
     __nv_bfloat16 *kc = (__nv_bfloat16 *)(p.cache + (size_t)layer * p.layer_bytes) + ((size_t)(b * 2) * p.H + h) * p.S * Dh;
     __nv_bfloat16 *vc = kc + (size_t)p.H * p.S * Dh;
     const int vpr = Dh >> 3;  // 16-byte vectors per row
     auto load_chunk = [&](int c) {
-        __nv_bfloat16 *Kb = KV + (size_t)(c & 1) * 2 * kAttnTile * pitch, *Vb = Kb + kAttnTile * pitch;
+        __nv_bfloat16 *Kb = KV + (size_t)(c % kAttnBufs) * 2 * kAttnTile * pitch, *Vb = Kb + kAttnTile * pitch;
         const int t0 = p_begin + c * kAttnTile, np = min(kAttnTile, p_end - t0);
-        for (int i = tid; i < kAttnTile * vpr; i += kAttnThreadsP) {
-            const int pp = i / vpr, v8 = i % vpr, pos = t0 + pp;
-            __nv_bfloat16 *dk = Kb + pp * pitch + v8 * 8, *dv = Vb + pp * pitch + v8 * 8;
-            if (pp >= np) {  // beyond the split: zeros (P is 0 there, but 0 * garbage must not be NaN)
-                *reinterpret_cast<uint4 *>(dk) = make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4 *>(dv) = make_uint4(0, 0, 0, 0);
-            } else if (pos < len) {
-                const size_t go = (size_t)pos * Dh + v8 * 8;
-                cp_async16(dk, kc + go);
-                cp_async16(dv, vc + go);
-            } else {  // a row of this pass: from qkv, position-encoded and rounded as the cache stores it
-                const int r = r0 + (pos - len);
-                const float *krow = p.qkv + (size_t)r * 3 * d + d + h * Dh;
-                const float *vrow = krow + d;
-                __nv_bfloat16 kb[8], vb[8];
+        const int prow = tid >> 4, v8 = tid & 15;  // 16 threads per row, 16 rows per pass
+        if (v8 < vpr) {
+            if (t0 + kAttnTile <= len) {  // the common case: all 64 positions come from the cache
+                const __nv_bfloat16 *ks = kc + (size_t)(t0 + prow) * Dh + v8 * 8, *vs = vc + (size_t)(t0 + prow) * Dh + v8 * 8;
+                __nv_bfloat16 *dk = Kb + prow * pitch + v8 * 8, *dv = Vb + prow * pitch + v8 * 8;
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int e = v8 * 8 + u;
-                    float k = __ldcg(krow + e);
-                    if (e < p.rotary_dim) {
-                        const int j = e < half ? e : e - half;
-                        const float c2 = __ldcg(p.ri.rope_cos + (size_t)r * half + j), s2 = __ldcg(p.ri.rope_sin + (size_t)r * half + j);
-                        k = e < half ? k * c2 - __ldcg(krow + e + half) * s2 : __ldcg(krow + e - half) * s2 + k * c2;
-                    }
-                    kb[u] = __float2bfloat16_rn(k);
-                    vb[u] = __float2bfloat16_rn(__ldcg(vrow + e));
+                for (int q = 0; q < kAttnTile / 16; ++q) {
+                    cp_async16(dk + q * 16 * pitch, ks + (size_t)q * 16 * Dh);
+                    cp_async16(dv + q * 16 * pitch, vs + (size_t)q * 16 * Dh);
                 }
-                const uint4 kq = *reinterpret_cast<uint4 *>(kb), vq = *reinterpret_cast<uint4 *>(vb);
-                *reinterpret_cast<uint4 *>(dk) = kq;
-                *reinterpret_cast<uint4 *>(dv) = vq;
-                if (mt == 0) {  // append: exactly one split owns this position
-                    const size_t go = (size_t)pos * Dh + v8 * 8;
-                    *reinterpret_cast<uint4 *>(kc + go) = kq;
-                    *reinterpret_cast<uint4 *>(vc + go) = vq;
+            } else {
+#pragma unroll 1
+                for (int q = 0; q < kAttnTile / 16; ++q) {
+                    const int pp = prow + 16 * q, pos = t0 + pp;
+                    __nv_bfloat16 *dk = Kb + pp * pitch + v8 * 8, *dv = Vb + pp * pitch + v8 * 8;
+                    if (pp >= np) {  // beyond the split: zeros (P is 0 there, but 0 * garbage must not be NaN)
+                        *reinterpret_cast<uint4 *>(dk) = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4 *>(dv) = make_uint4(0, 0, 0, 0);
+                    } else if (pos < len) {
+                        const size_t go = (size_t)pos * Dh + v8 * 8;
+                        cp_async16(dk, kc + go);
+                        cp_async16(dv, vc + go);
+                    } else {  // a row of this pass: from qkv, position-encoded and rounded as the cache stores it
+                        const int r = r0 + (pos - len);
+                        const float *krow = p.qkv + (size_t)r * 3 * d + d + h * Dh;
+                        float kf[8];
+                        rope_vec8(p, krow, r, v8 * 8, kf);
+                        const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(krow + d + v8 * 8));
+                        const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(krow + d + v8 * 8 + 4));
+                        const float vf[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                        __nv_bfloat16 kb[8], vb[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            kb[u] = __float2bfloat16_rn(kf[u]);
+                            vb[u] = __float2bfloat16_rn(vf[u]);
+                        }
+                        const uint4 kq = *reinterpret_cast<uint4 *>(kb), vq = *reinterpret_cast<uint4 *>(vb);
+                        *reinterpret_cast<uint4 *>(dk) = kq;
+                        *reinterpret_cast<uint4 *>(dv) = vq;
+                        if (mt == 0) {  // append: exactly one split owns this position
+                            const size_t go = (size_t)pos * Dh + v8 * 8;
+                            *reinterpret_cast<uint4 *>(kc + go) = kq;
+                            *reinterpret_cast<uint4 *>(vc + go) = vq;
+                        }
+                    }
                 }
             }
         }
@@ -526,18 +541,46 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
     const int n_chunks = p_begin < p_end ? (p_end - p_begin + kAttnTile - 1) / kAttnTile : 0;
 
-    if (n_chunks > 0) load_chunk(0);
-    for (int c = 0; c < n_chunks; ++c) {
-        if (c + 1 < n_chunks) load_chunk(c + 1); else cp_async_commit();
-        cp_async_wait<1>();
-        named_bar(3, kAttnThreadsP);  // chunk c (and, first time, Q) is in shared memory
-        const __nv_bfloat16 *Kb = KV + (size_t)(c & 1) * 2 * kAttnTile * pitch, *Vb = Kb + kAttnTile * pitch;
-        const int pos0 = p_begin + c * kAttnTile + 16 * pg;  // this warp's 16 positions
-        // ---- S = Q K^T for 16 rows x 16 positions ----
-        float s[2][4];
+    // kAttnBufs - 1 chunks are always in flight; one group is committed per chunk slot so that
+    // "at most kAttnBufs - 1 groups pending" means "chunk c has landed"
+    for (int c = 0; c < kAttnBufs - 1; ++c) {
+        if (c < n_chunks) load_chunk(c); else cp_async_commit();
+    }
+    // ---- Q rows (rotary applied) as bf16 hi / lo: thread = (row, 8 columns) ----
+    {
+        const int ml = tid >> 4, v8 = tid & 15, m = m_base + ml;
+        if (v8 < vpr) {
+            float q[8];
 #pragma unroll
-        for (int j = 0; j < 2; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+            for (int u = 0; u < 8; ++u) q[u] = 0.f;
+            if (m < n_rows) rope_vec8(p, p.qkv + (size_t)(r0 + m) * 3 * d + h * Dh, r0 + m, v8 * 8, q);
+            __nv_bfloat16 hq[8], lq[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                hq[u] = __float2bfloat16_rn(q[u]);
+                lq[u] = __float2bfloat16_rn(q[u] - __bfloat162float(hq[u]));
+            }
+            *reinterpret_cast<uint4 *>(Qhi + ml * pitch + v8 * 8) = *reinterpret_cast<uint4 *>(hq);
+            *reinterpret_cast<uint4 *>(Qlo + ml * pitch + v8 * 8) = *reinterpret_cast<uint4 *>(lq);
+        }
+    }
+    for (int c = 0; c < n_chunks; ++c) {
+        if (c + kAttnBufs - 1 < n_chunks) load_chunk(c + kAttnBufs - 1); else cp_async_commit();
+        cp_async_wait<kAttnBufs - 1>();
+        named_bar(3, kAttnThreadsP);  // chunk c (and, first time, Q) is in shared memory
+        const __nv_bfloat16 *Kb = KV + (size_t)(c % kAttnBufs) * 2 * kAttnTile * pitch, *Vb = Kb + kAttnTile * pitch;
+        const int pos0 = p_begin + c * kAttnTile + 16 * pg;  // this warp's 16 positions
+        // ---- S = Q K^T for 16 rows x 16 positions; four independent accumulator sets (Q hi / lo x
+        //      even / odd k-step) keep the dependent MMA chains short ----
+        float s[2][4];
         {
+            float sa[2][2][2][4];  // [hi|lo][even|odd][position tile][4]
+#pragma unroll
+            for (int x = 0; x < 2; ++x)
+#pragma unroll
+                for (int y = 0; y < 2; ++y)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) sa[x][y][j][0] = sa[x][y][j][1] = sa[x][y][j][2] = sa[x][y][j][3] = 0.f;
             const uint32_t qa = smem_u32(Qhi) + (uint32_t)(lane & 15) * pitchB + (uint32_t)(lane >> 4) * 16u;
             const uint32_t ql = qa + (uint32_t)kAttnRows * pitchB;
             const uint32_t ka = smem_u32(Kb) + (uint32_t)(16 * pg + (lane & 7) + 8 * (lane >> 4)) * pitchB + (uint32_t)((lane >> 3) & 1) * 16u;
@@ -548,12 +591,16 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
                     ldmatrix_x4(qa + ks * 32, a0, a1, a2, a3);
                     ldmatrix_x4(ql + ks * 32, c0, c1, c2, c3);
                     ldmatrix_x4(ka + ks * 32, k0, k1, k2, k3);  // (pos 0-7: k lo, k hi), (pos 8-15: k lo, k hi)
-                    mma_bf16(s[0], a0, a1, a2, a3, k0, k1);
-                    mma_bf16(s[0], c0, c1, c2, c3, k0, k1);
-                    mma_bf16(s[1], a0, a1, a2, a3, k2, k3);
-                    mma_bf16(s[1], c0, c1, c2, c3, k2, k3);
+                    mma_bf16(sa[0][ks & 1][0], a0, a1, a2, a3, k0, k1);
+                    mma_bf16(sa[1][ks & 1][0], c0, c1, c2, c3, k0, k1);
+                    mma_bf16(sa[0][ks & 1][1], a0, a1, a2, a3, k2, k3);
+                    mma_bf16(sa[1][ks & 1][1], c0, c1, c2, c3, k2, k3);
                 }
             }
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) s[j][e] = (sa[0][0][j][e] + sa[0][1][j][e]) + (sa[1][0][j][e] + sa[1][1][j][e]);
         }
         // ---- mask, running max / sum (rows g and g + 8) ----
         float pr[2][4];
@@ -632,8 +679,9 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
         lw[warp * kAttnRows + g] = l_run[0];
         lw[warp * kAttnRows + g + 8] = l_run[1];
     }
-    for (int i = tid; i < kAttnRows * Dh; i += kAttnThreadsP) o_acc[i] = 0.f;
     named_bar(3, kAttnThreadsP);
+    // every warp scales its block to the common maximum and stores it: o_part[pg][16][Dh] (fp32, in the
+    // chunk buffers, free now); the output loop adds the four position groups in a fixed order
 #pragma unroll
     for (int hrow = 0; hrow < 2; ++hrow) {
         const int row = g + 8 * hrow;
@@ -643,10 +691,9 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
         const float f = (m_run[hrow] > -INFINITY) ? exp2f(m_run[hrow] - mx) : 0.f;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            if (j < nk && f != 0.f) {
-                float *dst = o_acc + row * Dh + dh0 + 8 * j + 2 * t;
-                atomicAdd(dst, o[j][2 * hrow] * f);
-                atomicAdd(dst + 1, o[j][2 * hrow + 1] * f);
+            if (j < nk) {
+                float2 v2 = make_float2(o[j][2 * hrow] * f, o[j][2 * hrow + 1] * f);
+                *reinterpret_cast<float2 *>(o_acc + ((size_t)pg * kAttnRows + row) * Dh + dh0 + 8 * j + 2 * t) = v2;
             }
         }
     }
@@ -667,15 +714,17 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
             }
         }
         const bool live = m < n_rows && L > 0.f;
+        const int gs = kAttnRows * Dh;  // stride between position groups
+        const float osum = (o_acc[i] + o_acc[i + gs]) + (o_acc[i + 2 * gs] + o_acc[i + 3 * gs]);
         if (direct) {
-            store_hilo(p.op[OP_AO], p.rk, p.op_ld[OP_AO], r0 + m, h * Dh + e, live ? o_acc[i] / L : 0.f);
+            store_hilo(p.op[OP_AO], p.rk, p.op_ld[OP_AO], r0 + m, h * Dh + e, live ? osum / L : 0.f);
         } else {
             const size_t slot = ((size_t)(r0 + m) * p.H + h) * p.n_split + split;
             if (e == 0) {
                 p.part_m[slot] = live ? mx : -INFINITY;
                 p.part_l[slot] = live ? L : 0.f;
             }
-            p.part_o[slot * Dh + e] = live ? o_acc[i] : 0.f;
+            p.part_o[slot * Dh + e] = live ? osum : 0.f;
         }
     }
     if (!direct) {

@@ -332,19 +332,17 @@ int gemm(const GemmCall &c, const void *W, const CUtensorMap *tw, const Operand 
     return SSD_OK;
 }
 
-// Split of the position axis for a context of up to `ctx` positions.
-void plan_split(int B, int H, int ctx, int *chunk, int *n_split) {
+// Split of the position axis for a context of up to `ctx` positions, `groups` = independent
+// (sequence, head, row-tile) streams.  Every item pays a few microseconds of fixed latency, so the
+// aim is one round of items over the SMs: as many splits as keep groups * splits <= #SMs.
+void plan_split(int groups, int ctx, int *chunk, int *n_split) {
     if (ctx < 1) ctx = 1;
-    if (ctx <= 256) {  // short context: one item per (sequence, head) writes its result directly
-        *chunk = ceil_div(ctx, kAttnTile) * kAttnTile;
-        *n_split = 1;
-        return;
-    }
-    int want = ceil_div(2 * (g_num_sms > 0 ? g_num_sms : 148), B * H);
-    int max_by_len = ceil_div(ctx, kAttnTile);
-    int ns = want < 1 ? 1 : want;
+    const int sms = g_num_sms > 0 ? g_num_sms : 148;
+    int ns = ctx <= 256 ? 1 : sms / (groups > 0 ? groups : 1);
+    int max_by_len = ceil_div(ctx, 2 * kAttnTile);  // at least two chunks per split
     if (ns > max_by_len) ns = max_by_len;
     if (ns > kMaxSplit) ns = kMaxSplit;
+    if (ns < 1) ns = 1;
     int ch = ceil_div(ceil_div(ctx, ns), kAttnTile) * kAttnTile;
     *chunk = ch;
     *n_split = ceil_div(ctx, ch);
@@ -388,7 +386,7 @@ int run_attention(const ssd_model *m, ssd_kv *kv, int layer, const float *q, int
     at.M = M; at.H = a.n_heads; at.Dh = a.head_dim; at.S = kv->S; at.d = a.d_model;
     int ctx = kv->len_ub + M;
     if (ctx > kv->S) ctx = kv->S;
-    plan_split(kv->B, a.n_heads, ctx, &at.chunk, &at.n_split);
+    plan_split(kv->B * a.n_heads, ctx, &at.chunk, &at.n_split);
     at.scale = 1.0f / sqrtf((float)a.head_dim);
     at.ri = w.ri;
     at.part_m = w.part_m; at.part_l = w.part_l; at.part_o = w.part_o;
@@ -472,7 +470,7 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     p.gbar = w.sync; p.tickets = w.sync + 16;
     int ctx = kv->len_ub + M;
     if (ctx > kv->S) ctx = kv->S;
-    plan_split(kv->B, a.n_heads, ctx, &p.chunk, &p.n_split);
+    plan_split(kv->B * a.n_heads * ((M + 15) / 16), ctx, &p.chunk, &p.n_split);
     p.want_logits = want_logits ? 1 : 0;
     p.trace = (g_trace && 2 + barriers_needed(a) + 3 < kTraceSlots) ? w.trace : nullptr;
     CUDA_OK(cudaMemsetAsync(w.sync, 0, w.sync_bytes, st));
@@ -487,7 +485,8 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
 int forward(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int M, const int32_t *n_rows,
             bool want_logits, const Workspace &w, cudaStream_t st) {
     const ssd_arch &a = m->a;
-    if (a.dtype == 1 && g_persistent && m->dev_desc && a.head_dim % 16 == 0)  // the MMA attention tiles by 16
+    if (a.dtype == 1 && g_persistent && m->dev_desc && a.head_dim % 16 == 0 &&
+        (a.pos == 0 || a.rotary_dim % 16 == 0))  // the MMA attention tiles heads by 16 and rotary halves by 8
         return forward_persistent(m, kv, tokens, tok_stride, M, n_rows, want_logits, w, st);
     const int B = kv->B, R = B * M, d = a.d_model, F = a.d_ff;
     GemmCall gc{m, st, R, (R + 7) / 8 * 8};
