@@ -260,7 +260,8 @@ int ssd_read_trace(const ssd_model *m, int batch, int rows_per_seq, const void *
 /* Number of kernels this library has launched in this process so far. */
 uint64_t ssd_launch_count(void);
 
-/* Device time attributed to the weight-streaming GEMM kernel: when enabled, every launch of it
+/* Device time attributed to the kernel that streams the weights -- the single forward kernel of a
+ * bf16 model, or every GEMM launch on the one-launch-per-step path: when enabled, each such launch
  * is bracketed by CUDA events on its stream; ssd_gemm_profile_read synchronises and returns the
  * launches and total milliseconds since the last reset.  Off by default. */
 int ssd_gemm_profile(int enable);

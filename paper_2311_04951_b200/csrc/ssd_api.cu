@@ -28,12 +28,34 @@ int g_num_sms = 0;
 bool g_attr_done = false;
 std::mutex g_mu;
 
-// ---- optional per-launch timing of the weight-streaming GEMM ----
+// ---- optional per-launch timing of the kernel that streams the weights (forward_kernel for bf16
+//      models in single-kernel mode, otherwise every gemm launch) ----
 bool g_persistent = true;  // bf16 models: whole forward in one cooperative kernel
 bool g_trace = false;       // stamp the global timer after every grid barrier of the forward kernel
 bool g_prof = false;
 std::vector<cudaEvent_t> g_prof_events;  // pairs
 size_t g_prof_used = 0;
+
+// start/stop events around a launch when profiling is on (0 = ok)
+int prof_begin(cudaStream_t st, cudaEvent_t *stop) {
+    *stop = nullptr;
+    if (!g_prof) return 0;
+    if (g_prof_used + 2 > g_prof_events.size()) {
+        for (int i = 0; i < 2; ++i) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) return -1;
+            g_prof_events.push_back(e);
+        }
+    }
+    cudaEvent_t e0 = g_prof_events[g_prof_used];
+    *stop = g_prof_events[g_prof_used + 1];
+    g_prof_used += 2;
+    return cudaEventRecord(e0, st) == cudaSuccess ? 0 : -1;
+}
+int prof_end(cudaStream_t st, cudaEvent_t stop) {
+    if (!stop) return 0;
+    return cudaEventRecord(stop, st) == cudaSuccess ? 0 : -1;
+}
 
 #define CUDA_OK(expr)                        \
     do {                                     \
@@ -474,7 +496,10 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     p.want_logits = want_logits ? 1 : 0;
     p.trace = (g_trace && 2 + barriers_needed(a) + 3 < kTraceSlots) ? w.trace : nullptr;
     CUDA_OK(cudaMemsetAsync(w.sync, 0, w.sync_bytes, st));
+    cudaEvent_t prof_stop;
+    if (prof_begin(st, &prof_stop)) return SSD_E_CUDA;
     int rc = launch_forward_rows(p, Rk, st);
+    if (!rc && prof_end(st, prof_stop)) return SSD_E_CUDA;
     if (rc) return rc;
     kv->last_rows = M;
     return SSD_OK;
