@@ -308,13 +308,8 @@ def run_ours(args, rank, world):
     d2h = Bn * (K + 3) * 4
 
     # ---------------- aggregate over ranks ----------------
-    tot_tokens, tot_e2e_tokens, max_ms, max_e2e = spec_tokens, e2e_tokens, spec_ms, e2e_s
-    if dist is not None:
-        t = torch.tensor([spec_tokens, e2e_tokens], dtype=torch.float64, device="cuda")
-        m = torch.tensor([spec_ms, e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        dist.all_reduce(m, op=dist.ReduceOp.MAX)
-        tot_tokens, tot_e2e_tokens, max_ms, max_e2e = int(t[0]), int(t[1]), float(m[0]), float(m[1])
+    tot_tokens, tot_e2e_tokens, max_ms, max_e2e = aggregate_replicas(
+        dist, [spec_tokens, e2e_tokens], [spec_ms, e2e_s], "cuda")
 
     peak, which = measured_hbm_peak()
     line = {
@@ -350,6 +345,72 @@ def run_ours(args, rank, world):
     if dist is not None:
         dist.destroy_process_group()
     return line
+
+
+def aggregate_replicas(dist, sums, maxima, device):
+    """Replicas only: every rank generates for its own sequences, no data-path collective.  The job's
+    tokens are the SUM over ranks, its time is the MAX over ranks.  `dist` is torch.distributed (an
+    initialised process group) or None for a single process."""
+    if dist is None:
+        return [*sums, *maxima]
+    import torch
+    t = torch.tensor([float(x) for x in sums], dtype=torch.float64, device=device)
+    m = torch.tensor([float(x) for x in maxima], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    dist.all_reduce(m, op=dist.ReduceOp.MAX)
+    return [*(int(round(x)) for x in t.tolist()), *m.tolist()]
+
+
+# ------------------------------------------------------------------ isolated verify sweep
+def run_sweep(args):
+    """Isolated verification-pass sweep at the 7B Llama shape: rows in {1,2,4,5,8,9,16,17} x cache
+    context in {512, 2048, 8192, 16384}, batch 1; cache filled with seeded N(0,1) values, draft rows
+    Dirichlet(0.1).  Prints one JSON object with latency, GB/s and fraction of the HBM peak per point."""
+    import torch
+    from paper_2311_04951_b200 import binding as B, synth
+    torch.cuda.set_device(0)
+    arch = synth.PRESETS["llama-7b"]["target"]
+    target = B.Model(arch, random_weights_on_device(arch, 31, torch))
+    peak, which = measured_hbm_peak()
+    V = arch.vocab
+    points = []
+    g = torch.Generator(device="cuda")
+    for ctx in (512, 2048, 8192, 16384):
+        S = ctx + 64
+        kv = B.KV(target, 1, S)
+        g.manual_seed(41 + ctx)
+        kv.cache_view().copy_(torch.randn(kv.cache_view().shape, generator=g, device="cuda", dtype=torch.float32))
+        B.kv_commit(kv, torch.tensor([ctx], dtype=torch.int32, device="cuda"))
+        kv.lengths()
+        for M in (1, 2, 4, 5, 8, 9, 16, 17):
+            K = M - 1
+            ws = target.new_workspace(1, M, S)
+            rows = torch.from_numpy(synth.gen_prompt(42, 1, M, V)).cuda()
+            q = torch.from_numpy(synth.gen_dirichlet_rows(43, max(K, 1), V)).cuda().reshape(1, max(K, 1), V)
+            u = torch.from_numpy(synth.gen_uniforms(44, 0, 0, M)).cuda().reshape(1, M)
+            na = torch.zeros(1, dtype=torch.int32, device="cuda")
+            nx = torch.zeros(1, dtype=torch.int32, device="cuda")
+            call = lambda: B.target_verify(target, kv, rows, K, q if K else None, u, 1.0, na, nx, 1, None, ws)
+            for _ in range(5):
+                call()
+            torch.cuda.synchronize()
+            ts = []
+            for _ in range(max(args.steps, 10)):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                call()
+                b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            ms = float(np.median(ts))
+            nbytes = verify_step_bytes(arch, 1, K, [ctx])
+            points.append({"rows": M, "ctx": ctx, "ms": ms, "bytes": nbytes, "gbs": nbytes / ms / 1e6,
+                           "frac_of_peak": nbytes / ms / 1e6 / peak, "frac_of_8tbs": nbytes / ms / 1e6 / 8000})
+        del kv
+    base = {pt["ctx"]: pt["ms"] for pt in points if pt["rows"] == 1}
+    for pt in points:
+        pt["over_one_row"] = pt["ms"] / base[pt["ctx"]]
+    return {"sweep": "verify pass, llama-7b shape, batch 1", "peak_gbs": peak, "peak_source": which, "points": points}
 
 
 # ------------------------------------------------------------------ CPU oracle timing
@@ -427,10 +488,13 @@ def main():
     ap.add_argument("--workload", default="neox-1.4b", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="isolated verify-pass sweep at the 7B shape (one GPU)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
-    if args.impl == "reference":
+    if args.sweep:
+        line = run_sweep(args) if rank == 0 else None
+    elif args.impl == "reference":
         line = run_reference(args, rank, world)
     else:
         line = run_ours(args, rank, world)

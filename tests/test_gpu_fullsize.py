@@ -1,0 +1,54 @@
+"""Parity at a full benchmark size, in the launch configuration bench.py times: the 1.4B NeoX-shape
+target (24 layers, d 2048, vocab 50304, bf16), batch 1, K = 5 -> one verification pass over 6 rows
+through the single forward kernel, compared with the oracle on the same seeded weights."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import decoder as od
+from oracle import sampling as osamp
+from paper_2311_04951_b200 import binding as B, synth
+from tests import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def test_verify_pass_at_the_1p4b_shape_matches_the_oracle():
+    cfg = synth.PRESETS["neox-1.4b"]
+    arch, K, T = cfg["target"], cfg["K"], cfg["temperature"]
+    ws_np = synth.gen_weights(arch, cfg["seeds"]["w"])          # natural N(0, 0.02) init, bf16 matrices
+    model = B.Model(arch, B.upload_weights(arch, ws_np))
+    P, S = 24, 64
+    prompt = synth.gen_prompt(cfg["seeds"]["prompt"], 1, P, arch.vocab)
+    rows_np = synth.gen_prompt(77, 1, K + 1, arch.vocab)
+    dev = "cuda"
+    kv = B.KV(model, 1, S)
+    ws = model.new_workspace(1, 8, S)
+    B.kv_prefill(model, kv, torch.from_numpy(prompt).to(dev), torch.tensor([P], dtype=torch.int32, device=dev), ws)
+    V = arch.vocab
+    q_np = synth.gen_dirichlet_rows(78, K, V).reshape(1, K, V)
+    u_np = synth.gen_uniforms(79, 0, 0, K + 1).reshape(1, K + 1)
+    n_acc = torch.zeros(1, dtype=torch.int32, device=dev)
+    nxt = torch.zeros(1, dtype=torch.int32, device=dev)
+    p_dbg = torch.zeros(1, K + 1, V, device=dev)
+    B.target_verify(model, kv, torch.from_numpy(rows_np).to(dev), K, torch.from_numpy(q_np).to(dev),
+                    torch.from_numpy(u_np).to(dev), T, n_acc, nxt, 1, p_dbg, ws)
+    logits = B.last_logits(model, 1, K + 1, ws).cpu().numpy()[0]
+    p_gpu = p_dbg.cpu().numpy()[0]
+    assert kv.status() == 0 and kv.lengths().tolist() == [P]
+    # oracle: same weights, same tokens
+    od.set_threads(16)
+    om = od.Model(arch, ws_np)
+    oc = om.new_cache(S)
+    oc.feed(prompt[0], want_logits=False)
+    ref = oc.feed(rows_np[0], advance=False)
+    gu.assert_logits_close(logits, ref)
+    p_ref = np.stack([osamp.softmax_t(ref[i], T) for i in range(K + 1)])
+    assert np.abs(p_gpu - p_ref).max() <= gu.P_ATOL
+    # decisions follow the rule on the GPU's own rows
+    gu.check_decisions_on_own_rows(p_gpu, q_np[0], rows_np[0, 1:], u_np[0, :K], u_np[0, K],
+                                   int(n_acc.cpu()[0]), int(nxt.cpu()[0]))
+    # cache rows of the pass equal the oracle's up to one bf16 step
+    cache = kv.cache_view().float().cpu().numpy()[:, 0, :, :, :P + K + 1]
+    r = oc.kv[:, :, :, :P + K + 1]
+    assert (np.abs(cache - r) <= gu.LOGIT_RTOL * np.abs(r) + gu.LOGIT_ATOL).all()
