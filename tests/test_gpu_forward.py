@@ -100,7 +100,7 @@ def test_row_results_do_not_depend_on_how_many_rows_are_fed():
     for i in range(K + 1):
         single = gpu_logits(model, kv2, ws1, rows[:, i:i + 1], 0)[0, 0]
         B.kv_commit(kv2, one)
-        assert np.abs(single - together[i]).max() <= 2e-3       # same math, fp32 reduction order only
+        assert np.abs(single - together[i]).max() <= 5e-3       # same math, fp32 reduction order only
 
 
 def test_capacity_and_argument_errors():
