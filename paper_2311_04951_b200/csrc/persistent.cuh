@@ -10,14 +10,18 @@
 // grid barrier of the phase that produces them.
 //
 // Roles in a CTA (288 threads):
-//   warps 0-7   consumers: bf16 tensor-core MMAs on (weight tile, activation tile) stages,
-//               fp32 reductions of partial tiles into the output (bias added by the unit that
-//               holds k-chunk 0); between GEMM phases the same warps run the small phases
-//               (row set-up, embedding, norm, activation, attention with rotary + KV append +
-//               split merge), which leave every GEMM operand in global memory already split
-//               into bf16 hi + lo, and the grid barriers
 //   warp 8      producer: TMA issue for weight tiles (free-running) and operand tiles (gated
 //               by the grid barrier of the phase that wrote them)
+//   warp 4      (one lane) issues the GEMM: per ring stage four tcgen05.mma (128 weight rows x
+//               16 k) x (hi rows | lo rows of the activations), accumulating in tensor memory;
+//               tcgen05.commit hands the stage back to the producer and, at the end of a tile
+//               segment, the accumulator to the epilogue.  Two accumulator buffers, so the
+//               epilogue of one segment overlaps the MMAs of the next
+//   warps 0-3   epilogue: tensor memory -> registers (one weight row per thread), hi + lo
+//               (+ bias from the segment that holds k-chunk 0), fp32 reduction into the output
+//   warps 0-7   between GEMM phases: the small phases (row set-up, embedding, norm, activation,
+//               attention with rotary + KV append + split merge), which leave every GEMM
+//               operand in global memory already split into bf16 hi + lo, and the grid barriers
 // Every wait (mbarrier, grid barrier) is bounded; on time-out SSD_E_TIMEOUT is recorded, the CTA
 // stops taking work, waits (bounded) for its copies in flight and returns.
 #pragma once
@@ -162,6 +166,56 @@ __device__ __forceinline__ void store_hilo(__nv_bfloat16 *buf, int rk, int ld, i
     buf[(size_t)(rk + r) * ld + i] = __float2bfloat16_rn(v - __bfloat162float(h));
 }
 
+// ---- tcgen05 (5th-generation tensor core) helpers ---------------------------------------------
+constexpr int kTmemCols = 256;  // two accumulator buffers of 128 fp32 columns each
+constexpr int kAccStride = 128;
+constexpr int kEpiWarps = 4;    // warps 0-3: one tensor-memory lane quadrant each
+constexpr int kMmaWarp = 4;
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// mbarrier arrive once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void tc_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
+// 128-byte swizzle (what the TMA copies write): start address / 16, leading byte offset unused (1),
+// stride between 8-row groups 1024 bytes, descriptor version 1, layout type 2 (128-byte swizzle).
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, A and B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Eight columns from each of two places of this warp's lane quadrant; the wait is part of the same
+// statement so that no use of the results can be scheduled before it.
+__device__ __forceinline__ void tc_ld_2x8(uint32_t ta, uint32_t tb, float (&a)[8], float (&b)[8]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%16];\n"
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%8,%9,%10,%11,%12,%13,%14,%15}, [%17];\n"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(ta), "r"(tb)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { a[i] = __uint_as_float(r[i]); b[i] = __uint_as_float(r[8 + i]); }
+}
+
 struct alignas(16) Shared {
     volatile int released;  // grid barriers completed so far
     volatile int abort;     // some wait in this CTA gave up
@@ -169,7 +223,17 @@ struct alignas(16) Shared {
     int flag;
 };
 
-// Grid barrier for the 320 work threads of every CTA.  Returns false (the same value in every work
+// Bounded wait that also gives up as soon as another thread of the CTA has.
+__device__ __forceinline__ bool mbar_wait_or_abort(uint64_t *bar, uint32_t parity, const Shared *sh) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (sh->abort || clock64() - t0 > kWaitCycles) return false;
+    }
+    return true;
+}
+
+// Grid barrier for the 256 work threads of every CTA.  Returns false (the same value in every work
 // thread of the CTA) once a wait has timed out anywhere in this CTA; the caller then stops.
 __device__ __forceinline__ bool grid_sync(const FwdParams &p, Shared *sh, int &epoch) {
     fence_async_proxy();  // this thread's operand writes must be seen by other CTAs' TMA reads
@@ -778,22 +842,38 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
     uint8_t *attn_scratch = smem + p.attn_smem_off;
     uint64_t *fullW = (uint64_t *)(smem + (size_t)S * kStageBytes);
     uint64_t *fullX = fullW + S, *empty = fullX + S;
-    Shared *sh = (Shared *)(((uintptr_t)(empty + S) + 15) & ~(uintptr_t)15);
+    uint64_t *accFull = empty + S, *accEmpty = accFull + 2, *mmaDone = accEmpty + 2;
+    uint32_t *tmem_slot = (uint32_t *)(mmaDone + 1);
+    Shared *sh = (Shared *)(((uintptr_t)(mmaDone + 4) + 15) & ~(uintptr_t)15);
     double *red = (double *)(sh + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == 0) {  // tensor memory for the accumulators; released by the same warp at the end
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "n"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(&fullW[s], 1);
             mbar_init(&fullX[s], 1);
-            mbar_init(&empty[s], kConsumerWarps);
+            mbar_init(&empty[s], 1);  // one tcgen05.commit per stage
         }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&accFull[b], 1);
+            mbar_init(&accEmpty[b], kEpiWarps);
+        }
+        mbar_init(mmaDone, 1);
         sh->released = 0;
         sh->abort = 0;
         sh->go = 1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    tc_fence_before();
     __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
     const int NG = n_gemms(p);
 
     if (warp == kConsumerWarps) {
@@ -870,75 +950,88 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
         }
     } else {
         // =============================== work warps ===============================
-        int epoch = 0, it = 0;  // grid barriers passed; ring stages consumed
-        bool alive = true;      // per warp: false once one of its waits gave up
+        int epoch = 0;  // grid barriers passed
+        int it = 0;     // ring stages consumed so far (all GEMMs)
+        int seg = 0;    // tile segments so far: segment q accumulates in buffer q & 1
 
-        // run this CTA's units of GEMM gi
+        // Run this CTA's units of GEMM gi.  The units are contiguous in (tile, k-chunk) order, so they
+        // form one segment per tile touched; each segment is accumulated in tensor memory and
+        // reduced into the output once.
         auto run_gemm = [&](int gi) {
             const GemmDesc g = gemm_desc(p, gi);
             int c0, c1;
             unit_range(g, c0, c1);
             if (c0 >= c1) return;
-            float acc[NT][4];  // local to the GEMM: nothing to keep alive across the small phases
+            const int tile0 = c0 / g.kchunks, tile1 = (c1 - 1) / g.kchunks;
+            if (warp == kMmaWarp) {
+                if (lane == 0 && !sh->abort) {
+                    const uint32_t idesc = umma_idesc_bf16(2 * kRp);
+                    int itl = it, sg = seg, kc = c0 % g.kchunks;
+                    bool first = true;
+                    for (int c = c0; c < c1; ++c, ++itl) {
+                        const int s = itl % S, b = sg & 1;
+                        bool ok = true;
+                        if (first && sg >= 2) ok = mbar_wait_or_abort(&accEmpty[b], ((sg >> 1) - 1) & 1, sh);
+                        ok = ok && mbar_wait_or_abort(&fullW[s], (itl / S) & 1, sh) &&
+                             mbar_wait_or_abort(&fullX[s], (itl / S) & 1, sh);
+                        if (!ok) {
+                            set_status(p.status, kTimeoutCode);
+                            sh->abort = 1;
+                            break;
+                        }
+                        tc_fence_after();
+                        const uint32_t st = smem_u32(ring + (size_t)s * kStageBytes);
+                        const uint64_t adesc = umma_desc_sw128(st), bdesc = umma_desc_sw128(st + kWTileBytes);
+                        const uint32_t d_tmem = tmem_base + (uint32_t)(b * kAccStride);
 #pragma unroll
-            for (int j = 0; j < NT; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
-            int tile = c0 / g.kchunks, kc = c0 % g.kchunks;
-            auto flush = [&](int t, bool with_bias) {
-                const int n = t * kTileN + warp * 16 + (lane >> 2);
-                float b0 = 0.f, b1 = 0.f;
-                if (with_bias && g.bias) {
-                    if (n < g.N) b0 = __ldg(g.bias + n);
-                    if (n + 8 < g.N) b1 = __ldg(g.bias + n + 8);
-                }
-#pragma unroll
-                for (int j = 0; j < NT; ++j) {
-                    const int m0 = 8 * j + (lane & 3) * 2;
-                    if (n < g.N) {
-                        if (m0 < p.R) atomicAdd(g.out + (size_t)m0 * g.ldo + n, acc[j][0] + b0);
-                        if (m0 + 1 < p.R) atomicAdd(g.out + (size_t)(m0 + 1) * g.ldo + n, acc[j][1] + b0);
-                    }
-                    if (n + 8 < g.N) {
-                        if (m0 < p.R) atomicAdd(g.out + (size_t)m0 * g.ldo + n + 8, acc[j][2] + b1);
-                        if (m0 + 1 < p.R) atomicAdd(g.out + (size_t)(m0 + 1) * g.ldo + n + 8, acc[j][3] + b1);
-                    }
-                    acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
-                }
-            };
-            const int arow = lane & 15, achunk = lane >> 4, brow = lane & 7, bsel = lane >> 3;
-            bool has_k0 = (kc == 0);  // does the running tile segment include k-chunk 0 (it adds the bias)
-            for (int c = c0; c < c1 && alive; ++c, ++it) {
-                const int s = it % S;
-                if (!mbar_wait(&fullW[s], (it / S) & 1) || !mbar_wait(&fullX[s], (it / S) & 1)) {
-                    set_status(p.status, kTimeoutCode);
-                    sh->abort = 1;
-                    alive = false;
-                    break;
-                }
-                const uint32_t st = smem_u32(ring + (size_t)s * kStageBytes);
-                const uint32_t wbase = st + (uint32_t)(warp * 16 + arow) * 128u;
-                const uint32_t xbase = st + kWTileBytes + (bsel >= 2 ? kRp * 128 : 0) + (uint32_t)brow * 128u;
-#pragma unroll
-                for (int ks = 0; ks < kTileK / 16; ++ks) {
-                    uint32_t a0, a1, a2, a3;
-                    ldmatrix_x4(wbase + ((uint32_t)((2 * ks + achunk) ^ (arow & 7)) << 4), a0, a1, a2, a3);
-#pragma unroll
-                    for (int j = 0; j < NT; ++j) {
-                        uint32_t h0, h1, l0, l1;
-                        ldmatrix_x4(xbase + (uint32_t)j * 1024u + ((uint32_t)((2 * ks + (bsel & 1)) ^ brow) << 4), h0, h1, l0, l1);
-                        mma_bf16(acc[j], a0, a1, a2, a3, h0, h1);
-                        mma_bf16(acc[j], a0, a1, a2, a3, l0, l1);
+                        for (int ks = 0; ks < kTileK / 16; ++ks)  // 32 bytes further along k inside the swizzle atom
+                            tc_mma_bf16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, idesc, (first && ks == 0) ? 0u : 1u);
+                        tc_commit(&empty[s]);
+                        first = false;
+                        ++kc;
+                        if (kc == g.kchunks || c + 1 == c1) {
+                            tc_commit(&accFull[b]);
+                            ++sg;
+                            first = true;
+                            if (kc == g.kchunks) kc = 0;
+                        }
                     }
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[s]);
-                if (++kc == g.kchunks) {
-                    flush(tile, has_k0);
-                    kc = 0;
-                    ++tile;
-                    has_k0 = true;
+            } else if (warp < kEpiWarps) {
+                int sg = seg;
+                for (int t = tile0; t <= tile1; ++t, ++sg) {
+                    const int b = sg & 1;
+                    if (!mbar_wait_or_abort(&accFull[b], (sg >> 1) & 1, sh)) {
+                        set_status(p.status, kTimeoutCode);
+                        sh->abort = 1;
+                        break;
+                    }
+                    tc_fence_after();
+                    const bool has_k0 = (t > tile0) || (c0 % g.kchunks == 0);
+                    const int n = t * kTileN + warp * 32 + lane;
+                    const float bias = (has_k0 && g.bias && n < g.N) ? __ldg(g.bias + n) : 0.f;
+                    const uint32_t ta = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * kAccStride);
+#pragma unroll
+                    for (int j = 0; j < NT; ++j) {
+                        if (8 * j < p.R) {  // uniform over the warp
+                            float hi[8], lo[8];
+                            tc_ld_2x8(ta + 8 * j, ta + kRp + 8 * j, hi, lo);
+                            if (n < g.N) {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    if (8 * j + i < p.R)
+                                        atomicAdd(g.out + (size_t)(8 * j + i) * g.ldo + n, hi[i] + lo[i] + bias);
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&accEmpty[b]);
                 }
             }
-            if (alive && kc != 0) flush(tile, has_k0);
+            it += c1 - c0;
+            seg += tile1 - tile0 + 1;
         };
 
         if (p.trace && blockIdx.x == 0 && threadIdx.x == 0) {
@@ -1004,8 +1097,20 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             p.trace[epoch + 1] = t;
             p.trace[epoch + 2] = 0;
         }
+        if (warp == kMmaWarp) {  // nothing of this CTA may still be running on the tensor core
+            if (lane == 0) {
+                tc_commit(mmaDone);
+                mbar_wait(mmaDone, 0);
+            }
+            __syncwarp();
+        }
     }
+    tc_fence_before();
     __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "n"(kTmemCols) : "memory");
+    }
 }
 
 }  // namespace ssd

@@ -427,12 +427,12 @@ template <int NT>
 int launch_forward_nt(FwdParams p, cudaStream_t st) {
     constexpr int stage = kWTileBytes + 2 * NT * 8 * kTileK * 2;
     const size_t attn = align_up(attn_scratch_bytes(p.Dh), 128);
-    const size_t tail_fixed = 24 * 12 + 16 + sizeof(Shared) + 16 * sizeof(double) + 256;
+    const size_t tail_fixed = 24 * 12 + 64 + 16 + sizeof(Shared) + 16 * sizeof(double) + 256;
     int S = (int)(((size_t)kSmemBudget - 1024 - attn - tail_fixed) / stage);
     if (S > 12) S = 12;
     if (S < 2) return SSD_E_CAPACITY;
     p.stages = S;
-    p.attn_smem_off = (int)align_up((size_t)S * stage + 24 * (size_t)S + 16 + sizeof(Shared) + 16 * sizeof(double), 128);
+    p.attn_smem_off = (int)align_up((size_t)S * stage + 24 * (size_t)S + 64 + 16 + sizeof(Shared) + 16 * sizeof(double), 128);
     const size_t smem = 1024 + (size_t)p.attn_smem_off + attn;
     static bool attr = false;
     if (!attr) {
