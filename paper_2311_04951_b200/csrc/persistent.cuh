@@ -10,8 +10,9 @@
 // grid barrier of the phase that produces them.
 //
 // Roles in a CTA (288 threads):
-//   warp 8      producer: TMA issue for weight tiles (free-running) and operand tiles (gated
-//               by the grid barrier of the phase that wrote them)
+//   warp 8      producer: TMA issue for weight tiles, free-running across phase boundaries
+//   warp 5      (one lane) during a GEMM phase: bulk copies of that GEMM's operand tiles, which
+//               exist only once the grid barrier of the phase that wrote them has been passed
 //   warp 4      (one lane) issues the GEMM: per ring stage four tcgen05.mma (128 weight rows x
 //               16 k) x (hi rows | lo rows of the activations), accumulating in tensor memory;
 //               tcgen05.commit hands the stage back to the producer and, at the end of a tile
@@ -56,11 +57,13 @@ __device__ __forceinline__ const LayerDesc *layer_desc(const ModelDesc *md, int 
 enum { OP_XN1 = 0, OP_XN2 = 1, OP_AO = 2, OP_ACT = 3 };
 
 struct alignas(64) FwdParams {
-    // GEMM operands in global memory, bf16 hi rows [0, rk) then lo rows [rk, 2 rk), row pitch = K:
-    // normalised rows (two sets for parallel-residual blocks), attention output, MLP activation.
-    CUtensorMap tm_op[4];  // box 64 x (2 rk), 128-byte swizzle
+    // GEMM operands in global memory (normalised rows - two sets for parallel-residual blocks -,
+    // attention output, MLP activation), stored the way a ring stage wants them: one contiguous
+    // tile per 64-wide k-chunk, 2 rk rows of 128 bytes (bf16 hi rows [0, rk), lo rows [rk, 2 rk)),
+    // 16-byte chunks already in 128-byte-swizzle order, so one linear bulk copy fetches a tile.
+    // (A strided 2-D tensor copy of the same tile costs a sixth of the weight stream's bandwidth.)
     __nv_bfloat16 *op[4];
-    int op_ld[4];
+    int op_ld[4];  // K of each operand
     int rk;
     const ModelDesc *md;
     // architecture
@@ -87,14 +90,20 @@ struct alignas(64) FwdParams {
     unsigned *gbar;     // grid barrier counter (zeroed before launch)
     int chunk, n_split;
     int want_logits;
-    int stages, attn_smem_off;  // ring depth; byte offset of the attention scratch
+    // Shared-memory ring: slots [0, stages_lo) hold weights at any time; slots [stages_lo, stages) share
+    // their bytes with the attention scratch (at attn_smem_off = stages_lo * stage bytes) and are used
+    // only between attention phases.  bar_off: byte offset of the barriers behind both.
+    int stages, stages_lo, attn_smem_off, bar_off;
     unsigned long long *trace;  // optional: CTA 0 stamps the global timer after every grid barrier
 };
 
 struct GemmDesc {
-    const CUtensorMap *tmW, *tmX;
+    const CUtensorMap *tmW;
+    const __nv_bfloat16 *xop;  // tiled operand
     int N, Kd, n_tiles, kchunks;
     int need;  // grid barriers that must have completed before its operand exists
+    int need_hi;  // ... before its tiles may use the ring slots shared with the attention scratch
+    int kind;     // 0 qkv, 1 o, 2 in, 3 out, 4 LM head
     float *out;
     int ldo;
     const float *bias;
@@ -112,25 +121,30 @@ __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi) {
     const int l = gi >> 2, e = gi & 3;
     const int base = 2 + barriers_per_layer(p) * l;
     if (l >= p.n_layers) {  // LM head
-        g.tmW = &p.md->tm_lm; g.tmX = &p.tm_op[OP_XN1];
+        g.tmW = &p.md->tm_lm; g.xop = p.op[OP_XN1];
         g.N = p.V; g.Kd = p.d; g.need = base; g.out = p.logits; g.ldo = p.V; g.bias = nullptr;
+        g.kind = 4; g.need_hi = base - barriers_per_layer(p) + 2;  // end of the last attention phase
     } else {
         const LayerDesc *ld = layer_desc(p.md, l);
         int kind;  // 0 qkv, 1 o, 2 in, 3 out
         if (p.parallel) kind = (e == 0) ? 0 : (e == 1) ? 2 : (e == 2) ? 1 : 3;
         else kind = e;
         g.tmW = &ld->tm[kind];
+        g.kind = kind;
+        // the attention phase of layer l ends at barrier base + 2; qkv precedes it (previous layer's counts)
+        // (so does the MLP input GEMM of a parallel-residual block)
+        g.need_hi = (kind == 0 || (kind == 2 && p.parallel)) ? (l == 0 ? 0 : base - barriers_per_layer(p) + 2) : base + 2;
         if (kind == 0) {
-            g.tmX = &p.tm_op[OP_XN1]; g.N = 3 * p.d; g.Kd = p.d; g.need = base;
+            g.xop = p.op[OP_XN1]; g.N = 3 * p.d; g.Kd = p.d; g.need = base;
             g.out = p.qkv; g.ldo = 3 * p.d; g.bias = ld->b_qkv;
         } else if (kind == 1) {
-            g.tmX = &p.tm_op[OP_AO]; g.N = p.d; g.Kd = p.d; g.need = base + 2;
+            g.xop = p.op[OP_AO]; g.N = p.d; g.Kd = p.d; g.need = base + 2;
             g.out = p.x; g.ldo = p.d; g.bias = ld->b_o;
         } else if (kind == 2) {
-            g.tmX = &p.tm_op[p.parallel ? OP_XN2 : OP_XN1]; g.N = p.d_in; g.Kd = p.d; g.need = p.parallel ? base : base + 4;
+            g.xop = p.op[p.parallel ? OP_XN2 : OP_XN1]; g.N = p.d_in; g.Kd = p.d; g.need = p.parallel ? base : base + 4;
             g.out = p.t_in; g.ldo = p.d_in; g.bias = ld->b_in;
         } else {
-            g.tmX = &p.tm_op[OP_ACT]; g.N = p.d; g.Kd = p.F; g.need = p.parallel ? base + 2 : base + 6;
+            g.xop = p.op[OP_ACT]; g.N = p.d; g.Kd = p.F; g.need = p.parallel ? base + 2 : base + 6;
             g.out = p.x; g.ldo = p.d; g.bias = ld->b_out;
         }
     }
@@ -159,11 +173,22 @@ __device__ __forceinline__ void red_release_add(unsigned *p, unsigned v) {
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// operand element (r, i) of a hi/lo buffer
-__device__ __forceinline__ void store_hilo(__nv_bfloat16 *buf, int rk, int ld, int r, int i, float v) {
+// Element offset of (row, column i) in a tiled operand: row in [0, 2 rk) (hi rows, then lo rows).
+__device__ __forceinline__ size_t op_off(int rk, int row, int i) {
+    const int kc = i >> 6, w = i & 63;
+    return (size_t)kc * (size_t)(2 * rk * kTileK) + (size_t)(row * kTileK + ((((w >> 3) ^ (row & 7)) << 3) | (w & 7)));
+}
+// operand element (r, i) as hi + lo
+__device__ __forceinline__ void store_hilo(__nv_bfloat16 *buf, int rk, int r, int i, float v) {
     const __nv_bfloat16 h = __float2bfloat16_rn(v);
-    buf[(size_t)r * ld + i] = h;
-    buf[(size_t)(rk + r) * ld + i] = __float2bfloat16_rn(v - __bfloat162float(h));
+    buf[op_off(rk, r, i)] = h;
+    buf[op_off(rk, rk + r, i)] = __float2bfloat16_rn(v - __bfloat162float(h));
+}
+__device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
 }
 
 // ---- tcgen05 (5th-generation tensor core) helpers ---------------------------------------------
@@ -171,6 +196,7 @@ constexpr int kTmemCols = 256;  // two accumulator buffers of 128 fp32 columns e
 constexpr int kAccStride = 128;
 constexpr int kEpiWarps = 4;    // warps 0-3: one tensor-memory lane quadrant each
 constexpr int kMmaWarp = 4;
+constexpr int kXWarp = 5;      // issues the operand copies of a GEMM phase
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -215,6 +241,25 @@ __device__ __forceinline__ void tc_ld_2x8(uint32_t ta, uint32_t tb, float (&a)[8
 #pragma unroll
     for (int i = 0; i < 8; ++i) { a[i] = __uint_as_float(r[i]); b[i] = __uint_as_float(r[8 + i]); }
 }
+
+// Slot schedule of the ring, identical in every role that walks it (weight producer, operand issuer,
+// MMA issuer).  Unit j of this CTA's share of a GEMM takes the next slot of the full cycle, except
+// the first stages_lo units of an out-projection - the ones fetched while the attention phase still
+// owns the upper slots - which cycle through the lower slots only.  One parity bit per slot.
+struct RingPos {
+    int pos_all = 0, pos_lo = 0;
+    uint32_t par = 0, used = 0;
+};
+__device__ __forceinline__ int ring_next(RingPos &r, bool lo_only, int S, int S1, uint32_t &parity) {
+    int s;
+    if (lo_only) { s = r.pos_lo; if (++r.pos_lo == S1) r.pos_lo = 0; }
+    else { s = r.pos_all; if (++r.pos_all == S) r.pos_all = 0; }
+    parity = (r.par >> s) & 1u;
+    r.par ^= 1u << s;
+    r.used |= 1u << s;
+    return s;
+}
+__device__ __forceinline__ bool ring_lo_only(const GemmDesc &g, int j, int S1) { return g.kind == 1 && j < S1; }
 
 struct alignas(16) Shared {
     volatile int released;  // grid barriers completed so far
@@ -359,8 +404,8 @@ __device__ __noinline__ void norm_phase(const FwdParams &p, const float *g1, con
             const __nv_bfloat162 h01 = __floats2bfloat162_rn(y0, y1), h23 = __floats2bfloat162_rn(y2, y3);
             const __nv_bfloat162 l01 = __floats2bfloat162_rn(y0 - __low2float(h01), y1 - __high2float(h01));
             const __nv_bfloat162 l23 = __floats2bfloat162_rn(y2 - __low2float(h23), y3 - __high2float(h23));
-            __nv_bfloat16 *hi = p.op[op] + (size_t)r * p.op_ld[op] + 4 * i;
-            __nv_bfloat16 *lo = p.op[op] + (size_t)(p.rk + r) * p.op_ld[op] + 4 * i;
+            __nv_bfloat16 *hi = p.op[op] + op_off(p.rk, r, 4 * i);
+            __nv_bfloat16 *lo = p.op[op] + op_off(p.rk, p.rk + r, 4 * i);
             uint2 hv, lv;
             hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
             lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
@@ -406,12 +451,19 @@ __device__ __noinline__ void act_phase(const FwdParams &p) {
         hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
         lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
         __nv_bfloat16 *base = p.op[OP_ACT];
-        *reinterpret_cast<uint2 *>(base + (size_t)r * p.op_ld[OP_ACT] + 4 * c) = hv;
-        *reinterpret_cast<uint2 *>(base + (size_t)(p.rk + r) * p.op_ld[OP_ACT] + 4 * c) = lv;
+        *reinterpret_cast<uint2 *>(base + op_off(p.rk, r, 4 * c)) = hv;
+        *reinterpret_cast<uint2 *>(base + op_off(p.rk, p.rk + r, 4 * c)) = lv;
     }
 }
 
 __device__ __noinline__ void setup_phase(const FwdParams &p) {
+    // K not a multiple of 64: the last tile's unused columns must be finite (the weight copy zero-fills its own)
+    for (int o = 0; o < 4; ++o) {
+        const int K = p.op_ld[o], pad = (-K) & (kTileK - 1);
+        if (!p.op[o] || !pad) continue;
+        for (int e = blockIdx.x * kWorkThreads + threadIdx.x; e < 2 * p.rk * pad; e += gridDim.x * kWorkThreads)
+            p.op[o][op_off(p.rk, e / pad, K + e % pad)] = __float2bfloat16_rn(0.f);
+    }
     const int half = p.rotary_dim / 2;
     for (int r = blockIdx.x; r < p.R; r += gridDim.x) {
         const int b = r / p.M, j = r % p.M;
@@ -781,7 +833,7 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
         const int gs = kAttnRows * Dh;  // stride between position groups
         const float osum = (o_acc[i] + o_acc[i + gs]) + (o_acc[i + 2 * gs] + o_acc[i + 3 * gs]);
         if (direct) {
-            store_hilo(p.op[OP_AO], p.rk, p.op_ld[OP_AO], r0 + m, h * Dh + e, live ? osum / L : 0.f);
+            store_hilo(p.op[OP_AO], p.rk, r0 + m, h * Dh + e, live ? osum / L : 0.f);
         } else {
             const size_t slot = ((size_t)(r0 + m) * p.H + h) * p.n_split + split;
             if (e == 0) {
@@ -814,7 +866,7 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
                         acc = fmaf(__ldcg(p.part_o + (base + s2) * Dh + e), w, acc);
                     }
                 }
-                store_hilo(p.op[OP_AO], p.rk, p.op_ld[OP_AO], r0 + m, h * Dh + e, L > 0.f ? acc / L : 0.f);
+                store_hilo(p.op[OP_AO], p.rk, r0 + m, h * Dh + e, L > 0.f ? acc / L : 0.f);
             }
             if (tid == 0) p.tickets[bh] = 0;  // ready for the next layer (a grid barrier lies between)
         }
@@ -837,10 +889,10 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
     constexpr int kRp = NT * 8;
     constexpr int kXBytes = 2 * kRp * kTileK * 2;  // hi tile followed by lo tile
     constexpr int kStageBytes = kWTileBytes + kXBytes;
-    const int S = p.stages;
+    const int S = p.stages, S1 = p.stages_lo;
     uint8_t *ring = smem;
     uint8_t *attn_scratch = smem + p.attn_smem_off;
-    uint64_t *fullW = (uint64_t *)(smem + (size_t)S * kStageBytes);
+    uint64_t *fullW = (uint64_t *)(smem + p.bar_off);
     uint64_t *fullX = fullW + S, *empty = fullX + S;
     uint64_t *accFull = empty + S, *accEmpty = accFull + 2, *mmaDone = accEmpty + 2;
     uint32_t *tmem_slot = (uint32_t *)(mmaDone + 1);
@@ -878,80 +930,54 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
 
     if (warp == kConsumerWarps) {
         // =============================== producer ===============================
-        // Two cursors over the same unit sequence.  Weights never change, so their cursor runs as far
-        // ahead as the ring allows, across grid barriers; an operand tile is fetched once the phase
-        // that wrote it has been released.
+        // Weights never change, so this cursor runs as far ahead as the ring allows, across grid
+        // barriers.  The loop is kept minimal (no divisions, no clock reads while it makes progress):
+        // its rate bounds the weight stream.
         if (lane == 0) {
-            int issuedW = 0, issuedX = 0;
-            int gw = 0, cw = 0, cw1 = 0, tw = 0, kw = 0;
-            int gx = 0, cx = 0, cx1 = 0, kx = 0;
-            GemmDesc dw, dx;
-            bool have_w = false, have_x = false;
-            auto next_w = [&]() {
-                for (; gw < NG; ++gw) {
-                    dw = gemm_desc(p, gw);
-                    unit_range(dw, cw, cw1);
-                    if (cw < cw1) { tw = cw / dw.kchunks; kw = cw % dw.kchunks; have_w = true; return; }
-                }
-                have_w = false;
-            };
-            auto next_x = [&]() {
-                for (; gx < NG; ++gx) {
-                    dx = gemm_desc(p, gx);
-                    unit_range(dx, cx, cx1);
-                    if (cx < cx1) { kx = cx % dx.kchunks; have_x = true; return; }
-                }
-                have_x = false;
-            };
-            next_w();
-            next_x();
+            RingPos rp;
+            bool failed = false;
             int seen_release = 0;
-            long long idle_since = clock64();
-            while ((have_w || have_x) && !sh->abort) {
-                bool progressed = false;
-                if (have_w) {
-                    const int s = issuedW % S;
-                    if (issuedW < S || mbar_test_wait(&empty[s], ((issuedW / S) - 1) & 1)) {
-                        mbar_expect_tx(&fullW[s], kWTileBytes);
-                        tma_load_2d(ring + (size_t)s * kStageBytes, dw.tmW, kw * kTileK, tw * kTileN, &fullW[s]);
-                        ++issuedW;
-                        progressed = true;
-                        if (++kw == dw.kchunks) { kw = 0; ++tw; }
-                        if (++cw == cw1) { ++gw; next_w(); }
+            for (int gw = 0; gw < NG && !failed; ++gw) {
+                const GemmDesc dw = gemm_desc(p, gw);
+                int c0, c1;
+                unit_range(dw, c0, c1);
+                if (c0 >= c1) continue;
+                int tw = c0 / dw.kchunks, kw = c0 % dw.kchunks;
+                for (int c = c0; c < c1; ++c) {
+                    uint32_t ph;
+                    const int s = ring_next(rp, ring_lo_only(dw, c - c0, S1), S, S1, ph);
+                    if (s >= S1 && seen_release < dw.need_hi) {  // slot shared with the attention scratch
+                        const long long t0 = clock64();
+                        while ((seen_release = sh->released) < dw.need_hi) {
+                            if (sh->abort || clock64() - t0 > kWaitCycles) { failed = true; break; }
+                        }
+                        if (failed) { rp.par ^= 1u << s; break; }  // nothing was issued into s
                     }
-                }
-                if (have_x && issuedX < issuedW) {
-                    if (dx.need > seen_release) {
-                        seen_release = sh->released;
-                        if (dx.need <= seen_release) fence_async_proxy();  // that phase's writes -> visible to TMA
+                    if (!mbar_test_wait(&empty[s], ph ^ 1u)) {
+                        const long long t0 = clock64();
+                        while (!mbar_test_wait(&empty[s], ph ^ 1u)) {
+                            if (sh->abort || clock64() - t0 > kWaitCycles) { failed = true; break; }
+                        }
+                        if (failed) { rp.par ^= 1u << s; break; }  // nothing was issued into s
                     }
-                    if (dx.need <= seen_release) {
-                        const int s = issuedX % S;
-                        mbar_expect_tx(&fullX[s], kXBytes);
-                        tma_load_2d(ring + (size_t)s * kStageBytes + kWTileBytes, dx.tmX, kx * kTileK, 0, &fullX[s]);
-                        ++issuedX;
-                        progressed = true;
-                        if (++kx == dx.kchunks) kx = 0;
-                        if (++cx == cx1) { ++gx; next_x(); }
-                    }
+                    mbar_expect_tx(&fullW[s], kWTileBytes);
+                    tma_load_2d(ring + (size_t)s * kStageBytes, dw.tmW, kw * kTileK, tw * kTileN, &fullW[s]);
+                    if (++kw == dw.kchunks) { kw = 0; ++tw; }
                 }
-                if (progressed) {
-                    idle_since = clock64();
-                } else if (clock64() - idle_since > kWaitCycles) {
-                    set_status(p.status, kTimeoutCode);
-                    sh->abort = 1;
-                }
+            }
+            if (failed) {
+                set_status(p.status, kTimeoutCode);
+                sh->abort = 1;
             }
             // error path only: wait (bounded) for copies still in flight before the CTA may exit
-            if (sh->abort) {
-                for (int i = (issuedW > S ? issuedW - S : 0); i < issuedW; ++i) mbar_wait(&fullW[i % S], (i / S) & 1);
-                for (int i = (issuedX > S ? issuedX - S : 0); i < issuedX; ++i) mbar_wait(&fullX[i % S], (i / S) & 1);
-            }
+            if (sh->abort)
+                for (int s = 0; s < S; ++s)
+                    if ((rp.used >> s) & 1u) mbar_wait(&fullW[s], ((rp.par >> s) & 1u) ^ 1u);
         }
     } else {
         // =============================== work warps ===============================
         int epoch = 0;  // grid barriers passed
-        int it = 0;     // ring stages consumed so far (all GEMMs)
+        RingPos rp;     // this thread's walk of the ring (used by the MMA and the operand issuer)
         int seg = 0;    // tile segments so far: segment q accumulates in buffer q & 1
 
         // Run this CTA's units of GEMM gi.  The units are contiguous in (tile, k-chunk) order, so they
@@ -966,14 +992,14 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             if (warp == kMmaWarp) {
                 if (lane == 0 && !sh->abort) {
                     const uint32_t idesc = umma_idesc_bf16(2 * kRp);
-                    int itl = it, sg = seg, kc = c0 % g.kchunks;
+                    int sg = seg, kc = c0 % g.kchunks;
                     bool first = true;
-                    for (int c = c0; c < c1; ++c, ++itl) {
-                        const int s = itl % S, b = sg & 1;
+                    for (int c = c0; c < c1; ++c) {
+                        uint32_t ph;
+                        const int s = ring_next(rp, ring_lo_only(g, c - c0, S1), S, S1, ph), b = sg & 1;
                         bool ok = true;
                         if (first && sg >= 2) ok = mbar_wait_or_abort(&accEmpty[b], ((sg >> 1) - 1) & 1, sh);
-                        ok = ok && mbar_wait_or_abort(&fullW[s], (itl / S) & 1, sh) &&
-                             mbar_wait_or_abort(&fullX[s], (itl / S) & 1, sh);
+                        ok = ok && mbar_wait_or_abort(&fullW[s], ph, sh) && mbar_wait_or_abort(&fullX[s], ph, sh);
                         if (!ok) {
                             set_status(p.status, kTimeoutCode);
                             sh->abort = 1;
@@ -995,6 +1021,27 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                             first = true;
                             if (kc == g.kchunks) kc = 0;
                         }
+                    }
+                }
+                __syncwarp();
+            } else if (warp == kXWarp) {
+                // operand tiles of this GEMM (their phase has been released: this runs after its barrier)
+                if (lane == 0 && !sh->abort) {
+                    fence_async_proxy();  // that phase's generic-proxy writes -> visible to the bulk copies
+                    int kx = c0 % g.kchunks;
+                    for (int c = c0; c < c1; ++c) {
+                        uint32_t ph;
+                        const int s = ring_next(rp, ring_lo_only(g, c - c0, S1), S, S1, ph);
+                        if (!mbar_wait_or_abort(&empty[s], ph ^ 1u, sh)) {
+                            rp.par ^= 1u << s;  // nothing was issued into s
+                            set_status(p.status, kTimeoutCode);
+                            sh->abort = 1;
+                            break;
+                        }
+                        mbar_expect_tx(&fullX[s], kXBytes);
+                        bulk_load_1d(ring + (size_t)s * kStageBytes + kWTileBytes,
+                                     g.xop + (size_t)kx * (2 * kRp * kTileK), kXBytes, &fullX[s]);
+                        if (++kx == g.kchunks) kx = 0;
                     }
                 }
                 __syncwarp();
@@ -1030,7 +1077,6 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                     if (lane == 0) mbar_arrive(&accEmpty[b]);
                 }
             }
-            it += c1 - c0;
             seg += tile1 - tile0 + 1;
         };
 
@@ -1097,6 +1143,9 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             p.trace[epoch + 1] = t;
             p.trace[epoch + 2] = 0;
         }
+        if (warp == kXWarp && lane == 0 && sh->abort)  // error path only: copies still in flight
+            for (int s = 0; s < S; ++s)
+                if ((rp.used >> s) & 1u) mbar_wait(&fullX[s], ((rp.par >> s) & 1u) ^ 1u);
         if (warp == kMmaWarp) {  // nothing of this CTA may still be running on the tensor core
             if (lane == 0) {
                 tc_commit(mmaDone);

@@ -272,7 +272,7 @@ Workspace carve(const ssd_model *m, int B, int M, uint8_t *base) {
         if (a.dtype == 0) {
             o.f32 = (float *)take(sizeof(float) * (size_t)Rp * ld);
         } else {
-            o.hi = (__nv_bfloat16 *)take(2 * (size_t)2 * Rk * ld);
+            o.hi = (__nv_bfloat16 *)take(2 * (size_t)2 * Rk * align_up((size_t)ld, 64));  // whole 64-wide k tiles
             o.lo = o.hi + (size_t)Rk * ld;
         }
         return o;
@@ -425,15 +425,25 @@ inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 4 
 
 template <int NT>
 int launch_forward_nt(FwdParams p, cudaStream_t st) {
-    constexpr int stage = kWTileBytes + 2 * NT * 8 * kTileK * 2;
+    constexpr size_t stage = kWTileBytes + 2 * NT * 8 * kTileK * 2;
     const size_t attn = align_up(attn_scratch_bytes(p.Dh), 128);
-    const size_t tail_fixed = 24 * 12 + 64 + 16 + sizeof(Shared) + 16 * sizeof(double) + 256;
-    int S = (int)(((size_t)kSmemBudget - 1024 - attn - tail_fixed) / stage);
-    if (S > 12) S = 12;
-    if (S < 2) return SSD_E_CAPACITY;
-    p.stages = S;
-    p.attn_smem_off = (int)align_up((size_t)S * stage + 24 * (size_t)S + 64 + 16 + sizeof(Shared) + 16 * sizeof(double), 128);
-    const size_t smem = 1024 + (size_t)p.attn_smem_off + attn;
+    const size_t tail = 24 * 32 + 64 + 16 + sizeof(Shared) + 16 * sizeof(double) + 256;  // barriers and the small state
+    const size_t total = (size_t)kSmemBudget - 1024 - tail;
+    // upper slots share their bytes with the attention scratch; at least two slots never do
+    size_t S2 = (attn + stage - 1) / stage;
+    size_t region2 = S2 * stage;
+    if (region2 + 2 * stage > total) {
+        S2 = attn / stage;
+        region2 = attn;
+    }
+    if (region2 + 2 * stage > total) return SSD_E_CAPACITY;
+    size_t S1 = (total - region2) / stage;
+    if (S1 + S2 > 32) S1 = 32 - S2;  // one parity bit per slot
+    p.stages = (int)(S1 + S2);
+    p.stages_lo = (int)S1;
+    p.attn_smem_off = (int)(S1 * stage);
+    p.bar_off = (int)align_up(S1 * stage + region2, 128);
+    const size_t smem = 1024 + (size_t)p.bar_off + tail;
     static bool attr = false;
     if (!attr) {
         if (cudaFuncSetAttribute(forward_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) !=
@@ -473,7 +483,6 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     for (int i = 0; i < 4; ++i) {
         p.op[i] = ops[i]->hi;
         p.op_ld[i] = ops[i]->ld;
-        if (ops[i]->hi && make_map(&p.tm_op[i], ops[i]->hi, 2 * Rk, ops[i]->ld, 2 * Rk)) return SSD_E_CUDA;
     }
     p.rk = Rk;
     p.md = m->dev_desc;
