@@ -13,13 +13,18 @@
 //   warp 8      producer: TMA issue for weight tiles, free-running across phase boundaries
 //   warp 5      (one lane) during a GEMM phase: bulk copies of that GEMM's operand tiles, which
 //               exist only once the grid barrier of the phase that wrote them has been passed
-//   warp 4      (one lane) issues the GEMM: per ring stage four tcgen05.mma (128 weight rows x
-//               16 k) x (hi rows | lo rows of the activations), accumulating in tensor memory;
-//               tcgen05.commit hands the stage back to the producer and, at the end of a tile
-//               segment, the accumulator to the epilogue.  Two accumulator buffers, so the
-//               epilogue of one segment overlaps the MMAs of the next
-//   warps 0-3   epilogue: tensor memory -> registers (one weight row per thread), hi + lo
-//               (+ bias from the segment that holds k-chunk 0), fp32 reduction into the output
+//   warp 4      (one lane) issues the GEMM: per ring stage four tcgen05.mma, each (activation
+//               rows, hi and lo, as the M = 64 or 128 operand) x (256 weight rows as the N
+//               operand) x 16 k, accumulating in tensor memory.  A K = 16 MMA step costs about
+//               120 cycles whatever M and N are, so the weights sit on the side that lets one
+//               step consume the most of them (8 KB).  tcgen05.commit hands the stage back to
+//               the producer and, at the end of a tile segment, the accumulator to the
+//               epilogue; two accumulator buffers overlap that epilogue with the next MMAs
+//   warps 0-3   epilogue: tensor memory -> registers with the 16-lane x 256-bit load, which
+//               puts a row's hi and lo products in one thread; hi + lo goes through a small
+//               shared-memory tile so that all four warps add it (+ bias from the segment that
+//               holds k-chunk 0) to the output with 16-byte vector reductions: a reduction
+//               costs its warp a memory latency, so there must be few of them per thread
 //   warps 0-7   between GEMM phases: the small phases (row set-up, embedding, norm, activation,
 //               attention with rotary + KV append + split merge), which leave every GEMM
 //               operand in global memory already split into bf16 hi + lo, and the grid barriers
@@ -39,6 +44,8 @@ constexpr int kConsumerWarps = 8;
 constexpr int kWorkThreads = kConsumerWarps * 32;  // 256: everyone but the producer
 constexpr int kPersistThreads = kWorkThreads + 32;
 constexpr int kAttnThreadsP = 256;
+constexpr int kTileNP = 256;                        // weight rows per tile: the N of one MMA
+constexpr int kWTileBytesP = kTileNP * kTileK * 2;  // 32 KB
 
 struct alignas(64) LayerDesc {
     CUtensorMap tm[4];  // qkv, o, in, out
@@ -59,8 +66,9 @@ enum { OP_XN1 = 0, OP_XN2 = 1, OP_AO = 2, OP_ACT = 3 };
 struct alignas(64) FwdParams {
     // GEMM operands in global memory (normalised rows - two sets for parallel-residual blocks -,
     // attention output, MLP activation), stored the way a ring stage wants them: one contiguous
-    // tile per 64-wide k-chunk, 2 rk rows of 128 bytes (bf16 hi rows [0, rk), lo rows [rk, 2 rk)),
-    // 16-byte chunks already in 128-byte-swizzle order, so one linear bulk copy fetches a tile.
+    // tile per 64-wide k-chunk, 2 rk rows of 128 bytes (per block of 8 rows: their 8 bf16 hi rows, then
+    // their 8 lo rows), 16-byte chunks already in 128-byte-swizzle order, so one linear bulk copy
+    // fetches a tile.
     // (A strided 2-D tensor copy of the same tile costs a sixth of the weight stream's bandwidth.)
     __nv_bfloat16 *op[4];
     int op_ld[4];  // K of each operand
@@ -148,7 +156,7 @@ __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi) {
             g.out = p.x; g.ldo = p.d; g.bias = ld->b_out;
         }
     }
-    g.n_tiles = (g.N + kTileN - 1) / kTileN;
+    g.n_tiles = (g.N + kTileNP - 1) / kTileNP;
     g.kchunks = (g.Kd + kTileK - 1) / kTileK;
     return g;
 }
@@ -173,7 +181,10 @@ __device__ __forceinline__ void red_release_add(unsigned *p, unsigned v) {
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// Element offset of (row, column i) in a tiled operand: row in [0, 2 rk) (hi rows, then lo rows).
+// Tile row of the hi part of row r (the lo part is 8 further): rows come in blocks of 8, each block
+// as 8 hi rows followed by 8 lo rows, so that an accumulator load hands both to one thread.
+__device__ __forceinline__ int op_row(int r) { return 16 * (r >> 3) + (r & 7); }
+// Element offset of (tile row, column i) in a tiled operand: tile row in [0, 2 rk).
 __device__ __forceinline__ size_t op_off(int rk, int row, int i) {
     const int kc = i >> 6, w = i & 63;
     return (size_t)kc * (size_t)(2 * rk * kTileK) + (size_t)(row * kTileK + ((((w >> 3) ^ (row & 7)) << 3) | (w & 7)));
@@ -181,8 +192,8 @@ __device__ __forceinline__ size_t op_off(int rk, int row, int i) {
 // operand element (r, i) as hi + lo
 __device__ __forceinline__ void store_hilo(__nv_bfloat16 *buf, int rk, int r, int i, float v) {
     const __nv_bfloat16 h = __float2bfloat16_rn(v);
-    buf[op_off(rk, r, i)] = h;
-    buf[op_off(rk, rk + r, i)] = __float2bfloat16_rn(v - __bfloat162float(h));
+    buf[op_off(rk, op_row(r), i)] = h;
+    buf[op_off(rk, op_row(r) + 8, i)] = __float2bfloat16_rn(v - __bfloat162float(h));
 }
 __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -192,10 +203,12 @@ __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_
 }
 
 // ---- tcgen05 (5th-generation tensor core) helpers ---------------------------------------------
-constexpr int kTmemCols = 256;  // two accumulator buffers of 128 fp32 columns each
-constexpr int kAccStride = 128;
+constexpr int kTmemCols = 512;  // two accumulator buffers of 256 fp32 columns each
+constexpr int kAccStride = 256;
 constexpr int kEpiWarps = 4;    // warps 0-3: one tensor-memory lane quadrant each
 constexpr int kMmaWarp = 4;
+constexpr int kEpiPitch = kTileNP + 8;             // floats per row of the epilogue tile (bank spread)
+constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16;  // 8 rows, and the four warps' wait results
 constexpr int kXWarp = 5;      // issues the operand copies of a GEMM phase
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -212,9 +225,9 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
     return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) |
            (2ull << 61);
 }
-// Instruction descriptor, kind::f16: fp32 accumulate, A and B bf16, both K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t umma_idesc_bf16(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor, kind::f16: fp32 accumulate, A and B bf16, both K-major, M = m, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                             uint32_t accumulate) {
@@ -226,20 +239,26 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uin
         "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// Eight columns from each of two places of this warp's lane quadrant; the wait is part of the same
-// statement so that no use of the results can be scheduled before it.
-__device__ __forceinline__ void tc_ld_2x8(uint32_t ta, uint32_t tb, float (&a)[8], float (&b)[8]) {
+// 16 lanes x 32 columns of the accumulator (the 16-lane x 256-bit shape, four times along the columns).
+// Thread (g = lane / 4, t = lane % 4) receives, for column block k = 0..3: v[4k], v[4k+1] = lane g,
+// columns 8k + 2t, 8k + 2t + 1 and v[4k+2], v[4k+3] = lane g + 8, the same columns.  The wait is part
+// of the same statement so that no use of the results can be scheduled before it.
+__device__ __forceinline__ void tc_ld_16x32(uint32_t taddr, float (&v)[16]) {
     uint32_t r[16];
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%16];\n"
-        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%8,%9,%10,%11,%12,%13,%14,%15}, [%17];\n"
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
         "tcgen05.wait::ld.sync.aligned;\n"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(ta), "r"(tb)
+        : "r"(taddr)
         : "memory");
 #pragma unroll
-    for (int i = 0; i < 8; ++i) { a[i] = __uint_as_float(r[i]); b[i] = __uint_as_float(r[8 + i]); }
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void red_add_v4(float *dst, float4 v) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                 : "memory");
 }
 
 // Slot schedule of the ring, identical in every role that walks it (weight producer, operand issuer,
@@ -404,8 +423,8 @@ __device__ __noinline__ void norm_phase(const FwdParams &p, const float *g1, con
             const __nv_bfloat162 h01 = __floats2bfloat162_rn(y0, y1), h23 = __floats2bfloat162_rn(y2, y3);
             const __nv_bfloat162 l01 = __floats2bfloat162_rn(y0 - __low2float(h01), y1 - __high2float(h01));
             const __nv_bfloat162 l23 = __floats2bfloat162_rn(y2 - __low2float(h23), y3 - __high2float(h23));
-            __nv_bfloat16 *hi = p.op[op] + op_off(p.rk, r, 4 * i);
-            __nv_bfloat16 *lo = p.op[op] + op_off(p.rk, p.rk + r, 4 * i);
+            __nv_bfloat16 *hi = p.op[op] + op_off(p.rk, op_row(r), 4 * i);
+            __nv_bfloat16 *lo = p.op[op] + op_off(p.rk, op_row(r) + 8, 4 * i);
             uint2 hv, lv;
             hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
             lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
@@ -451,8 +470,8 @@ __device__ __noinline__ void act_phase(const FwdParams &p) {
         hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
         lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
         __nv_bfloat16 *base = p.op[OP_ACT];
-        *reinterpret_cast<uint2 *>(base + op_off(p.rk, r, 4 * c)) = hv;
-        *reinterpret_cast<uint2 *>(base + op_off(p.rk, p.rk + r, 4 * c)) = lv;
+        *reinterpret_cast<uint2 *>(base + op_off(p.rk, op_row(r), 4 * c)) = hv;
+        *reinterpret_cast<uint2 *>(base + op_off(p.rk, op_row(r) + 8, 4 * c)) = lv;
     }
 }
 
@@ -887,8 +906,11 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     constexpr int kRp = NT * 8;
-    constexpr int kXBytes = 2 * kRp * kTileK * 2;  // hi tile followed by lo tile
-    constexpr int kStageBytes = kWTileBytes + kXBytes;
+    constexpr int kXBytes = 2 * kRp * kTileK * 2;  // operand tile (hi and lo rows), then the weight tile
+    constexpr int kStageBytes = kXBytes + kWTileBytesP;
+    // M of the MMA: the operand tile's 2 kRp rows; the rows the MMA reads beyond them are the weight
+    // tile's bytes (finite or not, they only reach accumulator lanes that nobody loads)
+    constexpr int kM = 2 * kRp <= 64 ? 64 : 128;
     const int S = p.stages, S1 = p.stages_lo;
     uint8_t *ring = smem;
     uint8_t *attn_scratch = smem + p.attn_smem_off;
@@ -898,6 +920,8 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
     uint32_t *tmem_slot = (uint32_t *)(mmaDone + 1);
     Shared *sh = (Shared *)(((uintptr_t)(mmaDone + 4) + 15) & ~(uintptr_t)15);
     double *red = (double *)(sh + 1);
+    float *epi_tile = (float *)(red + 16);
+    volatile int *epi_ok = (volatile int *)(epi_tile + 8 * kEpiPitch);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp == 0) {  // tensor memory for the accumulators; released by the same warp at the end
@@ -960,8 +984,8 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                         }
                         if (failed) { rp.par ^= 1u << s; break; }  // nothing was issued into s
                     }
-                    mbar_expect_tx(&fullW[s], kWTileBytes);
-                    tma_load_2d(ring + (size_t)s * kStageBytes, dw.tmW, kw * kTileK, tw * kTileN, &fullW[s]);
+                    mbar_expect_tx(&fullW[s], kWTileBytesP);
+                    tma_load_2d(ring + (size_t)s * kStageBytes + kXBytes, dw.tmW, kw * kTileK, tw * kTileNP, &fullW[s]);
                     if (++kw == dw.kchunks) { kw = 0; ++tw; }
                 }
             }
@@ -991,7 +1015,7 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             const int tile0 = c0 / g.kchunks, tile1 = (c1 - 1) / g.kchunks;
             if (warp == kMmaWarp) {
                 if (lane == 0 && !sh->abort) {
-                    const uint32_t idesc = umma_idesc_bf16(2 * kRp);
+                    const uint32_t idesc = umma_idesc_bf16(kM, kTileNP);
                     int sg = seg, kc = c0 % g.kchunks;
                     bool first = true;
                     for (int c = c0; c < c1; ++c) {
@@ -1007,7 +1031,7 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                         }
                         tc_fence_after();
                         const uint32_t st = smem_u32(ring + (size_t)s * kStageBytes);
-                        const uint64_t adesc = umma_desc_sw128(st), bdesc = umma_desc_sw128(st + kWTileBytes);
+                        const uint64_t adesc = umma_desc_sw128(st), bdesc = umma_desc_sw128(st + kXBytes);
                         const uint32_t d_tmem = tmem_base + (uint32_t)(b * kAccStride);
 #pragma unroll
                         for (int ks = 0; ks < kTileK / 16; ++ks)  // 32 bytes further along k inside the swizzle atom
@@ -1039,38 +1063,69 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                             break;
                         }
                         mbar_expect_tx(&fullX[s], kXBytes);
-                        bulk_load_1d(ring + (size_t)s * kStageBytes + kWTileBytes,
-                                     g.xop + (size_t)kx * (2 * kRp * kTileK), kXBytes, &fullX[s]);
+                        bulk_load_1d(ring + (size_t)s * kStageBytes, g.xop + (size_t)kx * (2 * kRp * kTileK), kXBytes,
+                                     &fullX[s]);
                         if (++kx == g.kchunks) kx = 0;
                     }
                 }
                 __syncwarp();
             } else if (warp < kEpiWarps) {
                 int sg = seg;
+                const bool vec_ok = (((uintptr_t)g.out & 15) == 0) && ((g.ldo & 3) == 0) &&
+                                    (!g.bias || ((uintptr_t)g.bias & 15) == 0);
                 for (int t = tile0; t <= tile1; ++t, ++sg) {
                     const int b = sg & 1;
-                    if (!mbar_wait_or_abort(&accFull[b], (sg >> 1) & 1, sh)) {
+                    // the four warps take the same decision: the named barriers below need all of them
+                    const bool mine = mbar_wait_or_abort(&accFull[b], (sg >> 1) & 1, sh);
+                    if (lane == 0) epi_ok[warp] = mine ? 1 : 0;
+                    named_bar(5, kEpiWarps * 32);
+                    if (!(epi_ok[0] && epi_ok[1] && epi_ok[2] && epi_ok[3])) {
                         set_status(p.status, kTimeoutCode);
                         sh->abort = 1;
                         break;
                     }
                     tc_fence_after();
                     const bool has_k0 = (t > tile0) || (c0 % g.kchunks == 0);
-                    const int n = t * kTileN + warp * 32 + lane;
-                    const float bias = (has_k0 && g.bias && n < g.N) ? __ldg(g.bias + n) : 0.f;
-                    const uint32_t ta = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(b * kAccStride);
+                    const float *bias = (has_k0 && g.bias) ? g.bias : nullptr;
+                    const int g8 = lane >> 2, t4 = lane & 3;
+                    // Block q of 8 rows sits in accumulator lanes 32 q .. 32 q + 15 (M = 64) or 16 q .. 16 q + 15
+                    // (M = 128); a warp reaches the 32 lanes of its own quadrant only.
+#pragma unroll 1
+                    for (int q = 0; q < NT; ++q) {
+                        if (8 * q >= p.R) break;
+                        const int wq = kM == 64 ? q : (q >> 1), half = kM == 64 ? 0 : (q & 1);
+                        if (wq == warp) {
+                            const uint32_t ta = tmem_base + ((uint32_t)(warp * 32 + half * 16) << 16) + (uint32_t)(b * kAccStride);
+                            for (int cg = 0; cg < kTileNP / 32; ++cg) {
+                                if (t * kTileNP + cg * 32 >= g.N) break;
+                                float v[16];
+                                tc_ld_16x32(ta + (uint32_t)(cg * 32), v);
 #pragma unroll
-                    for (int j = 0; j < NT; ++j) {
-                        if (8 * j < p.R) {  // uniform over the warp
-                            float hi[8], lo[8];
-                            tc_ld_2x8(ta + 8 * j, ta + kRp + 8 * j, hi, lo);
-                            if (n < g.N) {
-#pragma unroll
-                                for (int i = 0; i < 8; ++i)
-                                    if (8 * j + i < p.R)
-                                        atomicAdd(g.out + (size_t)(8 * j + i) * g.ldo + n, hi[i] + lo[i] + bias);
+                                for (int k = 0; k < 4; ++k)
+                                    *reinterpret_cast<float2 *>(epi_tile + g8 * kEpiPitch + cg * 32 + 8 * k + 2 * t4) =
+                                        make_float2(v[4 * k] + v[4 * k + 2], v[4 * k + 1] + v[4 * k + 3]);
                             }
                         }
+                        named_bar(5, kEpiWarps * 32);
+                        const int rows_here = min(8, p.R - 8 * q);
+                        for (int i = threadIdx.x; i < rows_here * (kTileNP / 4); i += kEpiWarps * 32) {
+                            const int rr = i / (kTileNP / 4), c4 = (i % (kTileNP / 4)) * 4, n = t * kTileNP + c4;
+                            if (n >= g.N) continue;
+                            float4 v = *reinterpret_cast<const float4 *>(epi_tile + rr * kEpiPitch + c4);
+                            float *dst = g.out + (size_t)(8 * q + rr) * g.ldo + n;
+                            if (vec_ok && n + 3 < g.N) {
+                                if (bias) {
+                                    const float4 bb = __ldg(reinterpret_cast<const float4 *>(bias + n));
+                                    v.x += bb.x; v.y += bb.y; v.z += bb.z; v.w += bb.w;
+                                }
+                                red_add_v4(dst, v);
+                            } else {
+                                const float e[4] = {v.x, v.y, v.z, v.w};
+                                for (int u = 0; u < 4; ++u)
+                                    if (n + u < g.N) atomicAdd(dst + u, e[u] + (bias ? __ldg(bias + n + u) : 0.f));
+                            }
+                        }
+                        named_bar(5, kEpiWarps * 32);  // the tile is free for the next block
                     }
                     tc_fence_before();
                     __syncwarp();

@@ -425,9 +425,9 @@ inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 4 
 
 template <int NT>
 int launch_forward_nt(FwdParams p, cudaStream_t st) {
-    constexpr size_t stage = kWTileBytes + 2 * NT * 8 * kTileK * 2;
+    constexpr size_t stage = kWTileBytesP + 2 * NT * 8 * kTileK * 2;
     const size_t attn = align_up(attn_scratch_bytes(p.Dh), 128);
-    const size_t tail = 24 * 32 + 64 + 16 + sizeof(Shared) + 16 * sizeof(double) + 256;  // barriers and the small state
+    const size_t tail = 24 * 32 + 64 + 16 + sizeof(Shared) + 16 * sizeof(double) + kEpiBytes + 256;  // barriers, small state, epilogue tile
     const size_t total = (size_t)kSmemBudget - 1024 - tail;
     // upper slots share their bytes with the attention scratch; at least two slots never do
     size_t S2 = (attn + stage - 1) / stage;
@@ -661,18 +661,22 @@ int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n
         // the tensor maps and vector pointers the persistent kernel walks, copied once to the caller's block
         std::vector<uint8_t> host(ssd_model_desc_bytes(arch), 0);
         ModelDesc *md = reinterpret_cast<ModelDesc *>(host.data());
-        md->tm_lm = m->tm[(size_t)4 * arch->n_layers];
+        // (its own maps: 256-row boxes, one MMA's worth of weight rows)
+        int mrc = make_map(&md->tm_lm, lm_matrix(m), arch->vocab, arch->d_model, kTileNP);
         md->lnf_g = (const float *)fw(m, 0);
         md->lnf_b = (const float *)fw(m, 1);
         LayerDesc *ld = reinterpret_cast<LayerDesc *>(md + 1);
         for (int l = 0; l < arch->n_layers; ++l) {
-            for (int k = 0; k < 4; ++k) ld[l].tm[k] = m->tm[4 * l + k];
+            mrc |= make_map(&ld[l].tm[0], lw(m, l, L_WQKV), 3 * arch->d_model, arch->d_model, kTileNP);
+            mrc |= make_map(&ld[l].tm[1], lw(m, l, L_WO), arch->d_model, arch->d_model, kTileNP);
+            mrc |= make_map(&ld[l].tm[2], lw(m, l, L_WIN), m->d_in, arch->d_model, kTileNP);
+            mrc |= make_map(&ld[l].tm[3], lw(m, l, L_WOUT), arch->d_model, arch->d_ff, kTileNP);
             ld[l].ln1_g = (const float *)lw(m, l, L_LN1G); ld[l].ln1_b = (const float *)lw(m, l, L_LN1B);
             ld[l].b_qkv = (const float *)lw(m, l, L_BQKV); ld[l].b_o = (const float *)lw(m, l, L_BO);
             ld[l].ln2_g = (const float *)lw(m, l, L_LN2G); ld[l].ln2_b = (const float *)lw(m, l, L_LN2B);
             ld[l].b_in = (const float *)lw(m, l, L_BIN); ld[l].b_out = (const float *)lw(m, l, L_BOUT);
         }
-        if (cudaMemcpy(dev_desc, host.data(), host.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+        if (mrc || cudaMemcpy(dev_desc, host.data(), host.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
             delete m;
             return SSD_E_CUDA;
         }
