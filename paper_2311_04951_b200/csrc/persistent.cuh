@@ -834,9 +834,22 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
     }
     named_bar(3, kAttnThreadsP);
     const bool direct = p.n_split == 1;
-    for (int i = tid; i < kAttnRows * Dh; i += kAttnThreadsP) {
-        const int ml = i / Dh, e = i % Dh, m = m_base + ml;
-        if (m >= p.M) continue;
+    // four output columns of one real row per work item
+    auto store_ao4 = [&](int r, int col, float4 y) {
+        const __nv_bfloat162 h01 = __floats2bfloat162_rn(y.x, y.y), h23 = __floats2bfloat162_rn(y.z, y.w);
+        const __nv_bfloat162 l01 = __floats2bfloat162_rn(y.x - __low2float(h01), y.y - __high2float(h01));
+        const __nv_bfloat162 l23 = __floats2bfloat162_rn(y.z - __low2float(h23), y.w - __high2float(h23));
+        uint2 hv, lv;
+        hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
+        lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
+        __nv_bfloat16 *base = p.op[OP_AO];
+        *reinterpret_cast<uint2 *>(base + op_off(p.rk, op_row(r), col)) = hv;
+        *reinterpret_cast<uint2 *>(base + op_off(p.rk, op_row(r) + 8, col)) = lv;
+    };
+    const int q4 = Dh >> 2;  // float4 per row
+    const int rows_here = max(0, min(kAttnRows, p.M - m_base));
+    for (int i = tid; i < rows_here * q4; i += kAttnThreadsP) {
+        const int ml = i / q4, e = (i % q4) * 4, m = m_base + ml;
         float mx = -INFINITY;
 #pragma unroll
         for (int q = 0; q < 4; ++q) mx = fmaxf(mx, mw[q * kAttnRows + ml]);
@@ -850,16 +863,22 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
         }
         const bool live = m < n_rows && L > 0.f;
         const int gs = kAttnRows * Dh;  // stride between position groups
-        const float osum = (o_acc[i] + o_acc[i + gs]) + (o_acc[i + 2 * gs] + o_acc[i + 3 * gs]);
+        const float *oa = o_acc + ml * Dh + e;
+        const float4 a0 = *reinterpret_cast<const float4 *>(oa), a1 = *reinterpret_cast<const float4 *>(oa + gs);
+        const float4 a2 = *reinterpret_cast<const float4 *>(oa + 2 * gs), a3 = *reinterpret_cast<const float4 *>(oa + 3 * gs);
+        float4 osum = make_float4((a0.x + a1.x) + (a2.x + a3.x), (a0.y + a1.y) + (a2.y + a3.y),
+                                  (a0.z + a1.z) + (a2.z + a3.z), (a0.w + a1.w) + (a2.w + a3.w));
+        if (!live) osum = make_float4(0.f, 0.f, 0.f, 0.f);
         if (direct) {
-            store_hilo(p.op[OP_AO], p.rk, r0 + m, h * Dh + e, live ? osum / L : 0.f);
+            const float inv = live ? 1.f / L : 0.f;
+            store_ao4(r0 + m, h * Dh + e, make_float4(osum.x * inv, osum.y * inv, osum.z * inv, osum.w * inv));
         } else {
             const size_t slot = ((size_t)(r0 + m) * p.H + h) * p.n_split + split;
             if (e == 0) {
                 p.part_m[slot] = live ? mx : -INFINITY;
                 p.part_l[slot] = live ? L : 0.f;
             }
-            p.part_o[slot * Dh + e] = live ? osum : 0.f;
+            *reinterpret_cast<float4 *>(p.part_o + slot * Dh + e) = osum;
         }
     }
     if (!direct) {
@@ -870,22 +889,41 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
         named_bar(3, kAttnThreadsP);
         if (sh->flag) {
             __threadfence();
-            for (int idx = tid; idx < p.M * Dh; idx += kAttnThreadsP) {
-                const int m = idx / Dh, e = idx % Dh;
+            // one work item = four columns of one row; the loads of up to eight splits are issued together
+            for (int idx = tid; idx < p.M * q4; idx += kAttnThreadsP) {
+                const int m = idx / q4, e = (idx % q4) * 4;
                 const size_t base = ((size_t)(r0 + m) * p.H + h) * p.n_split;
-                float mx = -INFINITY;
-                for (int s2 = 0; s2 < p.n_split; ++s2) mx = fmaxf(mx, __ldcg(p.part_m + base + s2));
-                float L = 0.f, acc = 0.f;
-                if (mx > -INFINITY) {
-                    for (int s2 = 0; s2 < p.n_split; ++s2) {
-                        const float pm = __ldcg(p.part_m + base + s2);
-                        if (pm == -INFINITY) continue;
-                        const float w = exp2f(pm - mx);
-                        L = fmaf(__ldcg(p.part_l + base + s2), w, L);
-                        acc = fmaf(__ldcg(p.part_o + (base + s2) * Dh + e), w, acc);
+                float mx = -INFINITY, L = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int s0 = 0; s0 < p.n_split; s0 += 8) {
+                    float pm[8], pl[8];
+                    float4 po[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const bool in = s0 + u < p.n_split;
+                        pm[u] = in ? __ldcg(p.part_m + base + s0 + u) : -INFINITY;
+                        pl[u] = in ? __ldcg(p.part_l + base + s0 + u) : 0.f;
+                        po[u] = in ? __ldcg(reinterpret_cast<const float4 *>(p.part_o + (base + s0 + u) * Dh + e))
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
                     }
+                    float bm = mx;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) bm = fmaxf(bm, pm[u]);
+                    if (bm == -INFINITY) continue;
+                    const float f = exp2f(mx - bm);  // 0 while nothing has been accumulated
+                    L *= f; acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (pm[u] == -INFINITY) continue;
+                        const float w = exp2f(pm[u] - bm);
+                        L = fmaf(pl[u], w, L);
+                        acc.x = fmaf(po[u].x, w, acc.x); acc.y = fmaf(po[u].y, w, acc.y);
+                        acc.z = fmaf(po[u].z, w, acc.z); acc.w = fmaf(po[u].w, w, acc.w);
+                    }
+                    mx = bm;
                 }
-                store_hilo(p.op[OP_AO], p.rk, r0 + m, h * Dh + e, L > 0.f ? acc / L : 0.f);
+                const float inv = L > 0.f ? 1.f / L : 0.f;
+                store_ao4(r0 + m, h * Dh + e, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
             }
             if (tid == 0) p.tickets[bh] = 0;  // ready for the next layer (a grid barrier lies between)
         }
