@@ -574,15 +574,19 @@ __device__ __forceinline__ void rope_vec8(const FwdParams &p, const float *row, 
 constexpr int kAttnRows = 16;  // query rows per item (one MMA row tile)
 constexpr int kAttnBufs = 3;   // K/V chunk buffers: two chunks (64 KB at head 128) in flight per SM
 __host__ __device__ inline size_t attn_scratch_bytes(int Dh) {
-    // Q hi/lo [16][Dh+8] bf16, kAttnBufs K/V chunk buffers [2][64][Dh+8] bf16 each, per-warp (m, l) [8][16] fp32 x 2
-    return (size_t)2 * kAttnRows * (Dh + 8) * 2 + (size_t)kAttnBufs * 2 * kAttnTile * (Dh + 8) * 2 + 2 * 8 * kAttnRows * 4;
+    // Q hi/lo [16][Dh+8] bf16, kAttnBufs K/V chunk buffers [2][64][Dh+8] bf16 each, per-warp (m, l) [8][16] fp32 x 2,
+    // per-thread partial scores [256][8] fp32
+    return (size_t)2 * kAttnRows * (Dh + 8) * 2 + (size_t)kAttnBufs * 2 * kAttnTile * (Dh + 8) * 2 + 2 * 8 * kAttnRows * 4 +
+           (size_t)256 * 8 * 4;
 }
 
 // Attention of up to 16 query rows of one (sequence, head) over one split of the position axis, by
 // 256 threads, on tensor cores.  K/V chunks of 64 positions are fetched with cp.async into three
 // buffers (the next two chunks load while this one is used).  Warp w owns positions 16 (w & 3) .. +15
-// of each chunk and the output columns of half (w >> 2) of the head: it computes its 16 x 16 score
-// block S = Q K^T (Q as bf16 hi + lo), keeps its own running max / sum, and adds P V (P as bf16
+// of each chunk and the output columns of half (w >> 2) of the head.  The two warps of a position
+// group each contract half of the head dimension of the 16 x 16 score block S = Q K^T (Q as bf16
+// hi + lo) and exchange the halves, so both hold S; each keeps its own running max / sum (equal in
+// both, the sum of two halves being order-independent) and adds P V (P as bf16
 // hi + lo) to its 16 x Dh/2 accumulators -- no exchange between warps until the end, where the
 // four position groups are merged in shared memory.  Rows of this pass (positions >= len) take
 // their keys / values from qkv (rotary, cache rounding) and the split that owns them appends them
@@ -599,6 +603,7 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
     __nv_bfloat16 *KV = Qlo + kAttnRows * pitch;  // buffer i: K at KV + i * 2 * 64 * pitch, V 64 * pitch later
     float *mw = reinterpret_cast<float *>(KV + kAttnBufs * 2 * kAttnTile * pitch);
     float *lw = mw + 8 * kAttnRows;
+    float *sx = lw + 8 * kAttnRows;  // score halves exchanged between the two warps of a position group
     float *o_acc = reinterpret_cast<float *>(KV);  // [4][16][Dh] fp32, reuses the chunk buffers after the loop
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -719,9 +724,10 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
             const uint32_t qa = smem_u32(Qhi) + (uint32_t)(lane & 15) * pitchB + (uint32_t)(lane >> 4) * 16u;
             const uint32_t ql = qa + (uint32_t)kAttnRows * pitchB;
             const uint32_t ka = smem_u32(Kb) + (uint32_t)(16 * pg + (lane & 7) + 8 * (lane >> 4)) * pitchB + (uint32_t)((lane >> 3) & 1) * 16u;
+            const int ks_lo = dhh ? (nk + 1) / 2 : 0, ks_hi = dhh ? nk : (nk + 1) / 2;  // this warp's half of Dh
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
-                if (ks < nk) {
+                if (ks >= ks_lo && ks < ks_hi) {
                     uint32_t a0, a1, a2, a3, c0, c1, c2, c3, k0, k1, k2, k3;
                     ldmatrix_x4(qa + ks * 32, a0, a1, a2, a3);
                     ldmatrix_x4(ql + ks * 32, c0, c1, c2, c3);
@@ -736,6 +742,15 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
             for (int j = 0; j < 2; ++j)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) s[j][e] = (sa[0][0][j][e] + sa[0][1][j][e]) + (sa[1][0][j][e] + sa[1][1][j][e]);
+            // exchange with the warp that holds the other half (same position group, same lane = same elements)
+            float4 *mine = reinterpret_cast<float4 *>(sx + (size_t)tid * 8);
+            mine[0] = make_float4(s[0][0], s[0][1], s[0][2], s[0][3]);
+            mine[1] = make_float4(s[1][0], s[1][1], s[1][2], s[1][3]);
+            named_bar(8 + pg, 64);
+            const float4 *other = reinterpret_cast<const float4 *>(sx + (size_t)(tid ^ 128) * 8);
+            const float4 o0 = other[0], o1 = other[1];
+            s[0][0] += o0.x; s[0][1] += o0.y; s[0][2] += o0.z; s[0][3] += o0.w;
+            s[1][0] += o1.x; s[1][1] += o1.y; s[1][2] += o1.z; s[1][3] += o1.w;
         }
         // ---- mask, running max / sum (rows g and g + 8) ----
         float pr[2][4];
