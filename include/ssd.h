@@ -96,6 +96,15 @@ size_t ssd_model_desc_bytes(const ssd_arch *arch);
  * step instead (same results up to fp32 summation order; kept for comparison). */
 int ssd_set_persistent(int enable);
 
+/* The single forward kernel has two forms of the K-query attention over the cache (Section "KV Caching":
+ * the new rows attend to the stored keys / values): items on warp-level MMAs, 64 positions per step,
+ * and - head dimension 128 only - items on the tcgen05 tensor core with the scores in tensor memory,
+ * 128 positions per step, which start more slowly but stream twice as fast.  mode 0 (default) picks
+ * per pass (tensor-core items from 1024 positions per split), 1 forces the first form, 2 the second
+ * wherever it applies.  Same results up to fp32 summation order; for comparison and tests.
+ * SSD_E_ARG for any other mode. */
+int ssd_set_attention_mode(int mode);
+
 /* A layer-skip draft: the first n_layers layers of `target` plus its final norm and LM head
  * (an early-exit style draft, cf. Section "Speculative Sampling").  Shares the target's tensors. */
 int ssd_model_share_prefix(const ssd_model *target, int n_layers, ssd_model **draft_out);
@@ -111,7 +120,10 @@ size_t ssd_workspace_bytes(const ssd_model *m, int batch, int rows_per_seq, int 
 
 /*
  * Wrap a caller-owned slab (256-byte aligned, >= ssd_kv_bytes) as the KV cache of `batch`
- * sequences; queues the zeroing of the header (all lengths 0, status clear) on `stream`.
+ * sequences; queues the zeroing of the whole slab on `stream`: header (all lengths 0, status
+ * clear) and cache.  Attention reads whole position tiles and masks what lies beyond a sequence's
+ * length, so those bytes must always be finite numbers: zeros at first, later only rows that earlier
+ * passes wrote.
  * (Section "KV Caching": keys/values of past tokens are stored so later passes reuse them; one
  * cache per model, Section "So, what's the problem?".)
  */

@@ -34,7 +34,7 @@ class SsdArch(ctypes.Structure):
         ("rotary_base", ctypes.c_float), ("norm_eps", ctypes.c_float)]
 
 
-EXPORTS = ["ssd_model_create", "ssd_model_desc_bytes", "ssd_set_persistent", "ssd_model_share_prefix", "ssd_model_destroy", "ssd_kv_bytes",
+EXPORTS = ["ssd_model_create", "ssd_model_desc_bytes", "ssd_set_persistent", "ssd_set_attention_mode", "ssd_model_share_prefix", "ssd_model_destroy", "ssd_kv_bytes",
            "ssd_workspace_bytes", "kv_init", "kv_destroy", "kv_prefill", "draft_step", "target_verify",
            "kv_commit", "kv_rollback", "spec_advance", "kv_lengths", "ssd_device_status",
            "verify_from_logits", "verify_from_logits_noalloc", "verify_scratch_bytes", "attention_rows", "ssd_last_logits", "ssd_set_trace", "ssd_read_trace", "ssd_launch_count",
@@ -61,6 +61,7 @@ def load():
     L.ssd_model_desc_bytes.argtypes = [ctypes.POINTER(SsdArch)]
     L.ssd_model_desc_bytes.restype = sz
     L.ssd_set_persistent.argtypes = [i32]
+    L.ssd_set_attention_mode.argtypes = [i32]
     L.ssd_model_share_prefix.argtypes = [vp, i32, pp]
     L.ssd_model_destroy.argtypes = [vp]
     L.ssd_model_destroy.restype = None
@@ -302,6 +303,11 @@ def last_logits(model: Model, batch: int, rows_per_seq: int, ws: torch.Tensor) -
 
 def set_persistent(enable: bool) -> None:
     _check(load().ssd_set_persistent(1 if enable else 0), "ssd_set_persistent")
+
+
+def set_attention_mode(mode: int) -> None:
+    """0: per pass (default); 1: warp-MMA attention items; 2: tensor-core items wherever they apply."""
+    _check(load().ssd_set_attention_mode(int(mode)), "ssd_set_attention_mode")
 
 
 def set_trace(enable: bool) -> None:

@@ -103,6 +103,10 @@ struct alignas(64) FwdParams {
     // only between attention phases.  bar_off: byte offset of the barriers behind both.
     int stages, stages_lo, attn_smem_off, bar_off;
     unsigned long long *trace;  // optional: CTA 0 stamps the global timer after every grid barrier
+    // tensor-core attention (head dim 128): the whole cache as rows of Dh bf16, box 64 x 128 rows
+    CUtensorMap tm_kv;
+    int attn_tc;             // 1: attention_item_tc; 0: attention_item
+    int kv_rows_per_layer;   // B * 2 * H * S
 };
 
 struct GemmDesc {
@@ -208,7 +212,7 @@ constexpr int kAccStride = 256;
 constexpr int kEpiWarps = 4;    // warps 0-3: one tensor-memory lane quadrant each
 constexpr int kMmaWarp = 4;
 constexpr int kEpiPitch = kTileNP + 8;             // floats per row of the epilogue tile (bank spread)
-constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16;  // 8 rows, and the four warps' wait results
+constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 11 * 8 + 11 * 4 + 12;  // 8 rows, the four warps' wait results, attention barriers
 constexpr int kXWarp = 5;      // issues the operand copies of a GEMM phase
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -285,6 +289,10 @@ struct alignas(16) Shared {
     volatile int abort;     // some wait in this CTA gave up
     volatile int go;        // snapshot of !abort taken inside the grid barrier: uniform for all work threads
     int flag;
+    // for the tensor-core attention items (kept here so that they take no more arguments than the others):
+    uint32_t tmem_base;     // base address of this CTA's tensor memory
+    uint32_t attn_bar_off;  // byte offset from this block to the attention barriers, followed by their counts
+    uint32_t pad[2];
 };
 
 // Bounded wait that also gives up as soon as another thread of the CTA has.
@@ -292,6 +300,16 @@ __device__ __forceinline__ bool mbar_wait_or_abort(uint64_t *bar, uint32_t parit
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
+        if (sh->abort || clock64() - t0 > kWaitCycles) return false;
+    }
+    return true;
+}
+
+// The same as a pure poll (a suspended waiter wakes up late; used where a hand-off is on the critical path).
+__device__ __forceinline__ bool mbar_spin_or_abort(uint64_t *bar, uint32_t parity, const Shared *sh) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_test_wait(bar, parity)) {
         if (sh->abort || clock64() - t0 > kWaitCycles) return false;
     }
     return true;
@@ -569,6 +587,62 @@ __device__ __forceinline__ void rope_vec8(const FwdParams &p, const float *row, 
 #pragma unroll
         for (int u = 0; u < 8; ++u) out[u] = low ? out[u] * cc[u] - pb[u] * ss[u] : pb[u] * ss[u] + out[u] * cc[u];
     }
+}
+
+// four output columns of one row of the out-projection operand, as bf16 hi + lo
+__device__ __forceinline__ void store_ao4(const FwdParams &p, int r, int col, float4 y) {
+    const __nv_bfloat162 h01 = __floats2bfloat162_rn(y.x, y.y), h23 = __floats2bfloat162_rn(y.z, y.w);
+    const __nv_bfloat162 l01 = __floats2bfloat162_rn(y.x - __low2float(h01), y.y - __high2float(h01));
+    const __nv_bfloat162 l23 = __floats2bfloat162_rn(y.z - __low2float(h23), y.w - __high2float(h23));
+    uint2 hv, lv;
+    hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
+    lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
+    __nv_bfloat16 *base = p.op[OP_AO];
+    *reinterpret_cast<uint2 *>(base + op_off(p.rk, op_row(r), col)) = hv;
+    *reinterpret_cast<uint2 *>(base + op_off(p.rk, op_row(r) + 8, col)) = lv;
+}
+
+// The item that finishes last for a (sequence, head) merges the splits' partials (m, l, o) of all its
+// rows into the out-projection operand; 256 threads.
+__device__ __forceinline__ void merge_splits(const FwdParams &p, int r0, int h, int Dh) {
+    const int tid = threadIdx.x, q4 = Dh >> 2;
+    auto store_ao4 = [&](int r, int col, float4 y) { ssd::store_ao4(p, r, col, y); };
+            // one work item = four columns of one row; the loads of up to eight splits are issued together
+            for (int idx = tid; idx < p.M * q4; idx += kAttnThreadsP) {
+                const int m = idx / q4, e = (idx % q4) * 4;
+                const size_t base = ((size_t)(r0 + m) * p.H + h) * p.n_split;
+                float mx = -INFINITY, L = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int s0 = 0; s0 < p.n_split; s0 += 8) {
+                    float pm[8], pl[8];
+                    float4 po[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const bool in = s0 + u < p.n_split;
+                        pm[u] = in ? __ldcg(p.part_m + base + s0 + u) : -INFINITY;
+                        pl[u] = in ? __ldcg(p.part_l + base + s0 + u) : 0.f;
+                        po[u] = in ? __ldcg(reinterpret_cast<const float4 *>(p.part_o + (base + s0 + u) * Dh + e))
+                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    float bm = mx;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) bm = fmaxf(bm, pm[u]);
+                    if (bm == -INFINITY) continue;
+                    const float f = exp2f(mx - bm);  // 0 while nothing has been accumulated
+                    L *= f; acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (pm[u] == -INFINITY) continue;
+                        const float w = exp2f(pm[u] - bm);
+                        L = fmaf(pl[u], w, L);
+                        acc.x = fmaf(po[u].x, w, acc.x); acc.y = fmaf(po[u].y, w, acc.y);
+                        acc.z = fmaf(po[u].z, w, acc.z); acc.w = fmaf(po[u].w, w, acc.w);
+                    }
+                    mx = bm;
+                }
+                const float inv = L > 0.f ? 1.f / L : 0.f;
+                store_ao4(r0 + m, h * Dh + e, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
+            }
 }
 
 constexpr int kAttnRows = 16;  // query rows per item (one MMA row tile)
@@ -904,52 +978,426 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
         named_bar(3, kAttnThreadsP);
         if (sh->flag) {
             __threadfence();
-            // one work item = four columns of one row; the loads of up to eight splits are issued together
-            for (int idx = tid; idx < p.M * q4; idx += kAttnThreadsP) {
-                const int m = idx / q4, e = (idx % q4) * 4;
-                const size_t base = ((size_t)(r0 + m) * p.H + h) * p.n_split;
-                float mx = -INFINITY, L = 0.f;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int s0 = 0; s0 < p.n_split; s0 += 8) {
-                    float pm[8], pl[8];
-                    float4 po[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const bool in = s0 + u < p.n_split;
-                        pm[u] = in ? __ldcg(p.part_m + base + s0 + u) : -INFINITY;
-                        pl[u] = in ? __ldcg(p.part_l + base + s0 + u) : 0.f;
-                        po[u] = in ? __ldcg(reinterpret_cast<const float4 *>(p.part_o + (base + s0 + u) * Dh + e))
-                                   : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                    float bm = mx;
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) bm = fmaxf(bm, pm[u]);
-                    if (bm == -INFINITY) continue;
-                    const float f = exp2f(mx - bm);  // 0 while nothing has been accumulated
-                    L *= f; acc.x *= f; acc.y *= f; acc.z *= f; acc.w *= f;
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        if (pm[u] == -INFINITY) continue;
-                        const float w = exp2f(pm[u] - bm);
-                        L = fmaf(pl[u], w, L);
-                        acc.x = fmaf(po[u].x, w, acc.x); acc.y = fmaf(po[u].y, w, acc.y);
-                        acc.z = fmaf(po[u].z, w, acc.z); acc.w = fmaf(po[u].w, w, acc.w);
-                    }
-                    mx = bm;
-                }
-                const float inv = L > 0.f ? 1.f / L : 0.f;
-                store_ao4(r0 + m, h * Dh + e, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
-            }
+            merge_splits(p, r0, h, Dh);
             if (tid == 0) p.tickets[bh] = 0;  // ready for the next layer (a grid barrier lies between)
         }
     }
     named_bar(3, kAttnThreadsP);  // scratch is free for the next item
 }
 
+// ---- attention on tcgen05 (head dim 128) ----------------------------------------------------------
+// The same item as attention_item - up to 16 query rows of one (sequence, head) over one split of the
+// position axis - with the two products on the 5th-generation tensor core and the scores and the
+// output in tensor memory, 128 positions per chunk:
+//   S^T [128 positions x 32]  = K chunk (the M = 128 operand, straight from the TMA copy of the cache)
+//                               x Q rows (16 hi + 16 lo, the N = 32 operand)
+//   O^T [128 head dims x 32] += V chunk read as its transpose (MN-major M = 128 operand) x P (16 hi + 16 lo)
+// Roles: threads 0-127 = one position each (softmax: masks, running max shared through shared memory,
+// P as bf16 hi + lo into the P tile, rescale of O^T when a maximum moved) and, at the end, one head
+// dim each (output); warp 4: MMA issue; warp 5: TMA copies of K and V chunks into a 3-stage ring;
+// warps 6-7: rows of this pass (positions >= len) - rotary, rounding, append to the cache - written
+// into the chunk tiles over what the copy brought.  Positions behind them are masked (P = 0) and
+// multiply whatever the cache holds there: kv_init zeroes the cache, and all later writes are
+// finite rows of earlier passes, so 0 x stale is 0.  Per chunk 8 + 8 MMA steps of ~120 cycles against 1.5 us of HBM time for its
+// 64 KB: the chunk loop is bandwidth-bound instead of a latency chain.
+constexpr int kTcChunk = 128;
+constexpr int kTcKvStage = kTcChunk * 128 * 2;  // one K or V chunk: two 64-column panels of 128 rows x 128 B
+constexpr int kTcQOff = 3 * kTcKvStage, kTcPOff = kTcQOff + 8192, kTcMiscOff = kTcPOff + 8192;
+constexpr int kTcScratchBytes = kTcMiscOff + 1536 + kAttnRows * 128 * 4;  // + per-thread running sums [16][128]
+// Its mbarriers live outside the scratch (which the weight ring reuses), are initialised once per kernel
+// and keep running: cnt[i] = phases barrier i has completed before the current item.
+enum { AB_KV_FULL = 0, AB_KV_FREE = 3, AB_S_FULL = 6, AB_P_READY = 8, AB_O_DONE = 9, AB_FIXED = 10, AB_COUNT = 11 };
+
+__device__ __forceinline__ void tc_ld_32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,"
+        "%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// one column from each of two places of this warp's lane quadrant
+__device__ __forceinline__ void tc_ld_2(uint32_t ta, uint32_t tb, float &a, float &b) {
+    uint32_t x, y;
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%2];\n"
+        "tcgen05.ld.sync.aligned.32x32b.x1.b32 {%1}, [%3];\n"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=r"(x), "=r"(y)
+        : "r"(ta), "r"(tb)
+        : "memory");
+    a = __uint_as_float(x);
+    b = __uint_as_float(y);
+}
+__device__ __forceinline__ void tc_st_32(uint32_t taddr, const float (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,"
+        "%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+        "tcgen05.wait::st.sync.aligned;\n" ::"r"(taddr),
+        "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+        "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+        "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+        "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+        "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+        "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+        : "memory");
+}
+// shared-memory matrix descriptor, 128-byte swizzle, explicit leading / stride byte offsets
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+// byte offset of (row, 16-byte chunk c) in a tile of 128-byte rows with the 128-byte swizzle
+__device__ __forceinline__ uint32_t sw128(int row, int c) { return (uint32_t)(row * 128 + ((c ^ (row & 7)) << 4)); }
+
+__device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, int item, uint8_t *scratch, Shared *sh) {
+    const uint32_t tmem_base = sh->tmem_base;
+    uint64_t *abar = reinterpret_cast<uint64_t *>(reinterpret_cast<uint8_t *>(sh) + sh->attn_bar_off);
+    uint32_t *acnt = reinterpret_cast<uint32_t *>(abar + AB_COUNT);
+    constexpr int Dh = 128;
+    const int MT = (p.M + kAttnRows - 1) / kAttnRows;
+    const int mt = item % MT, rest = item / MT;
+    const int split = rest % p.n_split, bh = rest / p.n_split, b = bh / p.H, h = bh % p.H;
+    const int d = p.d;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint8_t *ring = scratch, *qt = scratch + kTcQOff, *pt = scratch + kTcPOff;
+    // [2][4][16] chunk maxima per warp: scores are one chunk ahead, so a fast warp may already write the next
+    // chunk's maxima while a slow one still reads this chunk's
+    float *wmax2 = reinterpret_cast<float *>(scratch + kTcMiscOff);
+    float *wsum = wmax2 + 128;                                      // [4][16]
+    float *wmrun = wsum + 64;                                       // [4][16] running maxima, one copy per warp
+    float *fsh = wmrun + 64;                                        // [4][16] this chunk's rescale factors
+    float *l_sh = fsh + 64;                                         // [16][128] running sums, one per (row, thread)
+    uint64_t *kv_full = abar + AB_KV_FULL, *kv_free = abar + AB_KV_FREE;  // [3] each
+    uint64_t *s_full = abar + AB_S_FULL;  // [2]: the scores are double-buffered in tensor memory
+    uint64_t *p_ready = abar + AB_P_READY, *o_done = abar + AB_O_DONE, *fixed = abar + AB_FIXED;
+
+    const int n_rows = __ldcg(p.ri.n_eff + b);
+    const int len = p.len[b];
+    const int r0 = b * p.M, m_base = mt * kAttnRows;
+    const int rows_here = max(0, min(kAttnRows, p.M - m_base));
+    const int p_begin = split * p.chunk;
+    const int p_end = min(p_begin + p.chunk, len + n_rows);
+    const int n_chunks = p_begin < p_end ? (p_end - p_begin + kTcChunk - 1) / kTcChunk : 0;
+    const float sc = p.attn_scale * 1.4426950408889634f;  // scores in log2 units
+    const uint32_t tS = tmem_base, tO = tmem_base + 64;  // scores of chunk c at tS + 32 (c & 1)
+    __nv_bfloat16 *kc = (__nv_bfloat16 *)(p.cache + (size_t)layer * p.layer_bytes) + ((size_t)(b * 2) * p.H + h) * p.S * Dh;
+    __nv_bfloat16 *vc = kc + (size_t)p.H * p.S * Dh;
+    const int krow0 = layer * p.kv_rows_per_layer + ((b * 2) * p.H + h) * p.S, vrow0 = krow0 + p.H * p.S;
+
+    // a wait that keeps the control flow of every role intact: once anything has timed out, waits fall through
+    auto wait = [&](uint64_t *bar, uint32_t parity) {
+        if (sh->abort) return;
+        if (!mbar_spin_or_abort(bar, parity, sh)) {
+            set_status(p.status, kTimeoutCode);
+            sh->abort = 1;
+        }
+    };
+
+    // phases completed before this item (written by thread 0 at the end of the previous item, behind a barrier)
+    uint32_t c_full[3], c_free[3];
+#pragma unroll
+    for (int i = 0; i < 3; ++i) { c_full[i] = acnt[AB_KV_FULL + i]; c_free[i] = acnt[AB_KV_FREE + i]; }
+    const uint32_t c_s0 = acnt[AB_S_FULL], c_s1 = acnt[AB_S_FULL + 1];
+    const uint32_t c_p = acnt[AB_P_READY], c_o = acnt[AB_O_DONE], c_fix = acnt[AB_FIXED];
+    auto full_par = [&](int j) { return (c_full[j % 3] + (uint32_t)(j / 3)) & 1u; };          // stage j has landed
+    auto free_par = [&](int j) { return ((c_free[j % 3] + (uint32_t)(j / 3)) & 1u) ^ 1u; };   // its slot was released
+    int n_fix_total = 0;
+    for (int c = 0; c < n_chunks; ++c) n_fix_total += (p_begin + (c + 1) * kTcChunk > len) ? 1 : 0;
+
+    // The copies of the first chunks do not depend on the set-up below: start them now.
+    auto issue_kv = [&](int j) {
+        const int slot = j % 3, c = j >> 1;
+        const int row = ((j & 1) ? vrow0 : krow0) + p_begin + c * kTcChunk;
+        uint8_t *dst = ring + slot * kTcKvStage;
+        mbar_expect_tx(&kv_full[slot], kTcKvStage);
+        tma_load_2d(dst, &p.tm_kv, 0, row, &kv_full[slot]);
+        tma_load_2d(dst + kTcKvStage / 2, &p.tm_kv, 64, row, &kv_full[slot]);
+    };
+    const int n_early = min(3, 2 * n_chunks);
+    if (warp == 5 && lane == 0 && !sh->abort) {
+        fence_async_proxy();  // the previous user of these slots wrote them through the generic proxy
+        for (int j = 0; j < n_early; ++j) issue_kv(j);
+    }
+    // ---- set-up: Q tile (rotary applied; 16 hi rows, 16 lo rows), P tile zeroed ----
+    {
+        const int ml = tid >> 4, v8 = tid & 15, m = m_base + ml;
+        float q[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) q[u] = 0.f;
+        if (m < n_rows && ml < rows_here) rope_vec8(p, p.qkv + (size_t)(r0 + m) * 3 * d + h * Dh, r0 + m, v8 * 8, q);
+        __nv_bfloat16 hq[8], lq[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            hq[u] = __float2bfloat16_rn(q[u]);
+            lq[u] = __float2bfloat16_rn(q[u] - __bfloat162float(hq[u]));
+        }
+        uint8_t *panel = qt + (v8 >> 3) * 4096;
+        *reinterpret_cast<uint4 *>(panel + sw128(ml, v8 & 7)) = *reinterpret_cast<uint4 *>(hq);
+        *reinterpret_cast<uint4 *>(panel + sw128(16 + ml, v8 & 7)) = *reinterpret_cast<uint4 *>(lq);
+        reinterpret_cast<uint4 *>(pt)[2 * tid] = make_uint4(0, 0, 0, 0);
+        reinterpret_cast<uint4 *>(pt)[2 * tid + 1] = make_uint4(0, 0, 0, 0);
+    }
+    fence_async_proxy();
+    named_bar(3, kAttnThreadsP);
+
+    if (warp == 5) {
+        // ---------------- K / V chunk copies: stage j = 2 c (K), 2 c + 1 (V), slot j % 3 ----------------
+        if (lane == 0) {
+            int issued = n_early;
+            for (int j = n_early; j < 2 * n_chunks && !sh->abort; ++j) {
+                wait(&kv_free[j % 3], free_par(j));
+                if (sh->abort) break;
+                issue_kv(j);
+                ++issued;
+            }
+            if (sh->abort)  // error path only: copies still in flight
+                for (int j = max(0, issued - 3); j < issued; ++j) mbar_wait(&kv_full[j % 3], full_par(j));
+        }
+        __syncwarp();
+    } else if (warp == 4) {
+        // ---------------- MMA issue ----------------
+        if (lane == 0) {
+            const uint32_t idS = umma_idesc_bf16(128, 32), idO = umma_idesc_bf16(128, 32) | (1u << 15);  // A of PV: MN-major
+            const uint32_t qa = smem_u32(qt), pa = smem_u32(pt);
+            int n_fix = 0;
+            // S(c): scores of chunk c into buffer c & 1; issued one chunk ahead of P V so that it runs
+            // while the softmax threads work on the previous chunk
+            auto issue_s = [&](int c) {
+                const int jk = 2 * c, jv = 2 * c + 1;
+                const bool fix = p_begin + (c + 1) * kTcChunk > len;
+                wait(&kv_full[jk % 3], full_par(jk));
+                if (fix) { wait(&kv_full[jv % 3], full_par(jv)); wait(fixed, (c_fix + n_fix) & 1u); ++n_fix; }
+                if (sh->abort) return;
+                tc_fence_after();
+                const uint32_t ka = smem_u32(ring + (jk % 3) * kTcKvStage);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)  // k = 16 head dims per step; panel ks / 4
+                    tc_mma_bf16(tS + 32 * (c & 1), umma_desc(ka + (ks >> 2) * (kTcKvStage / 2) + (ks & 3) * 32, 16, 1024),
+                                umma_desc(qa + (ks >> 2) * 4096 + (ks & 3) * 32, 16, 1024), idS, ks ? 1u : 0u);
+                tc_commit(&s_full[c & 1]);
+                tc_commit(&kv_free[jk % 3]);
+            };
+            if (n_chunks > 0) issue_s(0);
+            for (int c = 0; c < n_chunks && !sh->abort; ++c) {
+                const int jv = 2 * c + 1;
+                if (c + 1 < n_chunks) issue_s(c + 1);
+                wait(p_ready, (c_p + c) & 1u);
+                wait(&kv_full[jv % 3], full_par(jv));
+                if (sh->abort) break;
+                tc_fence_after();
+                const uint32_t va = smem_u32(ring + (jv % 3) * kTcKvStage);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)  // k = 16 positions per step: two 8-row groups of the V tile
+                    tc_mma_bf16(tO, umma_desc(va + ks * 2048, kTcKvStage / 2, 1024),
+                                umma_desc(pa + (ks >> 2) * 4096 + (ks & 3) * 32, 16, 1024), idO, (c | ks) ? 1u : 0u);
+                tc_commit(o_done);
+                tc_commit(&kv_free[jv % 3]);
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 6) {
+        // ---------------- rows of this pass, chunk by chunk ----------------
+        const int ft = tid - 192;  // 0..63
+        for (int c = 0; c < n_chunks; ++c) {
+            const int base = p_begin + c * kTcChunk;
+            if (base + kTcChunk <= len) continue;
+            const int jk = 2 * c, jv = 2 * c + 1;
+            uint8_t *kt = ring + (jk % 3) * kTcKvStage, *vt = ring + (jv % 3) * kTcKvStage;
+            const int first = max(0, len - base), last = min(kTcChunk, len + n_rows - base);  // tile rows [first, last)
+            // at most 32 rows x 16 vectors = 8 work items per thread: compute them all, then wait for the copies
+            uint4 kq[8], vq[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = ft + 64 * u, pr = first + (i >> 4), v8 = i & 15;
+                kq[u] = vq[u] = make_uint4(0, 0, 0, 0);
+                if (pr < last) {
+                    const int pos = base + pr, r = r0 + (pos - len);
+                    const float *krow = p.qkv + (size_t)r * 3 * d + d + h * Dh;
+                    float kf[8];
+                    rope_vec8(p, krow, r, v8 * 8, kf);
+                    const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(krow + d + v8 * 8));
+                    const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(krow + d + v8 * 8 + 4));
+                    const float vf[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+                    __nv_bfloat16 kb[8], vb[8];
+#pragma unroll
+                    for (int w = 0; w < 8; ++w) {
+                        kb[w] = __float2bfloat16_rn(kf[w]);
+                        vb[w] = __float2bfloat16_rn(vf[w]);
+                    }
+                    kq[u] = *reinterpret_cast<uint4 *>(kb);
+                    vq[u] = *reinterpret_cast<uint4 *>(vb);
+                }
+            }
+            wait(&kv_full[jk % 3], full_par(jk));
+            wait(&kv_full[jv % 3], full_par(jv));
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = ft + 64 * u, pr = first + (i >> 4), v8 = i & 15;
+                if (pr < last) {
+                    const uint32_t off = (uint32_t)(v8 >> 3) * (kTcKvStage / 2) + sw128(pr, v8 & 7);
+                    *reinterpret_cast<uint4 *>(kt + off) = kq[u];
+                    *reinterpret_cast<uint4 *>(vt + off) = vq[u];
+                    if (mt == 0) {  // append: exactly one split owns this position (stores after all the loads)
+                        const size_t go = (size_t)(base + pr) * Dh + v8 * 8;
+                        *reinterpret_cast<uint4 *>(kc + go) = kq[u];
+                        *reinterpret_cast<uint4 *>(vc + go) = vq[u];
+                    }
+                }
+            }
+            fence_async_proxy();
+            mbar_arrive(fixed);
+        }
+    } else {
+        // ---------------- softmax: thread = position tid of the chunk ----------------
+        // Runtime loops over the real rows (usually 5 of 16) and per-row tensor-memory loads keep this
+        // code small: it runs once per item and layer, so its instruction fetch is mostly cold.
+        const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+        float *lrow = l_sh + tid;
+        for (int r = 0; r < rows_here; ++r) lrow[r * 128] = 0.f;
+        if (lane < kAttnRows) { wmrun[warp * 16 + lane] = -INFINITY; fsh[warp * 16 + lane] = 1.f; }
+        __syncwarp();
+        for (int c = 0; c < n_chunks; ++c) {
+            const int pos = p_begin + c * kTcChunk + tid;
+            const uint32_t tSc = tS + 32 * (c & 1) + lane_sel;
+            float *wmax = wmax2 + 64 * (c & 1);
+            wait(&s_full[c & 1], ((c & 1 ? c_s1 : c_s0) + (uint32_t)(c >> 1)) & 1u);
+            tc_fence_after();
+            // the chunk's row maxima over its 128 positions
+#pragma unroll 1
+            for (int r = 0; r < rows_here; ++r) {
+                float a, b2;
+                tc_ld_2(tSc + r, tSc + 16 + r, a, b2);
+                const bool vis = pos < p_end && pos <= len + m_base + r;
+                float mx = vis ? (a + b2) * sc : -INFINITY;
+#pragma unroll
+                for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                if (lane == 0) wmax[warp * 16 + r] = mx;
+            }
+            named_bar(6, 128);
+            if (c > 0) {  // P V of the previous chunk has read the P tile and written O^T
+                wait(o_done, (c_o + c - 1) & 1u);
+                tc_fence_after();
+            }
+            bool moved = false;
+            uint8_t *panel = pt + (tid >> 6) * 4096;
+            const int cc = (tid & 63) >> 3, e = (tid & 7) * 2;
+#pragma unroll 1
+            for (int r = 0; r < rows_here; ++r) {
+                float a, b2;
+                tc_ld_2(tSc + r, tSc + 16 + r, a, b2);
+                const bool vis = pos < p_end && pos <= len + m_base + r;
+                const float v = vis ? (a + b2) * sc : -INFINITY;
+                const float mc = fmaxf(fmaxf(wmax[r], wmax[16 + r]), fmaxf(wmax[32 + r], wmax[48 + r]));
+                const float m_old = wmrun[warp * 16 + r], m_new = fmaxf(m_old, mc);
+                float f = 1.f, pv = 0.f;
+                if (m_new > -INFINITY) {
+                    f = exp2f(m_old - m_new);  // 0 on the first non-empty chunk
+                    pv = exp2f(v - m_new);
+                }
+                moved = moved || (f != 1.f);  // the same in all 128 threads: they read the same maxima
+                lrow[r * 128] = lrow[r * 128] * f + pv;
+                // P as bf16 hi + lo into the P tile: row r (hi) / 16 + r (lo), column = this position
+                const __nv_bfloat16 hv = __float2bfloat16_rn(pv);
+                *reinterpret_cast<__nv_bfloat16 *>(panel + sw128(r, cc) + e) = hv;
+                *reinterpret_cast<__nv_bfloat16 *>(panel + sw128(16 + r, cc) + e) = __float2bfloat16_rn(pv - __bfloat162float(hv));
+                __syncwarp();
+                if (lane == 0) { wmrun[warp * 16 + r] = m_new; fsh[warp * 16 + r] = f; }
+            }
+            __syncwarp();
+            if (c > 0 && moved) {  // thread = head dim tid: scale the accumulated O^T
+                float o[32];
+                tc_ld_32(tO + lane_sel, o);
+#pragma unroll
+                for (int r = 0; r < kAttnRows; ++r) {
+                    const float f = fsh[warp * 16 + r];  // 1 for rows beyond rows_here
+                    o[r] *= f;
+                    o[16 + r] *= f;
+                }
+                tc_st_32(tO + lane_sel, o);
+            }
+            fence_async_proxy();
+            tc_fence_before();
+            mbar_arrive(p_ready);
+        }
+        // ---- the sums over positions, then thread = head dim tid: output or partial ----
+#pragma unroll 1
+        for (int r = 0; r < rows_here; ++r) {
+            float t = lrow[r * 128];
+#pragma unroll
+            for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+            if (lane == 0) wsum[warp * 16 + r] = t;
+        }
+        if (n_chunks > 0) {
+            wait(o_done, (c_o + n_chunks - 1) & 1u);
+            tc_fence_after();
+        }
+        named_bar(6, 128);
+        const bool direct = p.n_split == 1;
+#pragma unroll 1
+        for (int r = 0; r < rows_here; ++r) {
+            const int m = m_base + r;
+            const float L = (wsum[r] + wsum[16 + r]) + (wsum[32 + r] + wsum[48 + r]);
+            const bool live = m < n_rows && L > 0.f && n_chunks > 0;
+            float a = 0.f, b2 = 0.f;
+            if (n_chunks > 0) tc_ld_2(tO + lane_sel + r, tO + lane_sel + 16 + r, a, b2);
+            const float acc = live ? a + b2 : 0.f;
+            if (direct) {
+                store_hilo(p.op[OP_AO], p.rk, r0 + m, h * Dh + tid, live ? acc / L : 0.f);
+            } else {
+                const size_t slot = ((size_t)(r0 + m) * p.H + h) * p.n_split + split;
+                if (tid == 0) {
+                    p.part_m[slot] = live ? wmrun[r] : -INFINITY;
+                    p.part_l[slot] = live ? L : 0.f;
+                }
+                p.part_o[slot * Dh + tid] = acc;
+            }
+        }
+        tc_fence_before();
+    }
+    if (p.n_split != 1) {
+        // ticket: the item that finishes last for this (sequence, head) merges all partials
+        __threadfence();
+        named_bar(3, kAttnThreadsP);
+        if (tid == 0) sh->flag = (atomicAdd(p.tickets + bh, 1u) == (unsigned)(p.n_split * MT - 1));
+        named_bar(3, kAttnThreadsP);
+        if (sh->flag) {
+            __threadfence();
+            merge_splits(p, r0, h, Dh);
+            if (tid == 0) p.tickets[bh] = 0;  // ready for the next layer (a grid barrier lies between)
+        }
+    }
+    if (tid == 0) {
+        for (int i = 0; i < 3; ++i) {
+            const uint32_t uses = (uint32_t)((2 * n_chunks + 2 - i) / 3);  // stages j < 2 n_chunks with j % 3 == i
+            acnt[AB_KV_FULL + i] = c_full[i] + uses;
+            acnt[AB_KV_FREE + i] = c_free[i] + uses;
+        }
+        acnt[AB_S_FULL] = c_s0 + (uint32_t)((n_chunks + 1) / 2);
+        acnt[AB_S_FULL + 1] = c_s1 + (uint32_t)(n_chunks / 2);
+        acnt[AB_P_READY] = c_p + n_chunks;
+        acnt[AB_O_DONE] = c_o + n_chunks;
+        acnt[AB_FIXED] = c_fix + n_fix_total;
+    }
+    named_bar(3, kAttnThreadsP);  // scratch, tensor memory and the counts are ready for the next item
+}
+
 __device__ __forceinline__ void attention_phase(const FwdParams &p, int layer, uint8_t *scratch, Shared *sh) {
     const int MT = (p.M + kAttnRows - 1) / kAttnRows;
     const int items = p.B * p.H * p.n_split * MT;
-    for (int item = blockIdx.x; item < items; item += gridDim.x) attention_item(p, layer, item, scratch, sh);
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        if (p.attn_tc) attention_item_tc(p, layer, item, scratch, sh);
+        else attention_item(p, layer, item, scratch, sh);
+    }
 }
 
 // ---- the kernel -----------------------------------------------------------------------------
@@ -975,6 +1423,8 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
     double *red = (double *)(sh + 1);
     float *epi_tile = (float *)(red + 16);
     volatile int *epi_ok = (volatile int *)(epi_tile + 8 * kEpiPitch);
+    uint64_t *abar = (uint64_t *)(epi_tile + 8 * kEpiPitch + 4);  // the tensor-core attention's barriers and counts
+    uint32_t *acnt = (uint32_t *)(abar + AB_COUNT);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp == 0) {  // tensor memory for the accumulators; released by the same warp at the end
@@ -994,15 +1444,21 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             mbar_init(&accEmpty[b], kEpiWarps);
         }
         mbar_init(mmaDone, 1);
+        for (int i = 0; i < AB_COUNT; ++i) {
+            mbar_init(&abar[i], i == AB_P_READY ? 128 : i == AB_FIXED ? 64 : 1);
+            acnt[i] = 0;
+        }
         sh->released = 0;
         sh->abort = 0;
         sh->go = 1;
+        sh->attn_bar_off = (uint32_t)((uint8_t *)abar - (uint8_t *)sh);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) sh->tmem_base = tmem_base;  // read after the next barrier only
     const int NG = n_gemms(p);
 
     if (warp == kConsumerWarps) {

@@ -31,6 +31,7 @@ std::mutex g_mu;
 // ---- optional per-launch timing of the kernel that streams the weights (forward_kernel for bf16
 //      models in single-kernel mode, otherwise every gemm launch) ----
 bool g_persistent = true;  // bf16 models: whole forward in one cooperative kernel
+int g_attn_mode = 0;       // 0: choose per pass; 1: warp-MMA attention items; 2: tensor-core items wherever they apply
 bool g_trace = false;       // stamp the global timer after every grid barrier of the forward kernel
 bool g_prof = false;
 std::vector<cudaEvent_t> g_prof_events;  // pairs
@@ -169,6 +170,8 @@ struct ssd_kv {
     int32_t *status, *len, *keep;
     uint8_t *cache;
     size_t layer_bytes, esize;
+    CUtensorMap tm_rows;  // bf16 caches of head dim 128: every (layer, sequence, K|V, head, position) row, box 64 x 128
+    bool tm_rows_ok;
     int len_ub;   // host-side upper bound of the committed lengths
     int last_rows;  // rows the last forward left uncommitted (upper bound bookkeeping)
 };
@@ -357,15 +360,15 @@ int gemm(const GemmCall &c, const void *W, const CUtensorMap *tw, const Operand 
 // Split of the position axis for a context of up to `ctx` positions, `groups` = independent
 // (sequence, head, row-tile) streams.  Every item pays a few microseconds of fixed latency, so the
 // aim is one round of items over the SMs: as many splits as keep groups * splits <= #SMs.
-void plan_split(int groups, int ctx, int *chunk, int *n_split) {
+void plan_split(int groups, int ctx, int *chunk, int *n_split, int tile = kAttnTile) {
     if (ctx < 1) ctx = 1;
     const int sms = g_num_sms > 0 ? g_num_sms : 148;
     int ns = ctx <= 256 ? 1 : sms / (groups > 0 ? groups : 1);
-    int max_by_len = ceil_div(ctx, 2 * kAttnTile);  // at least two chunks per split
+    int max_by_len = ceil_div(ctx, 2 * kAttnTile);  // at least 128 positions per split
     if (ns > max_by_len) ns = max_by_len;
     if (ns > kMaxSplit) ns = kMaxSplit;
     if (ns < 1) ns = 1;
-    int ch = ceil_div(ceil_div(ctx, ns), kAttnTile) * kAttnTile;
+    int ch = ceil_div(ceil_div(ctx, ns), tile) * tile;
     *chunk = ch;
     *n_split = ceil_div(ctx, ch);
 }
@@ -426,7 +429,8 @@ inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 4 
 template <int NT>
 int launch_forward_nt(FwdParams p, cudaStream_t st) {
     constexpr size_t stage = kWTileBytesP + 2 * NT * 8 * kTileK * 2;
-    const size_t attn = align_up(attn_scratch_bytes(p.Dh), 128);
+    size_t attn = align_up(attn_scratch_bytes(p.Dh), 128);
+    if (p.attn_tc && attn < (size_t)kTcScratchBytes) attn = kTcScratchBytes;
     const size_t tail = 24 * 32 + 64 + 16 + sizeof(Shared) + 16 * sizeof(double) + kEpiBytes + 256;  // barriers, small state, epilogue tile
     const size_t total = (size_t)kSmemBudget - 1024 - tail;
     // upper slots share their bytes with the attention scratch; at least two slots never do
@@ -501,7 +505,19 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     p.gbar = w.sync; p.tickets = w.sync + 16;
     int ctx = kv->len_ub + M;
     if (ctx > kv->S) ctx = kv->S;
-    plan_split(kv->B * a.n_heads * ((M + 15) / 16), ctx, &p.chunk, &p.n_split);
+    // Tensor-core attention items stream 128 positions per ~2 us but cost ~8 us more to start than the
+    // warp-MMA items (64 positions per ~2 us): they pay off from about a thousand positions per split.
+    const int groups = kv->B * a.n_heads * ((M + 15) / 16);
+    p.attn_tc = 0;
+    p.kv_rows_per_layer = kv->B * 2 * a.n_heads * kv->S;
+    if (a.head_dim == 128 && kv->tm_rows_ok && g_attn_mode != 1) {
+        plan_split(groups, ctx, &p.chunk, &p.n_split, kTcChunk);
+        if (p.chunk >= 1024 || g_attn_mode == 2) {
+            p.attn_tc = 1;
+            p.tm_kv = kv->tm_rows;
+        }
+    }
+    if (!p.attn_tc) plan_split(groups, ctx, &p.chunk, &p.n_split, kAttnTile);
     p.want_logits = want_logits ? 1 : 0;
     p.trace = (g_trace && 2 + barriers_needed(a) + 3 < kTraceSlots) ? w.trace : nullptr;
     CUDA_OK(cudaMemsetAsync(w.sync, 0, w.sync_bytes, st));
@@ -686,6 +702,12 @@ int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n
     return SSD_OK;
 }
 
+int ssd_set_attention_mode(int mode) {
+    if (mode < 0 || mode > 2) return SSD_E_ARG;
+    g_attn_mode = mode;
+    return SSD_OK;
+}
+
 int ssd_set_persistent(int enable) {
     g_persistent = enable != 0;
     return SSD_OK;
@@ -744,6 +766,17 @@ int kv_init(const ssd_model *m, int batch, int max_len, void *dev_buf, size_t by
     kv->layer_bytes = (size_t)batch * 2 * m->a.d_model * max_len * kv->esize;
     kv->len_ub = 0;
     kv->last_rows = 0;
+    // Rows beyond a sequence's length are read (masked) by the chunked attention: they must hold finite numbers.
+    if (cudaMemsetAsync(kv->cache, 0, kv->layer_bytes * m->a.n_layers, (cudaStream_t)stream) != cudaSuccess) {
+        delete kv;
+        return SSD_E_CUDA;
+    }
+    kv->tm_rows_ok = false;
+    {
+        const long long rows = (long long)m->a.n_layers * batch * 2 * m->a.n_heads * max_len;
+        if (m->a.dtype == 1 && m->a.head_dim == 128 && rows < (1ll << 31))
+            kv->tm_rows_ok = make_map(&kv->tm_rows, kv->cache, (int)rows, 128, kTcChunk) == SSD_OK;
+    }
     if (cudaMemsetAsync(dev_buf, 0, kv_header_bytes(batch), (cudaStream_t)stream) != cudaSuccess) {
         delete kv;
         return SSD_E_CUDA;

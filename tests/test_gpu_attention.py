@@ -43,3 +43,59 @@ def test_attention_rows_match_oracle(dtype, H, Dh, S, lens, rows):
     for b in range(Bn):
         ref = od.attention_rows(q[b], fill_f[0, b], lens[b], rows)
         assert np.abs(got[b] - ref).max() <= 2e-4, (b, np.abs(got[b] - ref).max())
+
+
+@pytest.mark.parametrize("mode", [2, 1])     # tensor-core items / warp-MMA items
+@pytest.mark.parametrize("lens,M", [
+    ([3000, 120], 20),      # 2 chunks per split, two 16-row tiles, rows of sequence 1 straddle position 128, empty splits
+    ([1000, 0], 5),         # one chunk per split; an empty cache beside it
+    ([255, 256], 3),        # rows start one before / exactly at a chunk boundary
+])
+def test_forward_over_a_long_seeded_cache_head_128(lens, M, mode):
+    """Whole verification pass (single forward kernel) of a 2-layer head-128 model over a seeded cache:
+    logits of all rows and the appended cache rows against the oracle.  Exercises the tensor-core
+    attention (mode 2) and the warp-MMA attention (mode 1): splits of several chunks, the merge of
+    splits, empty splits, more than 16 rows per sequence, and rows of the pass that cross a chunk
+    boundary."""
+    arch = synth.llama_like(2, 256, 2, 512, 512)
+    assert arch.head_dim == 128
+    from tests import gpu_util as gu
+    ws_np = gu.scaled_weights(synth, arch, 11, 6.0)
+    model = B.Model(arch, B.upload_weights(arch, ws_np))
+    omodel = od.Model(arch, ws_np)
+    Bn, S = len(lens), max(lens) + 64
+    kv = B.KV(model, Bn, S)
+    fill = synth.gen_kv_fill(12, (arch.n_layers, Bn, 2, arch.n_heads, S, arch.head_dim), arch.dtype)
+    fill_f = synth.bf16_bits_to_f32(fill) * np.float32(0.5)
+    fill = synth.f32_to_bf16_bits(fill_f)            # halving is exact in bf16
+    dev = "cuda"
+    kv.cache_view().copy_(torch.from_numpy(fill.view(np.int16)).to(dev).view(torch.bfloat16))
+    B.kv_commit(kv, torch.tensor(lens, dtype=torch.int32, device=dev))
+    assert kv.lengths().tolist() == lens      # also refreshes the host-side bound the splits are planned from
+    rows = synth.gen_prompt(13, Bn, M, arch.vocab)
+    ws = model.new_workspace(Bn, M, S)
+    V = arch.vocab
+    K = M - 1
+    n_acc = torch.zeros(Bn, dtype=torch.int32, device=dev)
+    nxt = torch.zeros(Bn, dtype=torch.int32, device=dev)
+    q = torch.full((Bn, max(K, 1), V), 1.0 / V, device=dev)
+    u = torch.full((Bn, M), 0.5, device=dev)
+    B.set_attention_mode(mode)
+    try:
+        B.target_verify(model, kv, torch.from_numpy(rows).to(dev), K, q, u, 1.0, n_acc, nxt, 1, None, ws)
+        got = B.last_logits(model, Bn, M, ws).cpu().numpy()
+    finally:
+        B.set_attention_mode(0)
+    assert kv.status() == 0
+    cache = kv.cache_view().float().cpu().numpy()
+    od.set_threads(8)
+    for b in range(Bn):
+        oc = omodel.new_cache(S)
+        oc.kv[...] = fill_f[:, b]
+        oc.len = lens[b]
+        ref = oc.feed(rows[b], advance=False)
+        gu.assert_logits_close(got[b], ref)
+        n0, n1 = lens[b], lens[b] + M
+        g, r = cache[:, b, :, :, n0:n1], oc.kv[:, :, :, n0:n1]
+        assert (np.abs(g - r) <= gu.LOGIT_RTOL * np.abs(r) + gu.LOGIT_ATOL).all()
+        assert np.array_equal(cache[:, b, :, :, :n0], fill_f[:, b, :, :, :n0])   # committed rows untouched
