@@ -212,7 +212,7 @@ constexpr int kAccStride = 256;
 constexpr int kEpiWarps = 4;    // warps 0-3: one tensor-memory lane quadrant each
 constexpr int kMmaWarp = 4;
 constexpr int kEpiPitch = kTileNP + 8;             // floats per row of the epilogue tile (bank spread)
-constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 11 * 8 + 11 * 4 + 12;  // 8 rows, the four warps' wait results, attention barriers
+constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 12 * 8 + 12 * 4 + 16;  // 8 rows, the four warps' wait results, attention barriers
 constexpr int kXWarp = 5;      // issues the operand copies of a GEMM phase
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -1005,8 +1005,12 @@ constexpr int kTcKvStage = kTcChunk * 128 * 2;  // one K or V chunk: two 64-colu
 constexpr int kTcQOff = 3 * kTcKvStage, kTcPOff = kTcQOff + 8192, kTcMiscOff = kTcPOff + 8192;
 constexpr int kTcScratchBytes = kTcMiscOff + 1536 + kAttnRows * 128 * 4;  // + per-thread running sums [16][128]
 // Its mbarriers live outside the scratch (which the weight ring reuses), are initialised once per kernel
-// and keep running: cnt[i] = phases barrier i has completed before the current item.
-enum { AB_KV_FULL = 0, AB_KV_FREE = 3, AB_S_FULL = 6, AB_P_READY = 8, AB_O_DONE = 9, AB_FIXED = 10, AB_COUNT = 11 };
+// and keep running: cnt[i] = phases barrier i has completed before the current item.  A parity wait is
+// only meaningful for a waiter that follows every phase of its barrier in order and that the barrier
+// cannot pass by two phases; the threads that patch this pass's rows into a chunk skip most chunks, so
+// they do not wait on the ring's barriers: the MMA issuer, which follows every stage, tells them through
+// `landed` when such a chunk has arrived, and hears back through `fixed`.
+enum { AB_KV_FULL = 0, AB_KV_FREE = 3, AB_S_FULL = 6, AB_P_READY = 8, AB_O_DONE = 9, AB_FIXED = 10, AB_LANDED = 11, AB_COUNT = 12 };
 
 __device__ __forceinline__ void tc_ld_32(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
@@ -1022,6 +1026,20 @@ __device__ __forceinline__ void tc_ld_32(uint32_t taddr, float (&v)[32]) {
         : "memory");
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+// eight columns from each of two places of this warp's lane quadrant, one round trip
+__device__ __forceinline__ void tc_ld_2x8(uint32_t ta, uint32_t tb, float (&a)[8], float (&b)[8]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%16];\n"
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%8,%9,%10,%11,%12,%13,%14,%15}, [%17];\n"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(ta), "r"(tb)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { a[i] = __uint_as_float(r[i]); b[i] = __uint_as_float(r[8 + i]); }
 }
 // one column from each of two places of this warp's lane quadrant
 __device__ __forceinline__ void tc_ld_2(uint32_t ta, uint32_t tb, float &a, float &b) {
@@ -1079,7 +1097,7 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
     float *l_sh = fsh + 64;                                         // [16][128] running sums, one per (row, thread)
     uint64_t *kv_full = abar + AB_KV_FULL, *kv_free = abar + AB_KV_FREE;  // [3] each
     uint64_t *s_full = abar + AB_S_FULL;  // [2]: the scores are double-buffered in tensor memory
-    uint64_t *p_ready = abar + AB_P_READY, *o_done = abar + AB_O_DONE, *fixed = abar + AB_FIXED;
+    uint64_t *p_ready = abar + AB_P_READY, *o_done = abar + AB_O_DONE, *fixed = abar + AB_FIXED, *landed = abar + AB_LANDED;
 
     const int n_rows = __ldcg(p.ri.n_eff + b);
     const int len = p.len[b];
@@ -1108,7 +1126,7 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
 #pragma unroll
     for (int i = 0; i < 3; ++i) { c_full[i] = acnt[AB_KV_FULL + i]; c_free[i] = acnt[AB_KV_FREE + i]; }
     const uint32_t c_s0 = acnt[AB_S_FULL], c_s1 = acnt[AB_S_FULL + 1];
-    const uint32_t c_p = acnt[AB_P_READY], c_o = acnt[AB_O_DONE], c_fix = acnt[AB_FIXED];
+    const uint32_t c_p = acnt[AB_P_READY], c_o = acnt[AB_O_DONE], c_fix = acnt[AB_FIXED], c_land = acnt[AB_LANDED];
     auto full_par = [&](int j) { return (c_full[j % 3] + (uint32_t)(j / 3)) & 1u; };          // stage j has landed
     auto free_par = [&](int j) { return ((c_free[j % 3] + (uint32_t)(j / 3)) & 1u) ^ 1u; };   // its slot was released
     int n_fix_total = 0;
@@ -1176,7 +1194,12 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
                 const int jk = 2 * c, jv = 2 * c + 1;
                 const bool fix = p_begin + (c + 1) * kTcChunk > len;
                 wait(&kv_full[jk % 3], full_par(jk));
-                if (fix) { wait(&kv_full[jv % 3], full_par(jv)); wait(fixed, (c_fix + n_fix) & 1u); ++n_fix; }
+                if (fix) {  // both tiles are here: let the patching threads in, wait for them
+                    wait(&kv_full[jv % 3], full_par(jv));
+                    if (!sh->abort) mbar_arrive(landed);
+                    wait(fixed, (c_fix + n_fix) & 1u);
+                    ++n_fix;
+                }
                 if (sh->abort) return;
                 tc_fence_after();
                 const uint32_t ka = smem_u32(ring + (jk % 3) * kTcKvStage);
@@ -1208,6 +1231,7 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
     } else if (warp >= 6) {
         // ---------------- rows of this pass, chunk by chunk ----------------
         const int ft = tid - 192;  // 0..63
+        int n_fixed = 0;
         for (int c = 0; c < n_chunks; ++c) {
             const int base = p_begin + c * kTcChunk;
             if (base + kTcChunk <= len) continue;
@@ -1238,8 +1262,8 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
                     vq[u] = *reinterpret_cast<uint4 *>(vb);
                 }
             }
-            wait(&kv_full[jk % 3], full_par(jk));
-            wait(&kv_full[jv % 3], full_par(jv));
+            wait(landed, (c_land + (uint32_t)n_fixed) & 1u);
+            ++n_fixed;
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const int i = ft + 64 * u, pr = first + (i >> 4), v8 = i & 15;
@@ -1272,16 +1296,30 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
             float *wmax = wmax2 + 64 * (c & 1);
             wait(&s_full[c & 1], ((c & 1 ? c_s1 : c_s0) + (uint32_t)(c >> 1)) & 1u);
             tc_fence_after();
-            // the chunk's row maxima over its 128 positions
+            // the chunk's row maxima over its 128 positions; 8 rows per tensor-memory round trip, unrolled
+            // over those 8 so that their shuffles and exponentials overlap
+            const int nblk = (rows_here + 7) >> 3;
 #pragma unroll 1
-            for (int r = 0; r < rows_here; ++r) {
-                float a, b2;
-                tc_ld_2(tSc + r, tSc + 16 + r, a, b2);
-                const bool vis = pos < p_end && pos <= len + m_base + r;
-                float mx = vis ? (a + b2) * sc : -INFINITY;
+            for (int blk = 0; blk < nblk; ++blk) {
+                float a[8], b2[8];
+                tc_ld_2x8(tSc + 8 * blk, tSc + 16 + 8 * blk, a, b2);
+                float mx[8];
 #pragma unroll
-                for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                if (lane == 0) wmax[warp * 16 + r] = mx;
+                for (int i = 0; i < 8; ++i) {
+                    const int r = 8 * blk + i;
+                    const bool vis = r < rows_here && pos < p_end && pos <= len + m_base + r;
+                    mx[i] = vis ? (a[i] + b2[i]) * sc : -INFINITY;
+                }
+#pragma unroll
+                for (int o = 16; o; o >>= 1)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], o));
+                if (lane < 8) {
+                    float sel = mx[0];
+#pragma unroll
+                    for (int i = 1; i < 8; ++i) sel = lane == i ? mx[i] : sel;
+                    wmax[warp * 16 + 8 * blk + lane] = sel;
+                }
             }
             named_bar(6, 128);
             if (c > 0) {  // P V of the previous chunk has read the P tile and written O^T
@@ -1292,26 +1330,46 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
             uint8_t *panel = pt + (tid >> 6) * 4096;
             const int cc = (tid & 63) >> 3, e = (tid & 7) * 2;
 #pragma unroll 1
-            for (int r = 0; r < rows_here; ++r) {
-                float a, b2;
-                tc_ld_2(tSc + r, tSc + 16 + r, a, b2);
-                const bool vis = pos < p_end && pos <= len + m_base + r;
-                const float v = vis ? (a + b2) * sc : -INFINITY;
-                const float mc = fmaxf(fmaxf(wmax[r], wmax[16 + r]), fmaxf(wmax[32 + r], wmax[48 + r]));
-                const float m_old = wmrun[warp * 16 + r], m_new = fmaxf(m_old, mc);
-                float f = 1.f, pv = 0.f;
-                if (m_new > -INFINITY) {
-                    f = exp2f(m_old - m_new);  // 0 on the first non-empty chunk
-                    pv = exp2f(v - m_new);
+            for (int blk = 0; blk < nblk; ++blk) {
+                float a[8], b2[8];
+                tc_ld_2x8(tSc + 8 * blk, tSc + 16 + 8 * blk, a, b2);
+                float fl[8], ml[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = 8 * blk + i;
+                    fl[i] = 1.f;
+                    ml[i] = -INFINITY;
+                    if (r < rows_here) {
+                        const bool vis = pos < p_end && pos <= len + m_base + r;
+                        const float v = vis ? (a[i] + b2[i]) * sc : -INFINITY;
+                        const float mc = fmaxf(fmaxf(wmax[r], wmax[16 + r]), fmaxf(wmax[32 + r], wmax[48 + r]));
+                        const float m_old = wmrun[warp * 16 + r], m_new = fmaxf(m_old, mc);
+                        float pv = 0.f;
+                        if (m_new > -INFINITY) {
+                            fl[i] = exp2f(m_old - m_new);  // 0 on the first non-empty chunk
+                            pv = exp2f(v - m_new);
+                        }
+                        ml[i] = m_new;
+                        moved = moved || (fl[i] != 1.f);  // the same in all 128 threads: they read the same maxima
+                        lrow[r * 128] = lrow[r * 128] * fl[i] + pv;
+                        // P as bf16 hi + lo into the P tile: row r (hi) / 16 + r (lo), column = this position
+                        const __nv_bfloat16 hv = __float2bfloat16_rn(pv);
+                        *reinterpret_cast<__nv_bfloat16 *>(panel + sw128(r, cc) + e) = hv;
+                        *reinterpret_cast<__nv_bfloat16 *>(panel + sw128(16 + r, cc) + e) =
+                            __float2bfloat16_rn(pv - __bfloat162float(hv));
+                    }
                 }
-                moved = moved || (f != 1.f);  // the same in all 128 threads: they read the same maxima
-                lrow[r * 128] = lrow[r * 128] * f + pv;
-                // P as bf16 hi + lo into the P tile: row r (hi) / 16 + r (lo), column = this position
-                const __nv_bfloat16 hv = __float2bfloat16_rn(pv);
-                *reinterpret_cast<__nv_bfloat16 *>(panel + sw128(r, cc) + e) = hv;
-                *reinterpret_cast<__nv_bfloat16 *>(panel + sw128(16 + r, cc) + e) = __float2bfloat16_rn(pv - __bfloat162float(hv));
-                __syncwarp();
-                if (lane == 0) { wmrun[warp * 16 + r] = m_new; fsh[warp * 16 + r] = f; }
+                __syncwarp();  // every lane has read this block's running maxima
+                if (lane < 8 && 8 * blk + lane < rows_here) {
+                    float msel = ml[0], fsel = fl[0];
+#pragma unroll
+                    for (int i = 1; i < 8; ++i) {
+                        msel = lane == i ? ml[i] : msel;
+                        fsel = lane == i ? fl[i] : fsel;
+                    }
+                    wmrun[warp * 16 + 8 * blk + lane] = msel;
+                    fsh[warp * 16 + 8 * blk + lane] = fsel;
+                }
             }
             __syncwarp();
             if (c > 0 && moved) {  // thread = head dim tid: scale the accumulated O^T
@@ -1387,6 +1445,7 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
         acnt[AB_P_READY] = c_p + n_chunks;
         acnt[AB_O_DONE] = c_o + n_chunks;
         acnt[AB_FIXED] = c_fix + n_fix_total;
+        acnt[AB_LANDED] = c_land + n_fix_total;
     }
     named_bar(3, kAttnThreadsP);  // scratch, tensor memory and the counts are ready for the next item
 }
@@ -1445,7 +1504,7 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
         }
         mbar_init(mmaDone, 1);
         for (int i = 0; i < AB_COUNT; ++i) {
-            mbar_init(&abar[i], i == AB_P_READY ? 128 : i == AB_FIXED ? 64 : 1);
+            mbar_init(&abar[i], i == AB_P_READY ? 128 : i == AB_FIXED ? 64 : 1);  // landed: the MMA issuer alone
             acnt[i] = 0;
         }
         sh->released = 0;

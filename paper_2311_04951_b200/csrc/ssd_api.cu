@@ -433,14 +433,15 @@ int launch_forward_nt(FwdParams p, cudaStream_t st) {
     if (p.attn_tc && attn < (size_t)kTcScratchBytes) attn = kTcScratchBytes;
     const size_t tail = 24 * 32 + 64 + 16 + sizeof(Shared) + 16 * sizeof(double) + kEpiBytes + 256;  // barriers, small state, epilogue tile
     const size_t total = (size_t)kSmemBudget - 1024 - tail;
-    // upper slots share their bytes with the attention scratch; at least two slots never do
+    // upper slots share their bytes with the attention scratch; two slots never do where they fit
+    // (one with the 48 KB stages of 64 rows, which only the prompt pass uses)
     size_t S2 = (attn + stage - 1) / stage;
     size_t region2 = S2 * stage;
     if (region2 + 2 * stage > total) {
         S2 = attn / stage;
         region2 = attn;
     }
-    if (region2 + 2 * stage > total) return SSD_E_CAPACITY;
+    if (region2 + stage > total) return SSD_E_CAPACITY;
     size_t S1 = (total - region2) / stage;
     if (S1 + S2 > 32) S1 = 32 - S2;  // one parity bit per slot
     p.stages = (int)(S1 + S2);

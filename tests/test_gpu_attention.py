@@ -52,15 +52,27 @@ def test_attention_rows_match_oracle(dtype, H, Dh, S, lens, rows):
     ([255, 256], 3),        # rows start one before / exactly at a chunk boundary
 ])
 def test_forward_over_a_long_seeded_cache_head_128(lens, M, mode):
-    """Whole verification pass (single forward kernel) of a 2-layer head-128 model over a seeded cache:
+    _forward_over_seeded_cache(synth.llama_like(2, 256, 2, 512, 512), lens, M, mode)
+
+
+@pytest.mark.parametrize("mode", [2, 1])
+def test_forward_many_heads_one_split_of_many_chunks(mode):
+    """160 (sequence, head) pairs on 148 SMs: one split per pair, up to ten 128-position chunks each (the
+    K/V ring wraps several times), some SMs run two items in a row, and lengths of 127 mod 128 put the rows
+    of the pass into the last two chunks."""
+    # weights x1.5: the same activation scale at d = 4096 as x6 gives at d = 256
+    _forward_over_seeded_cache(synth.llama_like(1, 4096, 32, 512, 512), [1151, 127, 1152, 64, 300], 5, mode, scale=1.5)
+
+
+def _forward_over_seeded_cache(arch, lens, M, mode, scale=6.0):
+    """Whole verification pass (single forward kernel) of a head-128 model over a seeded cache:
     logits of all rows and the appended cache rows against the oracle.  Exercises the tensor-core
     attention (mode 2) and the warp-MMA attention (mode 1): splits of several chunks, the merge of
     splits, empty splits, more than 16 rows per sequence, and rows of the pass that cross a chunk
     boundary."""
-    arch = synth.llama_like(2, 256, 2, 512, 512)
     assert arch.head_dim == 128
     from tests import gpu_util as gu
-    ws_np = gu.scaled_weights(synth, arch, 11, 6.0)
+    ws_np = gu.scaled_weights(synth, arch, 11, scale)
     model = B.Model(arch, B.upload_weights(arch, ws_np))
     omodel = od.Model(arch, ws_np)
     Bn, S = len(lens), max(lens) + 64
