@@ -165,11 +165,31 @@ __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi) {
     return g;
 }
 
-// This CTA's contiguous share of a GEMM's (tile, k-chunk) units.
-__device__ __forceinline__ void unit_range(const GemmDesc &g, int &c0, int &c1) {
+// This CTA's contiguous share of a GEMM's (tile, k-chunk) units.  Equal shares, except in the GEMM that
+// follows the attention phase (MLP-out of a parallel-residual block, out-projection otherwise) when
+// at most half of the CTAs ran an attention item: those enter the phase with only the lower ring
+// slots filled ahead, the others with the whole ring, so they get that many units fewer.
+__device__ __forceinline__ void unit_range(const FwdParams &p, const GemmDesc &g, int &c0, int &c1) {
     const long long total = (long long)g.n_tiles * g.kchunks;
-    c0 = (int)(total * blockIdx.x / gridDim.x);
-    c1 = (int)(total * (blockIdx.x + 1) / gridDim.x);
+    const int N = (int)gridDim.x, i = (int)blockIdx.x;
+    const int items = p.B * p.H * p.n_split * ((p.M + 15) / 16);
+    const int A = items < N ? items : N, bonus = p.stages - p.stages_lo;
+    const bool after_attention = p.parallel ? g.kind == 3 : g.kind == 1;
+    if (after_attention && 2 * A <= N && bonus > 0) {  // (with most CTAs on attention the few others would become the stragglers)
+        long long xa = (total + (long long)A * bonus) / N - bonus;  // an attention CTA's share
+        if (xa < 0) xa = 0;
+        const long long rest = total - xa * A;                      // over the N - A others
+        if (i < A) {
+            c0 = (int)(xa * i);
+            c1 = (int)(xa * (i + 1));
+        } else {
+            c0 = (int)(xa * A + rest * (i - A) / (N - A));
+            c1 = (int)(xa * A + rest * (i - A + 1) / (N - A));
+        }
+        return;
+    }
+    c0 = (int)(total * i / N);
+    c1 = (int)(total * (i + 1) / N);
 }
 
 __device__ __forceinline__ void named_bar(int id, int count) {
@@ -212,7 +232,7 @@ constexpr int kAccStride = 256;
 constexpr int kEpiWarps = 4;    // warps 0-3: one tensor-memory lane quadrant each
 constexpr int kMmaWarp = 4;
 constexpr int kEpiPitch = kTileNP + 8;             // floats per row of the epilogue tile (bank spread)
-constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 12 * 8 + 12 * 4 + 16;  // 8 rows, the four warps' wait results, attention barriers
+constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 12 * 8 + 12 * 4 + 16 + 2 * 16 + 8 * 4;  // 8 rows, the four warps' wait results, attention barriers
 constexpr int kXWarp = 5;      // issues the operand copies of a GEMM phase
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -1459,127 +1479,78 @@ __device__ __forceinline__ void attention_phase(const FwdParams &p, int layer, u
     }
 }
 
-// ---- the kernel -----------------------------------------------------------------------------
-// NT = padded rows / 8
+// Where the kernel's small state lives behind the ring (and the attention scratch) in shared memory.
+struct SmemMap {
+    uint64_t *fullW, *fullX, *empty, *accFull, *accEmpty, *mmaDone;
+    uint32_t *tmem_slot;
+    Shared *sh;
+    double *red;
+    float *epi_tile;
+    volatile int *epi_ok;
+    uint64_t *abar;
+    uint32_t *acnt;
+    RingPos *role_rp;  // [2]: the MMA issuer's and the operand issuer's walk of the ring, between GEMMs
+    int *role_seg;     // [8]: per work warp, tile segments so far
+};
+__device__ __forceinline__ SmemMap smem_map(const FwdParams &p, uint8_t *smem) {
+    SmemMap m;
+    const int S = p.stages;
+    m.fullW = (uint64_t *)(smem + p.bar_off);
+    m.fullX = m.fullW + S;
+    m.empty = m.fullX + S;
+    m.accFull = m.empty + S;
+    m.accEmpty = m.accFull + 2;
+    m.mmaDone = m.accEmpty + 2;
+    m.tmem_slot = (uint32_t *)(m.mmaDone + 1);
+    m.sh = (Shared *)(((uintptr_t)(m.mmaDone + 4) + 15) & ~(uintptr_t)15);
+    m.red = (double *)(m.sh + 1);
+    m.epi_tile = (float *)(m.red + 16);
+    m.epi_ok = (volatile int *)(m.epi_tile + 8 * kEpiPitch);
+    m.abar = (uint64_t *)(m.epi_tile + 8 * kEpiPitch + 4);
+    m.acnt = (uint32_t *)(m.abar + AB_COUNT);
+    m.role_rp = (RingPos *)(m.acnt + AB_COUNT);
+    m.role_seg = (int *)(m.role_rp + 2);
+    return m;
+}
+
+// Run this CTA's units of GEMM gi (all 256 work threads call it; NT = padded rows / 8).  The units are
+// contiguous in (tile, k-chunk) order, so they form one segment per tile touched; each segment is
+// accumulated in tensor memory and reduced into the output once.  A function of its own, with the
+// little state that survives from GEMM to GEMM kept in shared memory, so that the kernel's phase loop
+// holds nothing across its calls: with 227 KB of shared memory there is next to no L1 left, and a
+// value spilled to the stack costs an L2 round trip at every phase.
 template <int NT>
-__global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __grid_constant__ FwdParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+__device__ __noinline__ void run_gemm(const FwdParams &p, int gi, uint8_t *smem) {
     constexpr int kRp = NT * 8;
-    constexpr int kXBytes = 2 * kRp * kTileK * 2;  // operand tile (hi and lo rows), then the weight tile
+    constexpr int kXBytes = 2 * kRp * kTileK * 2;
     constexpr int kStageBytes = kXBytes + kWTileBytesP;
     // M of the MMA: the operand tile's 2 kRp rows; the rows the MMA reads beyond them are the weight
     // tile's bytes (finite or not, they only reach accumulator lanes that nobody loads)
     constexpr int kM = 2 * kRp <= 64 ? 64 : 128;
+    const SmemMap mp = smem_map(p, smem);
     const int S = p.stages, S1 = p.stages_lo;
     uint8_t *ring = smem;
-    uint8_t *attn_scratch = smem + p.attn_smem_off;
-    uint64_t *fullW = (uint64_t *)(smem + p.bar_off);
-    uint64_t *fullX = fullW + S, *empty = fullX + S;
-    uint64_t *accFull = empty + S, *accEmpty = accFull + 2, *mmaDone = accEmpty + 2;
-    uint32_t *tmem_slot = (uint32_t *)(mmaDone + 1);
-    Shared *sh = (Shared *)(((uintptr_t)(mmaDone + 4) + 15) & ~(uintptr_t)15);
-    double *red = (double *)(sh + 1);
-    float *epi_tile = (float *)(red + 16);
-    volatile int *epi_ok = (volatile int *)(epi_tile + 8 * kEpiPitch);
-    uint64_t *abar = (uint64_t *)(epi_tile + 8 * kEpiPitch + 4);  // the tensor-core attention's barriers and counts
-    uint32_t *acnt = (uint32_t *)(abar + AB_COUNT);
-
+    uint64_t *fullW = mp.fullW, *fullX = mp.fullX, *empty = mp.empty, *accFull = mp.accFull, *accEmpty = mp.accEmpty;
+    Shared *sh = mp.sh;
+    float *epi_tile = mp.epi_tile;
+    volatile int *epi_ok = mp.epi_ok;
+    const uint32_t tmem_base = sh->tmem_base;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (warp == 0) {  // tensor memory for the accumulators; released by the same warp at the end
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "n"(kTmemCols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(&fullW[s], 1);
-            mbar_init(&fullX[s], 1);
-            mbar_init(&empty[s], 1);  // one tcgen05.commit per stage
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&accFull[b], 1);
-            mbar_init(&accEmpty[b], kEpiWarps);
-        }
-        mbar_init(mmaDone, 1);
-        for (int i = 0; i < AB_COUNT; ++i) {
-            mbar_init(&abar[i], i == AB_P_READY ? 128 : i == AB_FIXED ? 64 : 1);  // landed: the MMA issuer alone
-            acnt[i] = 0;
-        }
-        sh->released = 0;
-        sh->abort = 0;
-        sh->go = 1;
-        sh->attn_bar_off = (uint32_t)((uint8_t *)abar - (uint8_t *)sh);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    if (threadIdx.x == 0) sh->tmem_base = tmem_base;  // read after the next barrier only
-    const int NG = n_gemms(p);
+    const bool walks_ring = lane == 0 && (warp == kMmaWarp || warp == kXWarp);
+    RingPos rp;
+    if (walks_ring) rp = mp.role_rp[warp == kMmaWarp ? 0 : 1];
+    int seg = mp.role_seg[warp];
+    auto save_state = [&]() {
+        if (walks_ring) mp.role_rp[warp == kMmaWarp ? 0 : 1] = rp;
+        __syncwarp();
+        if (lane == 0) mp.role_seg[warp] = seg;
+        __syncwarp();
+    };
 
-    if (warp == kConsumerWarps) {
-        // =============================== producer ===============================
-        // Weights never change, so this cursor runs as far ahead as the ring allows, across grid
-        // barriers.  The loop is kept minimal (no divisions, no clock reads while it makes progress):
-        // its rate bounds the weight stream.
-        if (lane == 0) {
-            RingPos rp;
-            bool failed = false;
-            int seen_release = 0;
-            for (int gw = 0; gw < NG && !failed; ++gw) {
-                const GemmDesc dw = gemm_desc(p, gw);
-                int c0, c1;
-                unit_range(dw, c0, c1);
-                if (c0 >= c1) continue;
-                int tw = c0 / dw.kchunks, kw = c0 % dw.kchunks;
-                for (int c = c0; c < c1; ++c) {
-                    uint32_t ph;
-                    const int s = ring_next(rp, ring_lo_only(dw, c - c0, S1), S, S1, ph);
-                    if (s >= S1 && seen_release < dw.need_hi) {  // slot shared with the attention scratch
-                        const long long t0 = clock64();
-                        while ((seen_release = sh->released) < dw.need_hi) {
-                            if (sh->abort || clock64() - t0 > kWaitCycles) { failed = true; break; }
-                        }
-                        if (failed) { rp.par ^= 1u << s; break; }  // nothing was issued into s
-                    }
-                    if (!mbar_test_wait(&empty[s], ph ^ 1u)) {
-                        const long long t0 = clock64();
-                        while (!mbar_test_wait(&empty[s], ph ^ 1u)) {
-                            if (sh->abort || clock64() - t0 > kWaitCycles) { failed = true; break; }
-                        }
-                        if (failed) { rp.par ^= 1u << s; break; }  // nothing was issued into s
-                    }
-                    mbar_expect_tx(&fullW[s], kWTileBytesP);
-                    tma_load_2d(ring + (size_t)s * kStageBytes + kXBytes, dw.tmW, kw * kTileK, tw * kTileNP, &fullW[s]);
-                    if (++kw == dw.kchunks) { kw = 0; ++tw; }
-                }
-            }
-            if (failed) {
-                set_status(p.status, kTimeoutCode);
-                sh->abort = 1;
-            }
-            // error path only: wait (bounded) for copies still in flight before the CTA may exit
-            if (sh->abort)
-                for (int s = 0; s < S; ++s)
-                    if ((rp.used >> s) & 1u) mbar_wait(&fullW[s], ((rp.par >> s) & 1u) ^ 1u);
-        }
-    } else {
-        // =============================== work warps ===============================
-        int epoch = 0;  // grid barriers passed
-        RingPos rp;     // this thread's walk of the ring (used by the MMA and the operand issuer)
-        int seg = 0;    // tile segments so far: segment q accumulates in buffer q & 1
-
-        // Run this CTA's units of GEMM gi.  The units are contiguous in (tile, k-chunk) order, so they
-        // form one segment per tile touched; each segment is accumulated in tensor memory and
-        // reduced into the output once.
-        auto run_gemm = [&](int gi) {
             const GemmDesc g = gemm_desc(p, gi);
             int c0, c1;
-            unit_range(g, c0, c1);
-            if (c0 >= c1) return;
+            unit_range(p, g, c0, c1);
+            if (c0 >= c1) return;  // (no state to save: nothing moved)
             const int tile0 = c0 / g.kchunks, tile1 = (c1 - 1) / g.kchunks;
             if (warp == kMmaWarp) {
                 if (lane == 0 && !sh->abort) {
@@ -1701,7 +1672,123 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                 }
             }
             seg += tile1 - tile0 + 1;
-        };
+            save_state();
+}
+
+// ---- the kernel -----------------------------------------------------------------------------
+// NT = padded rows / 8
+template <int NT>
+__global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __grid_constant__ FwdParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    constexpr int kRp = NT * 8;
+    constexpr int kXBytes = 2 * kRp * kTileK * 2;  // operand tile (hi and lo rows), then the weight tile
+    constexpr int kStageBytes = kXBytes + kWTileBytesP;
+    const int S = p.stages, S1 = p.stages_lo;
+    uint8_t *ring = smem;
+    uint8_t *attn_scratch = smem + p.attn_smem_off;
+    uint64_t *fullW = (uint64_t *)(smem + p.bar_off);
+    uint64_t *fullX = fullW + S, *empty = fullX + S;
+    uint64_t *accFull = empty + S, *accEmpty = accFull + 2, *mmaDone = accEmpty + 2;
+    uint32_t *tmem_slot = (uint32_t *)(mmaDone + 1);
+    Shared *sh = (Shared *)(((uintptr_t)(mmaDone + 4) + 15) & ~(uintptr_t)15);
+    double *red = (double *)(sh + 1);
+    float *epi_tile = (float *)(red + 16);
+    uint64_t *abar = (uint64_t *)(epi_tile + 8 * kEpiPitch + 4);  // the tensor-core attention's barriers and counts
+    uint32_t *acnt = (uint32_t *)(abar + AB_COUNT);
+    RingPos *role_rp = (RingPos *)(acnt + AB_COUNT);  // the same places smem_map() gives
+    int *role_seg = (int *)(role_rp + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == 0) {  // tensor memory for the accumulators; released by the same warp at the end
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "n"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(&fullW[s], 1);
+            mbar_init(&fullX[s], 1);
+            mbar_init(&empty[s], 1);  // one tcgen05.commit per stage
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&accFull[b], 1);
+            mbar_init(&accEmpty[b], kEpiWarps);
+        }
+        mbar_init(mmaDone, 1);
+        for (int i = 0; i < AB_COUNT; ++i) {
+            mbar_init(&abar[i], i == AB_P_READY ? 128 : i == AB_FIXED ? 64 : 1);  // landed: the MMA issuer alone
+            acnt[i] = 0;
+        }
+        role_rp[0] = RingPos();
+        role_rp[1] = RingPos();
+        for (int i = 0; i < 8; ++i) role_seg[i] = 0;
+        sh->released = 0;
+        sh->abort = 0;
+        sh->go = 1;
+        sh->attn_bar_off = (uint32_t)((uint8_t *)abar - (uint8_t *)sh);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) sh->tmem_base = tmem_base;  // read after the next barrier only
+    const int NG = n_gemms(p);
+
+    if (warp == kConsumerWarps) {
+        // =============================== producer ===============================
+        // Weights never change, so this cursor runs as far ahead as the ring allows, across grid
+        // barriers.  The loop is kept minimal (no divisions, no clock reads while it makes progress):
+        // its rate bounds the weight stream.
+        if (lane == 0) {
+            RingPos rp;
+            bool failed = false;
+            int seen_release = 0;
+            // a CTA that never runs an attention item (fewer items than CTAs) never uses the scratch: its
+            // upper slots take weights at any time
+            const bool scratch_used = (int)blockIdx.x < p.B * p.H * p.n_split * ((p.M + kAttnRows - 1) / kAttnRows);
+            for (int gw = 0; gw < NG && !failed; ++gw) {
+                const GemmDesc dw = gemm_desc(p, gw);
+                int c0, c1;
+                unit_range(p, dw, c0, c1);
+                if (c0 >= c1) continue;
+                int tw = c0 / dw.kchunks, kw = c0 % dw.kchunks;
+                for (int c = c0; c < c1; ++c) {
+                    uint32_t ph;
+                    const int s = ring_next(rp, ring_lo_only(dw, c - c0, S1), S, S1, ph);
+                    if (s >= S1 && scratch_used && seen_release < dw.need_hi) {  // slot shared with the attention scratch
+                        const long long t0 = clock64();
+                        while ((seen_release = sh->released) < dw.need_hi) {
+                            if (sh->abort || clock64() - t0 > kWaitCycles) { failed = true; break; }
+                        }
+                        if (failed) { rp.par ^= 1u << s; break; }  // nothing was issued into s
+                    }
+                    if (!mbar_test_wait(&empty[s], ph ^ 1u)) {
+                        const long long t0 = clock64();
+                        while (!mbar_test_wait(&empty[s], ph ^ 1u)) {
+                            if (sh->abort || clock64() - t0 > kWaitCycles) { failed = true; break; }
+                        }
+                        if (failed) { rp.par ^= 1u << s; break; }  // nothing was issued into s
+                    }
+                    mbar_expect_tx(&fullW[s], kWTileBytesP);
+                    tma_load_2d(ring + (size_t)s * kStageBytes + kXBytes, dw.tmW, kw * kTileK, tw * kTileNP, &fullW[s]);
+                    if (++kw == dw.kchunks) { kw = 0; ++tw; }
+                }
+            }
+            if (failed) {
+                set_status(p.status, kTimeoutCode);
+                sh->abort = 1;
+            }
+            // error path only: wait (bounded) for copies still in flight before the CTA may exit
+            if (sh->abort)
+                for (int s = 0; s < S; ++s)
+                    if ((rp.used >> s) & 1u) mbar_wait(&fullW[s], ((rp.par >> s) & 1u) ^ 1u);
+        }
+    } else {
+        // =============================== work warps ===============================
+        int epoch = 0;  // grid barriers passed
 
         if (p.trace && blockIdx.x == 0 && threadIdx.x == 0) {
             unsigned long long t;
@@ -1732,43 +1819,45 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             go = grid_sync(p, sh, epoch);
         }
         for (int l = 0; l < p.n_layers && go; ++l) {
-            run_gemm(4 * l + 0);                       // qkv
-            if (p.parallel) run_gemm(4 * l + 1);       // MLP in (same block input)
+            run_gemm<NT>(p, 4 * l + 0, smem);                       // qkv
+            if (p.parallel) run_gemm<NT>(p, 4 * l + 1, smem);       // MLP in (same block input)
             if (!(go = grid_sync(p, sh, epoch))) break;
             attention_phase(p, l, attn_scratch, sh);
             if (p.parallel) act_phase(p);
             if (!(go = grid_sync(p, sh, epoch))) break;
             if (p.parallel) {
-                run_gemm(4 * l + 2);                   // out-proj -> x
-                run_gemm(4 * l + 3);                   // MLP out  -> x
+                run_gemm<NT>(p, 4 * l + 2, smem);                   // out-proj -> x
+                run_gemm<NT>(p, 4 * l + 3, smem);                   // MLP out  -> x
                 if (!(go = grid_sync(p, sh, epoch))) break;
             } else {
-                run_gemm(4 * l + 1);                   // out-proj -> x
+                run_gemm<NT>(p, 4 * l + 1, smem);                   // out-proj -> x
                 if (!(go = grid_sync(p, sh, epoch))) break;
                 const LayerDesc *ld = layer_desc(p.md, l);
                 norm_phase(p, ld->ln2_g, ld->ln2_b, OP_XN1, nullptr, nullptr, 0, red);
                 grid_zero(p.t_in, p.R, p.d_in, p.d_in);
                 if (!(go = grid_sync(p, sh, epoch))) break;
-                run_gemm(4 * l + 2);                   // MLP in
+                run_gemm<NT>(p, 4 * l + 2, smem);                   // MLP in
                 if (!(go = grid_sync(p, sh, epoch))) break;
                 act_phase(p);
                 if (!(go = grid_sync(p, sh, epoch))) break;
-                run_gemm(4 * l + 3);                   // MLP out -> x
+                run_gemm<NT>(p, 4 * l + 3, smem);                   // MLP out -> x
                 if (!(go = grid_sync(p, sh, epoch))) break;
             }
             norm_for_layer(l + 1);
             if (!(go = grid_sync(p, sh, epoch))) break;
         }
-        if (go && p.want_logits) run_gemm(4 * p.n_layers);
+        if (go && p.want_logits) run_gemm<NT>(p, 4 * p.n_layers, smem);
         if (p.trace && blockIdx.x == 0 && threadIdx.x == 0) {
             unsigned long long t;
             asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
             p.trace[epoch + 1] = t;
             p.trace[epoch + 2] = 0;
         }
-        if (warp == kXWarp && lane == 0 && sh->abort)  // error path only: copies still in flight
+        if (warp == kXWarp && lane == 0 && sh->abort) {  // error path only: copies still in flight
+            const RingPos rp = role_rp[1];
             for (int s = 0; s < S; ++s)
                 if ((rp.used >> s) & 1u) mbar_wait(&fullX[s], ((rp.par >> s) & 1u) ^ 1u);
+        }
         if (warp == kMmaWarp) {  // nothing of this CTA may still be running on the tensor core
             if (lane == 0) {
                 tc_commit(mmaDone);
