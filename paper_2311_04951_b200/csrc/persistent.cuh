@@ -396,6 +396,22 @@ __device__ __forceinline__ double block_sum_work(double v, double *red) {
     return t;
 }
 
+// two sums in one exchange
+__device__ __forceinline__ void block_sum2_work(double &a, double &b, double *red) {
+    a = warp_sum(a);
+    b = warp_sum(b);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    named_bar(2, kWorkThreads);
+    if (lane == 0) { red[w] = a; red[kConsumerWarps + w] = b; }
+    named_bar(2, kWorkThreads);
+    double ta = 0.0, tb = 0.0;
+#pragma unroll
+    for (int i = 0; i < kConsumerWarps; ++i) { ta += red[i]; tb += red[kConsumerWarps + i]; }
+    a = ta;
+    b = tb;
+}
+__device__ __forceinline__ void prefetch_l1(const void *ptr) { asm volatile("prefetch.global.L1 [%0];" ::"l"(ptr)); }
+
 // zero a [R, n] fp32 buffer (row pitch ld), spread over the whole grid
 __device__ __forceinline__ void grid_zero(float *dst, int R, int n, int ld) {
     if (n == ld && ((R * (long long)n) & 3) == 0) {  // contiguous: 16-byte stores
@@ -430,6 +446,18 @@ __device__ __noinline__ void norm_phase(const FwdParams &p, const float *g1, con
             const int i = threadIdx.x + q * kWorkThreads;
             xv[q] = i < n4 ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
+        // the gain / bias vectors were last read a whole pass of weights ago: fetch them now, under the
+        // statistics, instead of as a second trip to DRAM after them
+#pragma unroll
+        for (int q = 0; q < kNormRegs; ++q) {
+            const int i = threadIdx.x + q * kWorkThreads;
+            if (i < n4) {
+                prefetch_l1(reinterpret_cast<const float4 *>(g1) + i);
+                if (b1) prefetch_l1(reinterpret_cast<const float4 *>(b1) + i);
+                if (g2) prefetch_l1(reinterpret_cast<const float4 *>(g2) + i);
+                if (b2) prefetch_l1(reinterpret_cast<const float4 *>(b2) + i);
+            }
+        }
         double s1 = 0.0, s2 = 0.0;
 #pragma unroll
         for (int q = 0; q < kNormRegs; ++q) {
@@ -441,8 +469,7 @@ __device__ __noinline__ void norm_phase(const FwdParams &p, const float *g1, con
             s1 += (double)v.x + (double)v.y + (double)v.z + (double)v.w;
             s2 += (double)v.x * v.x + (double)v.y * v.y + (double)v.z * v.z + (double)v.w * v.w;
         }
-        s1 = block_sum_work(s1, red);
-        s2 = block_sum_work(s2, red);
+        block_sum2_work(s1, s2, red);
         double mean = 0.0, var;
         if (p.norm_kind == 0) {
             mean = s1 / p.d;
