@@ -105,6 +105,7 @@ struct alignas(64) FwdParams {
     unsigned long long *trace;  // optional: CTA 0 stamps the global timer after every grid barrier
     // tensor-core attention (head dim 128): the whole cache as rows of Dh bf16, box 64 x 128 rows
     CUtensorMap tm_kv;
+    const CUtensorMap *tm_kv_ptr;  // where the copy engine can read tm_kv (set by the kernel: see params copy)
     int attn_tc;             // 1: attention_item_tc; 0: attention_item
     int kv_rows_per_layer;   // B * 2 * H * S
 };
@@ -232,7 +233,7 @@ constexpr int kAccStride = 256;
 constexpr int kEpiWarps = 4;    // warps 0-3: one tensor-memory lane quadrant each
 constexpr int kMmaWarp = 4;
 constexpr int kEpiPitch = kTileNP + 8;             // floats per row of the epilogue tile (bank spread)
-constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 12 * 8 + 12 * 4 + 16 + 2 * 16 + 8 * 4;  // 8 rows, the four warps' wait results, attention barriers
+constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 12 * 8 + 12 * 4 + 16 + 2 * 16 + 8 * 4 + 1024;  // ... + the parameter copy  // 8 rows, the four warps' wait results, attention barriers
 constexpr int kXWarp = 5;      // issues the operand copies of a GEMM phase
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -1185,8 +1186,8 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
         const int row = ((j & 1) ? vrow0 : krow0) + p_begin + c * kTcChunk;
         uint8_t *dst = ring + slot * kTcKvStage;
         mbar_expect_tx(&kv_full[slot], kTcKvStage);
-        tma_load_2d(dst, &p.tm_kv, 0, row, &kv_full[slot]);
-        tma_load_2d(dst + kTcKvStage / 2, &p.tm_kv, 64, row, &kv_full[slot]);
+        tma_load_2d(dst, p.tm_kv_ptr, 0, row, &kv_full[slot]);
+        tma_load_2d(dst + kTcKvStage / 2, p.tm_kv_ptr, 64, row, &kv_full[slot]);
     };
     const int n_early = min(3, 2 * n_chunks);
     if (warp == 5 && lane == 0 && !sh->abort) {
@@ -1518,6 +1519,7 @@ struct SmemMap {
     uint32_t *acnt;
     RingPos *role_rp;  // [2]: the MMA issuer's and the operand issuer's walk of the ring, between GEMMs
     int *role_seg;     // [8]: per work warp, tile segments so far
+    FwdParams *params; // the kernel parameters, copied once (see forward_kernel)
 };
 __device__ __forceinline__ SmemMap smem_map(const FwdParams &p, uint8_t *smem) {
     SmemMap m;
@@ -1537,6 +1539,7 @@ __device__ __forceinline__ SmemMap smem_map(const FwdParams &p, uint8_t *smem) {
     m.acnt = (uint32_t *)(m.abar + AB_COUNT);
     m.role_rp = (RingPos *)(m.acnt + AB_COUNT);
     m.role_seg = (int *)(m.role_rp + 2);
+    m.params = (FwdParams *)(((uintptr_t)(m.role_seg + 8) + 63) & ~(uintptr_t)63);
     return m;
 }
 
@@ -1705,9 +1708,19 @@ __device__ __noinline__ void run_gemm(const FwdParams &p, int gi, uint8_t *smem)
 // ---- the kernel -----------------------------------------------------------------------------
 // NT = padded rows / 8
 template <int NT>
-__global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __grid_constant__ FwdParams p) {
+__global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __grid_constant__ FwdParams kp) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // The phase functions are not inlined and read their parameters through a reference; a reference into the
+    // kernel-parameter bank makes every field a generic load at the head of each phase, so they get a copy in
+    // shared memory instead (tensor maps stay where the copy engine can read them: pointers into kp / global).
+    static_assert(sizeof(FwdParams) <= 960, "parameter copy area");
+    FwdParams *psm = smem_map(kp, smem).params;
+    for (int i = threadIdx.x; i < (int)(sizeof(FwdParams) / 4); i += blockDim.x)
+        reinterpret_cast<uint32_t *>(psm)[i] = reinterpret_cast<const uint32_t *>(&kp)[i];
+    __syncthreads();
+    if (threadIdx.x == 0) psm->tm_kv_ptr = &kp.tm_kv;
+    const FwdParams &p = *psm;  // (visible to everyone after the barrier below)
     constexpr int kRp = NT * 8;
     constexpr int kXBytes = 2 * kRp * kTileK * 2;  // operand tile (hi and lo rows), then the weight tile
     constexpr int kStageBytes = kXBytes + kWTileBytesP;
