@@ -44,6 +44,7 @@ constexpr int kConsumerWarps = 8;
 constexpr int kWorkThreads = kConsumerWarps * 32;  // 256: everyone but the producer
 constexpr int kPersistThreads = kWorkThreads + 32;
 constexpr int kAttnThreadsP = 256;
+constexpr int kMaxStagedLayers = 64;  // layers whose gain / bias pointers are staged in shared memory
 constexpr int kTileNP = 256;                        // weight rows per tile: the N of one MMA
 constexpr int kWTileBytesP = kTileNP * kTileK * 2;  // 32 KB
 
@@ -129,7 +130,7 @@ __device__ __forceinline__ int barriers_per_layer(const FwdParams &p) { return p
 // Barrier count before layer l: 2 (set-up; embedding + first norm) + barriers_per_layer * l.
 //   sequential layer: qkv | attention | o | norm2 | in | act | out | next norm   (8 barriers)
 //   parallel layer:   qkv, in | attention + act | o, out | next norms            (4 barriers)
-__device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi) {
+__device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi, const float *const *ltab = nullptr) {
     GemmDesc g;
     const int l = gi >> 2, e = gi & 3;
     const int base = 2 + barriers_per_layer(p) * l;
@@ -149,16 +150,16 @@ __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi) {
         g.need_hi = (kind == 0 || (kind == 2 && p.parallel)) ? (l == 0 ? 0 : base - barriers_per_layer(p) + 2) : base + 2;
         if (kind == 0) {
             g.xop = p.op[OP_XN1]; g.N = 3 * p.d; g.Kd = p.d; g.need = base;
-            g.out = p.qkv; g.ldo = 3 * p.d; g.bias = ld->b_qkv;
+            g.out = p.qkv; g.ldo = 3 * p.d; g.bias = ltab ? ltab[8 * l + 2] : ld->b_qkv;
         } else if (kind == 1) {
             g.xop = p.op[OP_AO]; g.N = p.d; g.Kd = p.d; g.need = base + 2;
-            g.out = p.x; g.ldo = p.d; g.bias = ld->b_o;
+            g.out = p.x; g.ldo = p.d; g.bias = ltab ? ltab[8 * l + 3] : ld->b_o;
         } else if (kind == 2) {
             g.xop = p.op[p.parallel ? OP_XN2 : OP_XN1]; g.N = p.d_in; g.Kd = p.d; g.need = p.parallel ? base : base + 4;
-            g.out = p.t_in; g.ldo = p.d_in; g.bias = ld->b_in;
+            g.out = p.t_in; g.ldo = p.d_in; g.bias = ltab ? ltab[8 * l + 6] : ld->b_in;
         } else {
             g.xop = p.op[OP_ACT]; g.N = p.d; g.Kd = p.F; g.need = p.parallel ? base + 2 : base + 6;
-            g.out = p.x; g.ldo = p.d; g.bias = ld->b_out;
+            g.out = p.x; g.ldo = p.d; g.bias = ltab ? ltab[8 * l + 7] : ld->b_out;
         }
     }
     g.n_tiles = (g.N + kTileNP - 1) / kTileNP;
@@ -233,7 +234,7 @@ constexpr int kAccStride = 256;
 constexpr int kEpiWarps = 4;    // warps 0-3: one tensor-memory lane quadrant each
 constexpr int kMmaWarp = 4;
 constexpr int kEpiPitch = kTileNP + 8;             // floats per row of the epilogue tile (bank spread)
-constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 12 * 8 + 12 * 4 + 16 + 2 * 16 + 8 * 4 + 1024;  // ... + the parameter copy  // 8 rows, the four warps' wait results, attention barriers
+constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 12 * 8 + 12 * 4 + 16 + 2 * 16 + 8 * 4 + 1024 + 512 + (8 * kMaxStagedLayers + 2) * 8;  // ... + parameter copy, staged tables  // 8 rows, the four warps' wait results, attention barriers
 constexpr int kXWarp = 5;      // issues the operand copies of a GEMM phase
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -313,8 +314,17 @@ struct alignas(16) Shared {
     // for the tensor-core attention items (kept here so that they take no more arguments than the others):
     uint32_t tmem_base;     // base address of this CTA's tensor memory
     uint32_t attn_bar_off;  // byte offset from this block to the attention barriers, followed by their counts
-    uint32_t pad[2];
+    // small tables staged in shared memory (byte offsets from this block), so that the head of a phase does
+    // not start with a trip to global memory:
+    uint32_t seq_off;       // int len[64], then int rows[64]: committed length and rows of this pass, per sequence
+    uint32_t ltab_off;      // const float *[8 n_layers + 2]: the layers' gain / bias pointers, then the final norm's; 0 = not staged
 };
+__device__ __forceinline__ const int *staged_len(const Shared *sh) {
+    return reinterpret_cast<const int *>(reinterpret_cast<const uint8_t *>(sh) + sh->seq_off);
+}
+__device__ __forceinline__ const float *const *staged_ltab(const Shared *sh) {
+    return sh->ltab_off ? reinterpret_cast<const float *const *>(reinterpret_cast<const uint8_t *>(sh) + sh->ltab_off) : nullptr;
+}
 
 // Bounded wait that also gives up as soon as another thread of the CTA has.
 __device__ __forceinline__ bool mbar_wait_or_abort(uint64_t *bar, uint32_t parity, const Shared *sh) {
@@ -733,8 +743,8 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
     const int pg = warp & 3, dhh = warp >> 2;
     const int nk = Dh >> 4;          // k-steps of Q K^T; also 8-column output tiles per head half
     const int dh0 = dhh * (Dh >> 1);
-    const int n_rows = __ldcg(p.ri.n_eff + b);
-    const int len = p.len[b];
+    const int n_rows = staged_len(sh)[64 + b];
+    const int len = staged_len(sh)[b];
     const int r0 = b * p.M, m_base = mt * kAttnRows;
     const int p_begin = split * p.chunk;
     const int p_end = min(p_begin + p.chunk, len + n_rows);
@@ -1147,8 +1157,8 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
     uint64_t *s_full = abar + AB_S_FULL;  // [2]: the scores are double-buffered in tensor memory
     uint64_t *p_ready = abar + AB_P_READY, *o_done = abar + AB_O_DONE, *fixed = abar + AB_FIXED, *landed = abar + AB_LANDED;
 
-    const int n_rows = __ldcg(p.ri.n_eff + b);
-    const int len = p.len[b];
+    const int n_rows = staged_len(sh)[64 + b];
+    const int len = staged_len(sh)[b];
     const int r0 = b * p.M, m_base = mt * kAttnRows;
     const int rows_here = max(0, min(kAttnRows, p.M - m_base));
     const int p_begin = split * p.chunk;
@@ -1520,6 +1530,8 @@ struct SmemMap {
     RingPos *role_rp;  // [2]: the MMA issuer's and the operand issuer's walk of the ring, between GEMMs
     int *role_seg;     // [8]: per work warp, tile segments so far
     FwdParams *params; // the kernel parameters, copied once (see forward_kernel)
+    int *seq;          // [128]: lengths, rows of this pass
+    const float **ltab;  // [8 * kMaxStagedLayers + 2]
 };
 __device__ __forceinline__ SmemMap smem_map(const FwdParams &p, uint8_t *smem) {
     SmemMap m;
@@ -1540,6 +1552,8 @@ __device__ __forceinline__ SmemMap smem_map(const FwdParams &p, uint8_t *smem) {
     m.role_rp = (RingPos *)(m.acnt + AB_COUNT);
     m.role_seg = (int *)(m.role_rp + 2);
     m.params = (FwdParams *)(((uintptr_t)(m.role_seg + 8) + 63) & ~(uintptr_t)63);
+    m.seq = (int *)((uint8_t *)m.params + 960);
+    m.ltab = (const float **)(m.seq + 128);
     return m;
 }
 
@@ -1577,7 +1591,7 @@ __device__ __noinline__ void run_gemm(const FwdParams &p, int gi, uint8_t *smem)
         __syncwarp();
     };
 
-            const GemmDesc g = gemm_desc(p, gi);
+            const GemmDesc g = gemm_desc(p, gi, staged_ltab(sh));
             int c0, c1;
             unit_range(p, g, c0, c1);
             if (c0 >= c1) return;  // (no state to save: nothing moved)
@@ -1738,6 +1752,14 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
     uint32_t *acnt = (uint32_t *)(abar + AB_COUNT);
     RingPos *role_rp = (RingPos *)(acnt + AB_COUNT);  // the same places smem_map() gives
     int *role_seg = (int *)(role_rp + 2);
+    int *seq_tab = smem_map(kp, smem).seq;
+    const float **ltab = smem_map(kp, smem).ltab;
+    if (kp.n_layers <= kMaxStagedLayers) {  // the layers' gain / bias pointers and the final norm's
+        for (int i = threadIdx.x; i < 8 * kp.n_layers + 2; i += blockDim.x) {
+            const int l = i >> 3, k = i & 7;
+            ltab[i] = l < kp.n_layers ? (&layer_desc(kp.md, l)->ln1_g)[k] : (k == 0 ? kp.md->lnf_g : kp.md->lnf_b);
+        }
+    }
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp == 0) {  // tensor memory for the accumulators; released by the same warp at the end
@@ -1768,6 +1790,8 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
         sh->abort = 0;
         sh->go = 1;
         sh->attn_bar_off = (uint32_t)((uint8_t *)abar - (uint8_t *)sh);
+        sh->seq_off = (uint32_t)((uint8_t *)seq_tab - (uint8_t *)sh);
+        sh->ltab_off = kp.n_layers <= kMaxStagedLayers ? (uint32_t)((uint8_t *)ltab - (uint8_t *)sh) : 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     tc_fence_before();
@@ -1840,19 +1864,29 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
         // below is reached by all of them or by none.
         auto norm_for_layer = [&](int l) {  // operand(s) of layer l's first GEMM(s), or of the LM head
             if (l < p.n_layers) {
+                const float *const *lt = staged_ltab(sh);
                 const LayerDesc *ld = layer_desc(p.md, l);
-                if (p.parallel) norm_phase(p, ld->ln1_g, ld->ln1_b, OP_XN1, ld->ln2_g, ld->ln2_b, OP_XN2, red);
-                else norm_phase(p, ld->ln1_g, ld->ln1_b, OP_XN1, nullptr, nullptr, 0, red);
+                const float *g1 = lt ? lt[8 * l + 0] : ld->ln1_g, *b1 = lt ? lt[8 * l + 1] : ld->ln1_b;
+                if (p.parallel)
+                    norm_phase(p, g1, b1, OP_XN1, lt ? lt[8 * l + 4] : ld->ln2_g, lt ? lt[8 * l + 5] : ld->ln2_b, OP_XN2, red);
+                else norm_phase(p, g1, b1, OP_XN1, nullptr, nullptr, 0, red);
                 grid_zero(p.qkv, p.R, 3 * p.d, 3 * p.d);
                 if (p.parallel) grid_zero(p.t_in, p.R, p.d_in, p.d_in);
             } else if (p.want_logits) {
-                norm_phase(p, p.md->lnf_g, p.md->lnf_b, OP_XN1, nullptr, nullptr, 0, red);
+                const float *const *lt = staged_ltab(sh);
+                norm_phase(p, lt ? lt[8 * p.n_layers] : p.md->lnf_g, lt ? lt[8 * p.n_layers + 1] : p.md->lnf_b, OP_XN1, nullptr,
+                           nullptr, 0, red);
                 grid_zero(p.logits, p.R, p.V, p.V);
             }
         };
         setup_phase(p);
         bool go = grid_sync(p, sh, epoch);
         if (go) {
+            if (threadIdx.x < 64) {  // lengths and rows of this pass (written by the set-up phase), for the attention items
+                const int b = threadIdx.x;
+                seq_tab[b] = b < p.B ? p.len[b] : 0;
+                seq_tab[64 + b] = b < p.B ? __ldcg(p.ri.n_eff + b) : 0;
+            }
             embed_phase(p);
             named_bar(2, kWorkThreads);  // the embedding rows are read back by the CTA that wrote them
             norm_for_layer(0);
@@ -1872,8 +1906,9 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             } else {
                 run_gemm<NT>(p, 4 * l + 1, smem);                   // out-proj -> x
                 if (!(go = grid_sync(p, sh, epoch))) break;
+                const float *const *lt = staged_ltab(sh);
                 const LayerDesc *ld = layer_desc(p.md, l);
-                norm_phase(p, ld->ln2_g, ld->ln2_b, OP_XN1, nullptr, nullptr, 0, red);
+                norm_phase(p, lt ? lt[8 * l + 4] : ld->ln2_g, lt ? lt[8 * l + 5] : ld->ln2_b, OP_XN1, nullptr, nullptr, 0, red);
                 grid_zero(p.t_in, p.R, p.d_in, p.d_in);
                 if (!(go = grid_sync(p, sh, epoch))) break;
                 run_gemm<NT>(p, 4 * l + 2, smem);                   // MLP in
