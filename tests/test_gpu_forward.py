@@ -160,3 +160,27 @@ def test_single_kernel_forward_equals_stepwise_forward(name):
     for b, n in enumerate((20 + K + 1, 13 + K + 1)):
         a, c = res[0][1][:, b, :, :, :n], res[1][1][:, b, :, :, :n]
         assert (np.abs(a - c) <= gu.LOGIT_RTOL * np.abs(c) + gu.LOGIT_ATOL).all()
+
+
+@pytest.mark.parametrize("Bn,M", [(1, 9), (1, 17), (3, 11), (8, 5), (2, 32), (8, 8)])
+def test_row_counts_of_the_single_kernel_gemms(Bn, M):
+    """The forward kernel is instantiated per padded row count (8, 16, 24, 32, 40, 64 rows: operand tiles of
+    1-8 blocks, MMA M = 64 up to 32 rows and 128 beyond, ring stages of 34-48 KB).  One verification pass of
+    Bn x M rows per variant, logits against the oracle."""
+    arch = ARCHS["neox_bf16"]
+    ws_np = gu.scaled_weights(synth, arch, 21, 6.0)
+    omodel = od.Model(arch, ws_np)
+    model = B.Model(arch, B.upload_weights(arch, ws_np))
+    S, P = 64, 7
+    prompts = synth.gen_prompt(22, Bn, P, arch.vocab)
+    kv = B.KV(model, Bn, S)
+    ws = model.new_workspace(Bn, max(M, 8), S)
+    dev = "cuda"
+    B.kv_prefill(model, kv, torch.from_numpy(prompts).to(dev), torch.full((Bn,), P, dtype=torch.int32, device=dev), ws)
+    rows = synth.gen_prompt(23, Bn, M, arch.vocab)
+    got = gpu_logits(model, kv, ws, rows, M - 1)
+    assert kv.status() == 0
+    for b in range(Bn):
+        oc = omodel.new_cache(S)
+        oc.feed(prompts[b], want_logits=False)
+        gu.assert_logits_close(got[b], oc.feed(rows[b], advance=False))
