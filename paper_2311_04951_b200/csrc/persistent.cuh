@@ -234,7 +234,7 @@ constexpr int kAccStride = 256;
 constexpr int kEpiWarps = 4;    // warps 0-3: one tensor-memory lane quadrant each
 constexpr int kMmaWarp = 4;
 constexpr int kEpiPitch = kTileNP + 8;             // floats per row of the epilogue tile (bank spread)
-constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 12 * 8 + 12 * 4 + 16 + 2 * 16 + 8 * 4 + 1024 + 512 + (8 * kMaxStagedLayers + 2) * 8;  // ... + parameter copy, staged tables  // 8 rows, the four warps' wait results, attention barriers
+constexpr int kEpiBytes = 8 * kEpiPitch * 4 + 16 + 16 * 8 + 16 * 4 + 16 + 2 * 16 + 8 * 4 + 1024 + 512 + (8 * kMaxStagedLayers + 2) * 8;  // ... + parameter copy, staged tables  // 8 rows, the four warps' wait results, attention barriers
 constexpr int kXWarp = 5;      // issues the operand copies of a GEMM phase
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -1052,15 +1052,16 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
 //   O^T [128 head dims x 32] += V chunk read as its transpose (MN-major M = 128 operand) x P (16 hi + 16 lo)
 // Roles: threads 0-127 = one position each (softmax: masks, running max shared through shared memory,
 // P as bf16 hi + lo into the P tile, rescale of O^T when a maximum moved) and, at the end, one head
-// dim each (output); warp 4: MMA issue; warp 5: TMA copies of K and V chunks into a 3-stage ring;
+// dim each (output); warp 4: MMA issue; warp 5: TMA copies of K and V chunks into a 4-stage ring;
 // warps 6-7: rows of this pass (positions >= len) - rotary, rounding, append to the cache - written
 // into the chunk tiles over what the copy brought.  Positions behind them are masked (P = 0) and
 // multiply whatever the cache holds there: kv_init zeroes the cache, and all later writes are
 // finite rows of earlier passes, so 0 x stale is 0.  Per chunk 8 + 8 MMA steps of ~120 cycles against 1.5 us of HBM time for its
 // 64 KB: the chunk loop is bandwidth-bound instead of a latency chain.
 constexpr int kTcChunk = 128;
+constexpr int kTcStages = 4;  // K / V ring stages of 32 KB: the bytes in flight set the chunk rate (3 stages: 2.7 us per chunk)
 constexpr int kTcKvStage = kTcChunk * 128 * 2;  // one K or V chunk: two 64-column panels of 128 rows x 128 B
-constexpr int kTcQOff = 3 * kTcKvStage, kTcPOff = kTcQOff + 8192, kTcMiscOff = kTcPOff + 8192;
+constexpr int kTcQOff = kTcStages * kTcKvStage, kTcPOff = kTcQOff + 8192, kTcMiscOff = kTcPOff + 8192;
 constexpr int kTcScratchBytes = kTcMiscOff + 1536 + kAttnRows * 128 * 4;  // + per-thread running sums [16][128]
 // Its mbarriers live outside the scratch (which the weight ring reuses), are initialised once per kernel
 // and keep running: cnt[i] = phases barrier i has completed before the current item.  A parity wait is
@@ -1068,7 +1069,7 @@ constexpr int kTcScratchBytes = kTcMiscOff + 1536 + kAttnRows * 128 * 4;  // + p
 // cannot pass by two phases; the threads that patch this pass's rows into a chunk skip most chunks, so
 // they do not wait on the ring's barriers: the MMA issuer, which follows every stage, tells them through
 // `landed` when such a chunk has arrived, and hears back through `fixed`.
-enum { AB_KV_FULL = 0, AB_KV_FREE = 3, AB_S_FULL = 6, AB_P_READY = 8, AB_O_DONE = 9, AB_FIXED = 10, AB_LANDED = 11, AB_COUNT = 12 };
+enum { AB_KV_FULL = 0, AB_KV_FREE = kTcStages, AB_S_FULL = 2 * kTcStages, AB_P_READY = AB_S_FULL + 2, AB_O_DONE, AB_FIXED, AB_LANDED, AB_COUNT };
 
 __device__ __forceinline__ void tc_ld_32(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
@@ -1153,7 +1154,7 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
     float *wmrun = wsum + 64;                                       // [4][16] running maxima, one copy per warp
     float *fsh = wmrun + 64;                                        // [4][16] this chunk's rescale factors
     float *l_sh = fsh + 64;                                         // [16][128] running sums, one per (row, thread)
-    uint64_t *kv_full = abar + AB_KV_FULL, *kv_free = abar + AB_KV_FREE;  // [3] each
+    uint64_t *kv_full = abar + AB_KV_FULL, *kv_free = abar + AB_KV_FREE;  // [kTcStages] each
     uint64_t *s_full = abar + AB_S_FULL;  // [2]: the scores are double-buffered in tensor memory
     uint64_t *p_ready = abar + AB_P_READY, *o_done = abar + AB_O_DONE, *fixed = abar + AB_FIXED, *landed = abar + AB_LANDED;
 
@@ -1180,26 +1181,26 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
     };
 
     // phases completed before this item (written by thread 0 at the end of the previous item, behind a barrier)
-    uint32_t c_full[3], c_free[3];
+    uint32_t c_full[kTcStages], c_free[kTcStages];
 #pragma unroll
-    for (int i = 0; i < 3; ++i) { c_full[i] = acnt[AB_KV_FULL + i]; c_free[i] = acnt[AB_KV_FREE + i]; }
+    for (int i = 0; i < kTcStages; ++i) { c_full[i] = acnt[AB_KV_FULL + i]; c_free[i] = acnt[AB_KV_FREE + i]; }
     const uint32_t c_s0 = acnt[AB_S_FULL], c_s1 = acnt[AB_S_FULL + 1];
     const uint32_t c_p = acnt[AB_P_READY], c_o = acnt[AB_O_DONE], c_fix = acnt[AB_FIXED], c_land = acnt[AB_LANDED];
-    auto full_par = [&](int j) { return (c_full[j % 3] + (uint32_t)(j / 3)) & 1u; };          // stage j has landed
-    auto free_par = [&](int j) { return ((c_free[j % 3] + (uint32_t)(j / 3)) & 1u) ^ 1u; };   // its slot was released
+    auto full_par = [&](int j) { return (c_full[j % kTcStages] + (uint32_t)(j / kTcStages)) & 1u; };          // stage j has landed
+    auto free_par = [&](int j) { return ((c_free[j % kTcStages] + (uint32_t)(j / kTcStages)) & 1u) ^ 1u; };   // its slot was released
     int n_fix_total = 0;
     for (int c = 0; c < n_chunks; ++c) n_fix_total += (p_begin + (c + 1) * kTcChunk > len) ? 1 : 0;
 
     // The copies of the first chunks do not depend on the set-up below: start them now.
     auto issue_kv = [&](int j) {
-        const int slot = j % 3, c = j >> 1;
+        const int slot = j % kTcStages, c = j >> 1;
         const int row = ((j & 1) ? vrow0 : krow0) + p_begin + c * kTcChunk;
         uint8_t *dst = ring + slot * kTcKvStage;
         mbar_expect_tx(&kv_full[slot], kTcKvStage);
         tma_load_2d(dst, p.tm_kv_ptr, 0, row, &kv_full[slot]);
         tma_load_2d(dst + kTcKvStage / 2, p.tm_kv_ptr, 64, row, &kv_full[slot]);
     };
-    const int n_early = min(3, 2 * n_chunks);
+    const int n_early = min(kTcStages, 2 * n_chunks);
     if (warp == 5 && lane == 0 && !sh->abort) {
         fence_async_proxy();  // the previous user of these slots wrote them through the generic proxy
         for (int j = 0; j < n_early; ++j) issue_kv(j);
@@ -1227,17 +1228,17 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
     named_bar(3, kAttnThreadsP);
 
     if (warp == 5) {
-        // ---------------- K / V chunk copies: stage j = 2 c (K), 2 c + 1 (V), slot j % 3 ----------------
+        // ---------------- K / V chunk copies: stage j = 2 c (K), 2 c + 1 (V), slot j % kTcStages ----------------
         if (lane == 0) {
             int issued = n_early;
             for (int j = n_early; j < 2 * n_chunks && !sh->abort; ++j) {
-                wait(&kv_free[j % 3], free_par(j));
+                wait(&kv_free[j % kTcStages], free_par(j));
                 if (sh->abort) break;
                 issue_kv(j);
                 ++issued;
             }
             if (sh->abort)  // error path only: copies still in flight
-                for (int j = max(0, issued - 3); j < issued; ++j) mbar_wait(&kv_full[j % 3], full_par(j));
+                for (int j = max(0, issued - kTcStages); j < issued; ++j) mbar_wait(&kv_full[j % kTcStages], full_par(j));
         }
         __syncwarp();
     } else if (warp == 4) {
@@ -1251,38 +1252,38 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
             auto issue_s = [&](int c) {
                 const int jk = 2 * c, jv = 2 * c + 1;
                 const bool fix = p_begin + (c + 1) * kTcChunk > len;
-                wait(&kv_full[jk % 3], full_par(jk));
+                wait(&kv_full[jk % kTcStages], full_par(jk));
                 if (fix) {  // both tiles are here: let the patching threads in, wait for them
-                    wait(&kv_full[jv % 3], full_par(jv));
+                    wait(&kv_full[jv % kTcStages], full_par(jv));
                     if (!sh->abort) mbar_arrive(landed);
                     wait(fixed, (c_fix + n_fix) & 1u);
                     ++n_fix;
                 }
                 if (sh->abort) return;
                 tc_fence_after();
-                const uint32_t ka = smem_u32(ring + (jk % 3) * kTcKvStage);
+                const uint32_t ka = smem_u32(ring + (jk % kTcStages) * kTcKvStage);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)  // k = 16 head dims per step; panel ks / 4
                     tc_mma_bf16(tS + 32 * (c & 1), umma_desc(ka + (ks >> 2) * (kTcKvStage / 2) + (ks & 3) * 32, 16, 1024),
                                 umma_desc(qa + (ks >> 2) * 4096 + (ks & 3) * 32, 16, 1024), idS, ks ? 1u : 0u);
                 tc_commit(&s_full[c & 1]);
-                tc_commit(&kv_free[jk % 3]);
+                tc_commit(&kv_free[jk % kTcStages]);
             };
             if (n_chunks > 0) issue_s(0);
             for (int c = 0; c < n_chunks && !sh->abort; ++c) {
                 const int jv = 2 * c + 1;
                 if (c + 1 < n_chunks) issue_s(c + 1);
                 wait(p_ready, (c_p + c) & 1u);
-                wait(&kv_full[jv % 3], full_par(jv));
+                wait(&kv_full[jv % kTcStages], full_par(jv));
                 if (sh->abort) break;
                 tc_fence_after();
-                const uint32_t va = smem_u32(ring + (jv % 3) * kTcKvStage);
+                const uint32_t va = smem_u32(ring + (jv % kTcStages) * kTcKvStage);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)  // k = 16 positions per step: two 8-row groups of the V tile
                     tc_mma_bf16(tO, umma_desc(va + ks * 2048, kTcKvStage / 2, 1024),
                                 umma_desc(pa + (ks >> 2) * 4096 + (ks & 3) * 32, 16, 1024), idO, (c | ks) ? 1u : 0u);
                 tc_commit(o_done);
-                tc_commit(&kv_free[jv % 3]);
+                tc_commit(&kv_free[jv % kTcStages]);
             }
         }
         __syncwarp();
@@ -1294,7 +1295,7 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
             const int base = p_begin + c * kTcChunk;
             if (base + kTcChunk <= len) continue;
             const int jk = 2 * c, jv = 2 * c + 1;
-            uint8_t *kt = ring + (jk % 3) * kTcKvStage, *vt = ring + (jv % 3) * kTcKvStage;
+            uint8_t *kt = ring + (jk % kTcStages) * kTcKvStage, *vt = ring + (jv % kTcStages) * kTcKvStage;
             const int first = max(0, len - base), last = min(kTcChunk, len + n_rows - base);  // tile rows [first, last)
             // at most 32 rows x 16 vectors = 8 work items per thread: compute them all, then wait for the copies
             uint4 kq[8], vq[8];
@@ -1493,8 +1494,8 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
         }
     }
     if (tid == 0) {
-        for (int i = 0; i < 3; ++i) {
-            const uint32_t uses = (uint32_t)((2 * n_chunks + 2 - i) / 3);  // stages j < 2 n_chunks with j % 3 == i
+        for (int i = 0; i < kTcStages; ++i) {
+            const uint32_t uses = (uint32_t)((2 * n_chunks + kTcStages - 1 - i) / kTcStages);  // stages j < 2 n_chunks with j % kTcStages == i
             acnt[AB_KV_FULL + i] = c_full[i] + uses;
             acnt[AB_KV_FREE + i] = c_free[i] + uses;
         }
