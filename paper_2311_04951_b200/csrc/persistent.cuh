@@ -26,10 +26,18 @@
 //               holds k-chunk 0) to the output with 16-byte vector reductions: a reduction
 //               costs its warp a memory latency, so there must be few of them per thread
 //   warps 0-7   between GEMM phases: the small phases (row set-up, embedding, norm, activation,
-//               attention with rotary + KV append + split merge), which leave every GEMM
-//               operand in global memory already split into bf16 hi + lo, and the grid barriers
+//               attention with rotary + KV append + split merge - on warp-level MMAs, or for head
+//               dim 128 and long splits on tcgen05 with its own roles, see attention_item_tc),
+//               which leave every GEMM operand in global memory already split into bf16 hi + lo,
+//               and the grid barriers
+// Every phase is a function of its own (not inlined) that reads a shared-memory copy of the kernel
+// parameters and keeps what must survive between calls in shared memory: the phase loop holds nothing
+// across calls, because a spilled value or a read through the parameter bank would be a trip to L2 at
+// the head of every one of the pass's ~130-260 phases (227 KB of shared memory leave next to no L1).
 // Every wait (mbarrier, grid barrier) is bounded; on time-out SSD_E_TIMEOUT is recorded, the CTA
-// stops taking work, waits (bounded) for its copies in flight and returns.
+// stops taking work, waits (bounded) for its copies in flight, drains the tensor core, frees its
+// tensor memory and returns.  A parity wait is used only where the waiter follows every phase of its
+// barrier in order and the barrier cannot pass it by two phases.
 #pragma once
 #include <cuda.h>
 
