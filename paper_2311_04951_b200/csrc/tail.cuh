@@ -57,16 +57,33 @@ __device__ __forceinline__ RowStat row_stats(const float *logits, int V, float i
                                              double *sd) {
     float mx = -INFINITY;
     int am = 0x7fffffff;
-    for (int j = threadIdx.x; j < V; j += blockDim.x) {
-        float l = logits[j];
-        if (l > mx) { mx = l; am = j; }  // strided ascending: first maximum per thread
+    // eight loads in flight per thread: the row comes from L2, and one latency per element is the whole cost
+    for (int j0 = threadIdx.x; j0 < V; j0 += 8 * blockDim.x) {
+        float l[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int j = j0 + u * blockDim.x;
+            l[u] = j < V ? __ldcg(logits + j) : -INFINITY;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (l[u] > mx) { mx = l[u]; am = j0 + u * blockDim.x; }  // strided ascending: first maximum per thread
     }
     RowStat st;
     block_argmax(mx, am, sv, si, st.mx, st.amax);
     double z = 0.0;
     if (inv_t != 0.f) {
         float part = 0.f;
-        for (int j = threadIdx.x; j < V; j += blockDim.x) part += expf((logits[j] - st.mx) * inv_t);
+        for (int j0 = threadIdx.x; j0 < V; j0 += 8 * blockDim.x) {
+            float l[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int j = j0 + u * blockDim.x;
+                l[u] = j < V ? __ldcg(logits + j) : -INFINITY;  // exp(-inf) = 0
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) part += expf((l[u] - st.mx) * inv_t);
+        }
         z = block_sum((double)part, sd);
     }
     st.z = (float)z;
