@@ -833,7 +833,7 @@ int draft_step(ssd_model *draft, ssd_kv *dkv, const int32_t *dev_tokens_in, int 
     t.u = dev_u; t.u_stride = u_stride;
     t.token_out = dev_token_out; t.token_stride = token_out_stride;
     t.q_out = dev_q_out; t.q_stride = q_stride;
-    LAUNCH(draft_tail_kernel, dkv->B, kTailThreads, 0, st, t);
+    LAUNCH(draft_tail_kernel, dkv->B * kTailCluster, kTailThreads, 0, st, t);
     LAUNCH(kv_commit_rows_kernel, ceil_div(dkv->B, 64), 64, 0, st, dkv->len, w.ri.n_eff, dkv->B);
     dkv->len_ub += rows_in;
     if (dkv->len_ub > dkv->S) dkv->len_ub = dkv->S;
@@ -853,8 +853,8 @@ static int run_verify_tail(const float *logits, int B, int K, int V, const int32
     v.inv_t = temperature > 0.f ? 1.0f / temperature : 0.f;
     v.n_accepted = n_acc; v.next_token = next; v.next_stride = next_stride;
     v.p_debug = p_debug; v.keep = keep; v.stats = stats;
-    LAUNCH(row_stats_kernel, dim3(K + 1, B), kTailThreads, 0, st, v);
-    LAUNCH(verify_kernel, B, kTailThreads, 0, st, v);
+    LAUNCH(row_stats_kernel, dim3((K + 1) * kTailCluster, B), kTailThreads, 0, st, v);
+    LAUNCH(verify_kernel, B * kTailCluster, kTailThreads, 0, st, v);
     return SSD_OK;
 }
 

@@ -3,12 +3,38 @@
 // (Section "Speculative Sampling", Figure 2: the target "qualifies and accepts (or rejects)" the
 // draft tokens and generates one token itself.)  No host round-trip: everything a decision
 // needs stays on the device; reductions use warp shuffles, prefix sums run in fp64.
+//
+// One row of the vocabulary is worked on by a thread-block cluster of kTailCluster CTAs (one SM alone
+// is issue- and latency-bound on a 50 K-entry row: ncu shows 52 % issue slots busy on the statistics
+// and long-scoreboard stalls of 18 per issue on the draw).  CTA `rank` owns a contiguous slice of the
+// row; block results are published in shared memory and read by the other CTAs of the cluster through
+// distributed shared memory, always combined in rank order so that sums keep the index order.
 #pragma once
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace ssd {
 
+namespace cg = cooperative_groups;
+
 constexpr int kTailThreads = 1024;
+constexpr int kTailCluster = 8;
+
+// What a CTA publishes to its cluster.  Every exchange uses slots of its own, so one cluster barrier
+// per exchange suffices; a kernel ends with a cluster barrier (nobody leaves while its slots are read).
+struct ClusterSlots {
+    float v[2];
+    int i[6];
+    double d[4];
+};
+
+// CTA `rank`'s slice [lo, hi) of a row of V entries: whole rows of 32 indices, split evenly.
+__device__ __forceinline__ void tail_slice(int V, int rank, int &lo, int &hi) {
+    const int rows = (V + 31) >> 5, per = (rows + kTailCluster - 1) / kTailCluster;
+    lo = min(V, rank * per * 32);
+    hi = min(V, lo + per * 32);
+}
 
 struct RowStat {
     float mx;      // max logit of the row
@@ -52,53 +78,78 @@ __device__ __forceinline__ void block_argmax(float v, int idx, float *sv, int *s
     out_i = si[0];
 }
 
-// Row statistics of logits[row, :]; every thread returns the same RowStat.
-__device__ __forceinline__ RowStat row_stats(const float *logits, int V, float inv_t, float *sv, int *si,
-                                             double *sd) {
+// Row statistics of logits[row, :] by the whole cluster; every thread of every CTA returns the same RowStat.
+__device__ __forceinline__ RowStat row_stats(const float *logits, int V, float inv_t, float *sv, int *si, double *sd,
+                                             ClusterSlots *pub, cg::cluster_group &cl) {
+    const int rank = (int)cl.block_rank();
+    int lo, hi;
+    tail_slice(V, rank, lo, hi);
     float mx = -INFINITY;
     int am = 0x7fffffff;
     // eight loads in flight per thread: the row comes from L2, and one latency per element is the whole cost
-    for (int j0 = threadIdx.x; j0 < V; j0 += 8 * blockDim.x) {
+    for (int j0 = lo + threadIdx.x; j0 < hi; j0 += 8 * blockDim.x) {
         float l[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int j = j0 + u * blockDim.x;
-            l[u] = j < V ? __ldcg(logits + j) : -INFINITY;
+            l[u] = j < hi ? __ldcg(logits + j) : -INFINITY;
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u)
             if (l[u] > mx) { mx = l[u]; am = j0 + u * blockDim.x; }  // strided ascending: first maximum per thread
     }
+    float bmx;
+    int bam;
+    block_argmax(mx, am, sv, si, bmx, bam);
+    if (threadIdx.x == 0) { pub->v[0] = bmx; pub->i[0] = bam; }
+    cl.sync();
     RowStat st;
-    block_argmax(mx, am, sv, si, st.mx, st.amax);
+    st.mx = -INFINITY;
+    st.amax = 0x7fffffff;
+    for (int r = 0; r < kTailCluster; ++r) {  // lowest index among the maxima
+        const ClusterSlots *o = cl.map_shared_rank(pub, r);
+        const float v = o->v[0];
+        const int i = o->i[0];
+        if (v > st.mx || (v == st.mx && i < st.amax)) { st.mx = v; st.amax = i; }
+    }
     double z = 0.0;
     if (inv_t != 0.f) {
         float part = 0.f;
-        for (int j0 = threadIdx.x; j0 < V; j0 += 8 * blockDim.x) {
+        for (int j0 = lo + threadIdx.x; j0 < hi; j0 += 8 * blockDim.x) {
             float l[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const int j = j0 + u * blockDim.x;
-                l[u] = j < V ? __ldcg(logits + j) : -INFINITY;  // exp(-inf) = 0
+                l[u] = j < hi ? __ldcg(logits + j) : -INFINITY;  // exp(-inf) = 0
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) part += expf((l[u] - st.mx) * inv_t);
         }
-        z = block_sum((double)part, sd);
+        const double zb = block_sum((double)part, sd);
+        if (threadIdx.x == 0) pub->d[0] = zb;
+        cl.sync();
+        for (int r = 0; r < kTailCluster; ++r) z += cl.map_shared_rank(pub, r)->d[0];
     }
     st.z = (float)z;
     st.pad = 0;
     return st;
 }
 
-// Inverse-CDF draw over V weights w(j) >= 0: the smallest j whose inclusive prefix sum exceeds
-// u * S; prefix sums in index order, fp64.  If rounding leaves none: the largest j with w > 0.
-// Each thread owns a contiguous segment so the prefix order is the index order.  Returns S via
-// *total (all threads); the drawn index is valid in all threads.  S <= 0 returns -1.
+// Inverse-CDF draw over V weights w(j) >= 0 by the whole cluster: the smallest j whose inclusive prefix
+// sum exceeds u * S; prefix sums in index order, fp64.  If rounding leaves none: the largest j with
+// w > 0.  Each CTA owns a slice, each thread a contiguous segment of it, so the prefix order is the
+// index order: thread sums are scanned inside the CTA, CTA totals in rank order across the cluster.
+// `slot` (0 or 1) selects the exchange slots, so that two draws in one kernel need no extra barrier.
+// Returns S via *total; S and the drawn index are the same in every thread of the cluster.  S <= 0
+// returns -1.
 template <typename WeightFn>
-__device__ __forceinline__ int inv_cdf_block(WeightFn w, int V, float u, double *sd, int *si, double *total) {
-    const int seg = (V + blockDim.x - 1) / blockDim.x;
-    const int j0 = min(V, (int)threadIdx.x * seg), j1 = min(V, j0 + seg);
+__device__ __forceinline__ int inv_cdf_cluster(WeightFn w, int V, float u, double *sd, int *si, double *total,
+                                               ClusterSlots *pub, cg::cluster_group &cl, int slot) {
+    const int rank = (int)cl.block_rank();
+    int lo, hi;
+    tail_slice(V, rank, lo, hi);
+    const int seg = (hi - lo + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int j0 = min(hi, lo + (int)threadIdx.x * seg), j1 = min(hi, j0 + seg);
     double local = 0.0;
     int last_pos = -1;
     for (int j = j0; j < j1; ++j) {
@@ -118,16 +169,24 @@ __device__ __forceinline__ int inv_cdf_block(WeightFn w, int V, float u, double 
     if (lane == 31) sd[wid] = incl;
     if (threadIdx.x == 0) { si[0] = 0x7fffffff; si[1] = -1; }
     __syncthreads();
-    double warp_off = 0.0, S = 0.0;
+    double warp_off = 0.0, T = 0.0;
     for (int k = 0; k < nw; ++k) {  // nw <= 32: short serial pass keeps the order fixed
         double t = sd[k];
         if (k < wid) warp_off += t;
+        T += t;
+    }
+    if (threadIdx.x == 0) pub->d[1 + slot] = T;
+    cl.sync();
+    double cta_off = 0.0, S = 0.0;
+    for (int r = 0; r < kTailCluster; ++r) {
+        const double t = cl.map_shared_rank(pub, r)->d[1 + slot];
+        if (r < rank) cta_off += t;
         S += t;
     }
     *total = S;
-    if (!(S > 0.0)) { __syncthreads(); return -1; }
+    if (!(S > 0.0)) return -1;  // the same decision in every CTA of the cluster
     const double target = (double)u * S;
-    double run = warp_off + (incl - local);
+    double run = cta_off + warp_off + (incl - local);
     int hit = 0x7fffffff;
     if (run + local > target || run > target) {
         for (int j = j0; j < j1; ++j) {
@@ -139,9 +198,15 @@ __device__ __forceinline__ int inv_cdf_block(WeightFn w, int V, float u, double 
     if (hit != 0x7fffffff) atomicMin(&si[0], hit);
     if (last_pos >= 0) atomicMax(&si[1], last_pos);
     __syncthreads();
-    int res = si[0] != 0x7fffffff ? si[0] : si[1];
-    __syncthreads();
-    return res;
+    if (threadIdx.x == 0) { pub->i[1 + 2 * slot] = si[0]; pub->i[2 + 2 * slot] = si[1]; }
+    cl.sync();
+    int first = 0x7fffffff, last = -1;
+    for (int r = 0; r < kTailCluster; ++r) {
+        const ClusterSlots *o = cl.map_shared_rank(pub, r);
+        first = min(first, o->i[1 + 2 * slot]);
+        last = max(last, o->i[2 + 2 * slot]);
+    }
+    return first != 0x7fffffff ? first : last;
 }
 
 struct VerifyArgs {
@@ -159,29 +224,36 @@ struct VerifyArgs {
     RowStat *stats;         // scratch [B, K+1]
 };
 
-// grid (K+1, B): statistics of every row (+ optional export of the p row)
-__global__ void __launch_bounds__(kTailThreads) row_stats_kernel(VerifyArgs a) {
+// grid (kTailCluster (K+1), B), one cluster per row: statistics of every row (+ optional export of the p row)
+__global__ void __cluster_dims__(kTailCluster, 1, 1) __launch_bounds__(kTailThreads) row_stats_kernel(VerifyArgs a) {
     __shared__ float sv[32];
     __shared__ int si[32];
     __shared__ double sd[32];
-    const int i = blockIdx.x, b = blockIdx.y;
+    __shared__ ClusterSlots pub;
+    cg::cluster_group cl = cg::this_cluster();
+    const int i = blockIdx.x / kTailCluster, b = blockIdx.y;
     const float *lg = a.logits + ((size_t)b * (a.K + 1) + i) * a.V;
-    RowStat st = row_stats(lg, a.V, a.inv_t, sv, si, sd);
-    if (threadIdx.x == 0) a.stats[b * (a.K + 1) + i] = st;
+    RowStat st = row_stats(lg, a.V, a.inv_t, sv, si, sd, &pub, cl);
+    if (cl.block_rank() == 0 && threadIdx.x == 0) a.stats[b * (a.K + 1) + i] = st;
     if (a.p_debug) {
+        int lo, hi;
+        tail_slice(a.V, (int)cl.block_rank(), lo, hi);
         float *p = a.p_debug + ((size_t)b * (a.K + 1) + i) * a.V;
-        for (int j = threadIdx.x; j < a.V; j += blockDim.x) p[j] = prob_of(lg[j], st, a.inv_t, j);
+        for (int j = lo + threadIdx.x; j < hi; j += blockDim.x) p[j] = prob_of(lg[j], st, a.inv_t, j);
     }
+    cl.sync();
 }
 
-// grid (B): accept scan, then residual / bonus draw
-__global__ void __launch_bounds__(kTailThreads) verify_kernel(VerifyArgs a) {
+// grid (kTailCluster B), one cluster per sequence: accept scan, then residual / bonus draw
+__global__ void __cluster_dims__(kTailCluster, 1, 1) __launch_bounds__(kTailThreads) verify_kernel(VerifyArgs a) {
     __shared__ double sd[32];
     __shared__ int si[32];
     __shared__ int s_acc;
-    const int b = blockIdx.x, K = a.K, V = a.V;
+    __shared__ ClusterSlots pub;
+    cg::cluster_group cl = cg::this_cluster();
+    const int b = blockIdx.x / kTailCluster, K = a.K, V = a.V;
     const RowStat *st = a.stats + b * (K + 1);
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0) {  // (every CTA of the cluster takes the same few steps)
         int acc = 0;
         for (int i = 0; i < K; ++i) {
             int x = a.rows[b * (K + 1) + 1 + i];
@@ -203,17 +275,18 @@ __global__ void __launch_bounds__(kTailThreads) verify_kernel(VerifyArgs a) {
     int y = -1;
     if (acc < K) {
         const float *qr = a.q + ((size_t)b * K + acc) * V;
-        y = inv_cdf_block([&](int j) { return fmaxf(0.f, __fsub_rn(prob_of(lg[j], rs, inv_t, j), qr[j])); }, V, u,
-                          sd, si, &S);
+        y = inv_cdf_cluster([&](int j) { return fmaxf(0.f, __fsub_rn(prob_of(lg[j], rs, inv_t, j), qr[j])); }, V, u,
+                            sd, si, &S, &pub, cl, 0);
     }
     if (y < 0)  // all accepted: bonus from p_{K+1}; or an all-zero residual: fall back to p
-        y = inv_cdf_block([&](int j) { return prob_of(lg[j], rs, inv_t, j); }, V, u, sd, si, &S);
+        y = inv_cdf_cluster([&](int j) { return prob_of(lg[j], rs, inv_t, j); }, V, u, sd, si, &S, &pub, cl, 1);
     if (y < 0) y = rs.amax;  // a row whose probabilities all vanished (non-finite logits)
-    if (threadIdx.x == 0) {
+    if (cl.block_rank() == 0 && threadIdx.x == 0) {
         a.n_accepted[b] = acc;
         a.next_token[(size_t)b * a.next_stride] = y;
         if (a.keep) a.keep[b] = acc + 1;
     }
+    cl.sync();
 }
 
 struct DraftTailArgs {
@@ -226,23 +299,28 @@ struct DraftTailArgs {
     float *q_out; size_t q_stride;
 };
 
-// grid (B): q = softmax(last row / T), exported; x~ = inverse-CDF(q, u)
-__global__ void __launch_bounds__(kTailThreads) draft_tail_kernel(DraftTailArgs a) {
+// grid (kTailCluster B), one cluster per sequence: q = softmax(last row / T), exported; x~ = inverse-CDF(q, u)
+__global__ void __cluster_dims__(kTailCluster, 1, 1) __launch_bounds__(kTailThreads) draft_tail_kernel(DraftTailArgs a) {
     __shared__ float sv[32];
     __shared__ int si[32];
     __shared__ double sd[32];
-    const int b = blockIdx.x;
+    __shared__ ClusterSlots pub;
+    cg::cluster_group cl = cg::this_cluster();
+    const int b = blockIdx.x / kTailCluster;
     int row = a.n_eff[b] - 1;
     if (row < 0) row = 0;
     const float *lg = a.logits + ((size_t)b * a.M + row) * a.V;
-    const RowStat st = row_stats(lg, a.V, a.inv_t, sv, si, sd);
+    const RowStat st = row_stats(lg, a.V, a.inv_t, sv, si, sd, &pub, cl);
     float *q = a.q_out + (size_t)b * a.q_stride;
-    for (int j = threadIdx.x; j < a.V; j += blockDim.x) q[j] = prob_of(lg[j], st, a.inv_t, j);
-    __syncthreads();
+    int lo, hi;
+    tail_slice(a.V, (int)cl.block_rank(), lo, hi);
+    for (int j = lo + threadIdx.x; j < hi; j += blockDim.x) q[j] = prob_of(lg[j], st, a.inv_t, j);
+    __syncthreads();  // the draw below reads this CTA's own slice of q
     double S;
-    int y = inv_cdf_block([&](int j) { return q[j]; }, a.V, a.u[(size_t)b * a.u_stride], sd, si, &S);
+    int y = inv_cdf_cluster([&](int j) { return q[j]; }, a.V, a.u[(size_t)b * a.u_stride], sd, si, &S, &pub, cl, 0);
     if (y < 0) y = st.amax;
-    if (threadIdx.x == 0) a.token_out[(size_t)b * a.token_stride] = y;
+    if (cl.block_rank() == 0 && threadIdx.x == 0) a.token_out[(size_t)b * a.token_stride] = y;
+    cl.sync();
 }
 
 // ---------------- cache length bookkeeping ----------------
