@@ -31,7 +31,7 @@ METRIC = "generated tok/s, speculative vs autoregressive; verify-step HBM GB/s v
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one verify launch of forward_kernel from the ncu
 # capture summarised under profiles/ (taken on the kernel as it stands); other workloads: not captured
-NCU_TRAFFIC_PER_VERIFY_LAUNCH = {"neox-1.4b": 2.6699e9}
+NCU_TRAFFIC_PER_VERIFY_LAUNCH = {"neox-1.4b": 2.6699e9, "llama-7b-l4-ctx8k": 2.4913e9}
 
 # bench workloads: name -> (preset, batch, prompt, K, temperature)
 WORKLOADS = {
@@ -39,6 +39,9 @@ WORKLOADS = {
     "neox-2.7b": dict(preset="neox-2.7b"),
     "llama-7b-b8": dict(preset="llama-7b"),
     "llama-7b-b1": dict(preset="llama-7b", batch=1, prompt=2048),
+    # a four-layer cut of the 7B shape at a long context, small enough for a full profiler capture: the same
+    # per-layer phases (tensor-core attention items from this context on); time and bytes scale with the layers
+    "llama-7b-l4-ctx8k": dict(preset="llama-7b", batch=1, prompt=8192, layers=4),
     "tiny": dict(preset="tiny"),
 }
 
@@ -142,7 +145,10 @@ def resolve(workload):
     from paper_2311_04951_b200 import synth
     w = dict(WORKLOADS[workload])
     cfg = dict(synth.PRESETS[w.pop("preset")])
+    layers = w.pop("layers", None)
     cfg.update(w)
+    if layers:
+        cfg["target"] = cfg["target"].replace(n_layers=layers)
     return cfg
 
 
