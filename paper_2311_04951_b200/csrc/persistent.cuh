@@ -117,6 +117,8 @@ struct alignas(64) FwdParams {
     const CUtensorMap *tm_kv_ptr;  // where the copy engine can read tm_kv (set by the kernel: see params copy)
     int attn_tc;             // 1: attention_item_tc; 0: attention_item
     int kv_rows_per_layer;   // B * 2 * H * S
+    int attn_ctas;           // min(attention items, CTAs): set by the host together with the split plan
+    int overlap_out;         // parallel-residual block and at most half of the CTAs on attention
 };
 
 struct GemmDesc {
@@ -132,12 +134,19 @@ struct GemmDesc {
 };
 
 __device__ __forceinline__ int n_gemms(const FwdParams &p) { return 4 * p.n_layers + (p.want_logits ? 1 : 0); }
-__device__ __forceinline__ int barriers_per_layer(const FwdParams &p) { return p.parallel ? 4 : 8; }
+// CTAs that run an attention item in a phase (each at most one when this is below the grid size).
+__device__ __forceinline__ int attention_ctas(const FwdParams &p) { return p.attn_ctas; }
+// Parallel-residual blocks with at most half of the CTAs on attention: the MLP-out GEMM depends on the
+// activation, not on attention, so the CTAs without an attention item run it during the attention phase.
+__device__ __forceinline__ bool overlap_mlp_out(const FwdParams &p) { return p.overlap_out != 0; }
+__device__ __forceinline__ int barriers_per_layer(const FwdParams &p) { return p.parallel ? (overlap_mlp_out(p) ? 5 : 4) : 8; }
+__device__ __forceinline__ int attention_end(const FwdParams &p) { return overlap_mlp_out(p) ? 3 : 2; }  // barriers into the layer
 
 // GEMM number gi in execution order.  sequential: qkv, o, in, out; parallel: qkv, in, o, out.
 // Barrier count before layer l: 2 (set-up; embedding + first norm) + barriers_per_layer * l.
 //   sequential layer: qkv | attention | o | norm2 | in | act | out | next norm   (8 barriers)
 //   parallel layer:   qkv, in | attention + act | o, out | next norms            (4 barriers)
+//   ... with few attention items: qkv, in | act | attention (some CTAs) and out (the others) | o | next norms   (5)
 __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi, const float *const *ltab = nullptr) {
     GemmDesc g;
     const int l = gi >> 2, e = gi & 3;
@@ -145,17 +154,19 @@ __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi, const 
     if (l >= p.n_layers) {  // LM head
         g.tmW = &p.md->tm_lm; g.xop = p.op[OP_XN1];
         g.N = p.V; g.Kd = p.d; g.need = base; g.out = p.logits; g.ldo = p.V; g.bias = nullptr;
-        g.kind = 4; g.need_hi = base - barriers_per_layer(p) + 2;  // end of the last attention phase
+        g.kind = 4; g.need_hi = base - barriers_per_layer(p) + attention_end(p);  // end of the last attention phase
     } else {
         const LayerDesc *ld = layer_desc(p.md, l);
         int kind;  // 0 qkv, 1 o, 2 in, 3 out
-        if (p.parallel) kind = (e == 0) ? 0 : (e == 1) ? 2 : (e == 2) ? 1 : 3;
+        if (p.parallel && overlap_mlp_out(p)) kind = (e == 0) ? 0 : (e == 1) ? 2 : (e == 2) ? 3 : 1;  // out before o
+        else if (p.parallel) kind = (e == 0) ? 0 : (e == 1) ? 2 : (e == 2) ? 1 : 3;
         else kind = e;
         g.tmW = &ld->tm[kind];
         g.kind = kind;
         // the attention phase of layer l ends at barrier base + 2; qkv precedes it (previous layer's counts)
         // (so does the MLP input GEMM of a parallel-residual block)
-        g.need_hi = (kind == 0 || (kind == 2 && p.parallel)) ? (l == 0 ? 0 : base - barriers_per_layer(p) + 2) : base + 2;
+        g.need_hi = (kind == 0 || (kind == 2 && p.parallel)) ? (l == 0 ? 0 : base - barriers_per_layer(p) + attention_end(p))
+                                                             : base + attention_end(p);
         if (kind == 0) {
             g.xop = p.op[OP_XN1]; g.N = 3 * p.d; g.Kd = p.d; g.need = base;
             g.out = p.qkv; g.ldo = 3 * p.d; g.bias = ltab ? ltab[8 * l + 2] : ld->b_qkv;
@@ -182,8 +193,17 @@ __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi, const 
 __device__ __forceinline__ void unit_range(const FwdParams &p, const GemmDesc &g, int &c0, int &c1) {
     const long long total = (long long)g.n_tiles * g.kchunks;
     const int N = (int)gridDim.x, i = (int)blockIdx.x;
-    const int items = p.B * p.H * p.n_split * ((p.M + 15) / 16);
-    const int A = items < N ? items : N, bonus = p.stages - p.stages_lo;
+    const int A = attention_ctas(p), bonus = p.stages - p.stages_lo;
+    if (overlap_mlp_out(p)) {  // MLP-out runs beside attention on the CTAs without an item; everything else in equal shares
+        if (g.kind == 3) {
+            c0 = i < A ? 0 : (int)(total * (i - A) / (N - A));
+            c1 = i < A ? 0 : (int)(total * (i - A + 1) / (N - A));
+            return;
+        }
+        c0 = (int)(total * i / N);
+        c1 = (int)(total * (i + 1) / N);
+        return;
+    }
     const bool after_attention = p.parallel ? g.kind == 3 : g.kind == 1;
     if (after_attention && 2 * A <= N && bonus > 0) {  // (with most CTAs on attention the few others would become the stragglers)
         long long xa = (total + (long long)A * bonus) / N - bonus;  // an attention CTA's share
@@ -388,6 +408,16 @@ __device__ __forceinline__ bool grid_sync(const FwdParams &p, Shared *sh, int &e
     }
     named_bar(1, kWorkThreads);
     return sh->go != 0;
+}
+
+// Arrival at the next grid barrier without waiting for it (for a CTA whose next work does not depend on
+// what the others publish there).  Its own writes are published like at a full barrier.
+__device__ __forceinline__ void grid_arrive(const FwdParams &p, Shared *sh, int &epoch) {
+    fence_async_proxy();
+    __threadfence();
+    named_bar(1, kWorkThreads);
+    ++epoch;
+    if (threadIdx.x == 0 && sh->abort == 0) red_release_add(p.gbar, 1u);
 }
 
 // ---- non-GEMM phases (256 work threads) -------------------------------------------------------
@@ -1905,14 +1935,28 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             run_gemm<NT>(p, 4 * l + 0, smem);                       // qkv
             if (p.parallel) run_gemm<NT>(p, 4 * l + 1, smem);       // MLP in (same block input)
             if (!(go = grid_sync(p, sh, epoch))) break;
-            attention_phase(p, l, attn_scratch, sh);
-            if (p.parallel) act_phase(p);
-            if (!(go = grid_sync(p, sh, epoch))) break;
-            if (p.parallel) {
+            if (overlap_mlp_out(p)) {
+                act_phase(p);
+                if ((int)blockIdx.x < attention_ctas(p)) {
+                    grid_arrive(p, sh, epoch);  // the activation is out; attention needs nothing from the others
+                    attention_phase(p, l, attn_scratch, sh);
+                } else {
+                    if (!(go = grid_sync(p, sh, epoch))) break;
+                    run_gemm<NT>(p, 4 * l + 2, smem);               // MLP out -> x, beside the attention items
+                }
+                if (!(go = grid_sync(p, sh, epoch))) break;
+                run_gemm<NT>(p, 4 * l + 3, smem);                   // out-proj -> x
+                if (!(go = grid_sync(p, sh, epoch))) break;
+            } else if (p.parallel) {
+                attention_phase(p, l, attn_scratch, sh);
+                act_phase(p);
+                if (!(go = grid_sync(p, sh, epoch))) break;
                 run_gemm<NT>(p, 4 * l + 2, smem);                   // out-proj -> x
                 run_gemm<NT>(p, 4 * l + 3, smem);                   // MLP out  -> x
                 if (!(go = grid_sync(p, sh, epoch))) break;
             } else {
+                attention_phase(p, l, attn_scratch, sh);
+                if (!(go = grid_sync(p, sh, epoch))) break;
                 run_gemm<NT>(p, 4 * l + 1, smem);                   // out-proj -> x
                 if (!(go = grid_sync(p, sh, epoch))) break;
                 const float *const *lt = staged_ltab(sh);

@@ -424,7 +424,7 @@ int run_attention(const ssd_model *m, ssd_kv *kv, int layer, const float *q, int
     return SSD_OK;
 }
 
-inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 4 : 8) * a.n_layers; }
+inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 5 : 8) * a.n_layers; }  // upper bound
 
 template <int NT>
 int launch_forward_nt(FwdParams p, cudaStream_t st) {
@@ -519,6 +519,11 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
         }
     }
     if (!p.attn_tc) plan_split(groups, ctx, &p.chunk, &p.n_split, kAttnTile);
+    {
+        const int items = groups * p.n_split, sms = g_num_sms > 0 ? g_num_sms : 148;
+        p.attn_ctas = items < sms ? items : sms;
+        p.overlap_out = (a.parallel_residual && 2 * p.attn_ctas <= sms) ? 1 : 0;
+    }
     p.want_logits = want_logits ? 1 : 0;
     p.trace = (g_trace && 2 + barriers_needed(a) + 3 < kTraceSlots) ? w.trace : nullptr;
     CUDA_OK(cudaMemsetAsync(w.sync, 0, w.sync_bytes, st));
