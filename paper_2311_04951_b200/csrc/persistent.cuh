@@ -86,6 +86,7 @@ struct alignas(64) FwdParams {
     // architecture
     int n_layers, d, H, Dh, F, d_in, V, norm_kind, swiglu, parallel, rotary_dim, learned_pos, is_bf16_emb;
     float eps, rotary_base, attn_scale;
+    double inv_d;  // 1 / d (the norms' statistics are taken in fp64; a division there is a long routine)
     // rows
     int B, M, R;
     const int32_t *tokens;
@@ -480,25 +481,47 @@ __device__ __forceinline__ void grid_zero(float *dst, int R, int n, int ld) {
 }
 
 // Norm of every row of x into hi/lo operand buffers (one or two gain/bias sets from the same
-// statistics); one CTA per row.  The row (up to kNormRegs * 256 floats) stays in registers between
-// the statistics and the write pass, and all loads of a pass are issued before the first use, so
-// the phase costs about two L2 round trips instead of one per element.
-constexpr int kNormRegs = 8;  // float4 per thread: rows up to 8192 wide; wider rows are re-read
-__device__ __noinline__ void norm_phase(const FwdParams &p, const float *g1, const float *b1, int op1,
-                                           const float *g2, const float *b2, int op2, double *red) {
+// statistics); one CTA per row.  The row (Q float4 per thread) stays in registers between the
+// statistics and the write pass, and all loads of a pass are issued before the first use, so the
+// phase costs about two L2 round trips instead of one per element.  Q is a template parameter so
+// that a call executes only the code its row width needs: the instructions of a phase are not in
+// the instruction cache when it starts (the kernel is far larger than that cache), and every KB of
+// straight-line code costs a fraction of a microsecond to fetch.
+__device__ __forceinline__ void norm_emit(const FwdParams &p, int r, int i, const float4 v, float mu, float rs,
+                                          const float *g, const float *b, int op) {
+    const float4 gg = __ldg(reinterpret_cast<const float4 *>(g) + i);
+    float4 bb = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (b) bb = __ldg(reinterpret_cast<const float4 *>(b) + i);
+    const float y0 = (v.x - mu) * rs * gg.x + bb.x, y1 = (v.y - mu) * rs * gg.y + bb.y;
+    const float y2 = (v.z - mu) * rs * gg.z + bb.z, y3 = (v.w - mu) * rs * gg.w + bb.w;
+    const __nv_bfloat162 h01 = __floats2bfloat162_rn(y0, y1), h23 = __floats2bfloat162_rn(y2, y3);
+    const __nv_bfloat162 l01 = __floats2bfloat162_rn(y0 - __low2float(h01), y1 - __high2float(h01));
+    const __nv_bfloat162 l23 = __floats2bfloat162_rn(y2 - __low2float(h23), y3 - __high2float(h23));
+    __nv_bfloat16 *hi = p.op[op] + op_off(p.rk, op_row(r), 4 * i);
+    __nv_bfloat16 *lo = p.op[op] + op_off(p.rk, op_row(r) + 8, 4 * i);
+    uint2 hv, lv;
+    hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
+    lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
+    *reinterpret_cast<uint2 *>(hi) = hv;
+    *reinterpret_cast<uint2 *>(lo) = lv;
+}
+
+template <int Q>  // float4 per thread held in registers: rows up to Q * 1024 wide; wider rows are re-read
+__device__ __noinline__ void norm_rows(const FwdParams &p, const float *g1, const float *b1, int op1,
+                                          const float *g2, const float *b2, int op2, double *red) {
     const int n4 = p.d >> 2;  // d is a multiple of 8
     for (int r = blockIdx.x; r < p.R; r += gridDim.x) {
         const float4 *x4 = reinterpret_cast<const float4 *>(p.x + (size_t)r * p.d);
-        float4 xv[kNormRegs];
+        float4 xv[Q];
 #pragma unroll
-        for (int q = 0; q < kNormRegs; ++q) {
+        for (int q = 0; q < Q; ++q) {
             const int i = threadIdx.x + q * kWorkThreads;
             xv[q] = i < n4 ? __ldcg(x4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         // the gain / bias vectors were last read a whole pass of weights ago: fetch them now, under the
         // statistics, instead of as a second trip to DRAM after them
 #pragma unroll
-        for (int q = 0; q < kNormRegs; ++q) {
+        for (int q = 0; q < Q; ++q) {
             const int i = threadIdx.x + q * kWorkThreads;
             if (i < n4) {
                 prefetch_l1(reinterpret_cast<const float4 *>(g1) + i);
@@ -509,11 +532,12 @@ __device__ __noinline__ void norm_phase(const FwdParams &p, const float *g1, con
         }
         double s1 = 0.0, s2 = 0.0;
 #pragma unroll
-        for (int q = 0; q < kNormRegs; ++q) {
+        for (int q = 0; q < Q; ++q) {
             s1 += (double)xv[q].x + (double)xv[q].y + (double)xv[q].z + (double)xv[q].w;
             s2 += (double)xv[q].x * xv[q].x + (double)xv[q].y * xv[q].y + (double)xv[q].z * xv[q].z + (double)xv[q].w * xv[q].w;
         }
-        for (int i = threadIdx.x + kNormRegs * kWorkThreads; i < n4; i += kWorkThreads) {
+#pragma unroll 1
+        for (int i = threadIdx.x + Q * kWorkThreads; i < n4; i += kWorkThreads) {
             const float4 v = __ldcg(x4 + i);
             s1 += (double)v.x + (double)v.y + (double)v.z + (double)v.w;
             s2 += (double)v.x * v.x + (double)v.y * v.y + (double)v.z * v.z + (double)v.w * v.w;
@@ -521,44 +545,36 @@ __device__ __noinline__ void norm_phase(const FwdParams &p, const float *g1, con
         block_sum2_work(s1, s2, red);
         double mean = 0.0, var;
         if (p.norm_kind == 0) {
-            mean = s1 / p.d;
-            var = s2 / p.d - mean * mean;
+            mean = s1 * p.inv_d;
+            var = s2 * p.inv_d - mean * mean;
             if (var < 0.0) var = 0.0;
         } else {
-            var = s2 / p.d;
+            var = s2 * p.inv_d;
         }
         const float mu = (float)mean, rs = (float)rsqrt(var + (double)p.eps);
-        auto emit = [&](int i, const float4 v, const float *g, const float *b, int op) {
-            const float4 gg = __ldg(reinterpret_cast<const float4 *>(g) + i);
-            float4 bb = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (b) bb = __ldg(reinterpret_cast<const float4 *>(b) + i);
-            const float y0 = (v.x - mu) * rs * gg.x + bb.x, y1 = (v.y - mu) * rs * gg.y + bb.y;
-            const float y2 = (v.z - mu) * rs * gg.z + bb.z, y3 = (v.w - mu) * rs * gg.w + bb.w;
-            const __nv_bfloat162 h01 = __floats2bfloat162_rn(y0, y1), h23 = __floats2bfloat162_rn(y2, y3);
-            const __nv_bfloat162 l01 = __floats2bfloat162_rn(y0 - __low2float(h01), y1 - __high2float(h01));
-            const __nv_bfloat162 l23 = __floats2bfloat162_rn(y2 - __low2float(h23), y3 - __high2float(h23));
-            __nv_bfloat16 *hi = p.op[op] + op_off(p.rk, op_row(r), 4 * i);
-            __nv_bfloat16 *lo = p.op[op] + op_off(p.rk, op_row(r) + 8, 4 * i);
-            uint2 hv, lv;
-            hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
-            lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
-            *reinterpret_cast<uint2 *>(hi) = hv;
-            *reinterpret_cast<uint2 *>(lo) = lv;
-        };
+#pragma unroll 1
+        for (int e = 0; e < (g2 ? 2 : 1); ++e) {  // (rolled: the second gain set reuses the first one's code)
+            const float *g = e ? g2 : g1, *b = e ? b2 : b1;
+            const int op = e ? op2 : op1;
 #pragma unroll
-        for (int q = 0; q < kNormRegs; ++q) {
-            const int i = threadIdx.x + q * kWorkThreads;
-            if (i < n4) {
-                emit(i, xv[q], g1, b1, op1);
-                if (g2) emit(i, xv[q], g2, b2, op2);
+            for (int q = 0; q < Q; ++q) {
+                const int i = threadIdx.x + q * kWorkThreads;
+                if (i < n4) norm_emit(p, r, i, xv[q], mu, rs, g, b, op);
             }
-        }
-        for (int i = threadIdx.x + kNormRegs * kWorkThreads; i < n4; i += kWorkThreads) {
-            const float4 v = __ldcg(x4 + i);
-            emit(i, v, g1, b1, op1);
-            if (g2) emit(i, v, g2, b2, op2);
+#pragma unroll 1
+            for (int i = threadIdx.x + Q * kWorkThreads; i < n4; i += kWorkThreads)
+                norm_emit(p, r, i, __ldcg(x4 + i), mu, rs, g, b, op);
         }
     }
+}
+
+__device__ __noinline__ void norm_phase(const FwdParams &p, const float *g1, const float *b1, int op1,
+                                           const float *g2, const float *b2, int op2, double *red) {
+    const int n4 = p.d >> 2;
+    if (n4 <= kWorkThreads) norm_rows<1>(p, g1, b1, op1, g2, b2, op2, red);
+    else if (n4 <= 2 * kWorkThreads) norm_rows<2>(p, g1, b1, op1, g2, b2, op2, red);
+    else if (n4 <= 4 * kWorkThreads) norm_rows<4>(p, g1, b1, op1, g2, b2, op2, red);
+    else norm_rows<8>(p, g1, b1, op1, g2, b2, op2, red);
 }
 
 // MLP activation of t_in into the hi/lo operand of the down projection, spread over the grid

@@ -494,6 +494,7 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     p.n_layers = a.n_layers; p.d = a.d_model; p.H = a.n_heads; p.Dh = a.head_dim; p.F = a.d_ff; p.d_in = m->d_in;
     p.V = a.vocab; p.norm_kind = a.norm; p.swiglu = a.act == 1; p.parallel = a.parallel_residual;
     p.rotary_dim = a.pos == 1 ? a.rotary_dim : 0; p.learned_pos = a.pos == 0; p.is_bf16_emb = 1;
+    p.inv_d = 1.0 / (double)a.d_model;
     p.eps = a.norm_eps; p.rotary_base = a.rotary_base; p.attn_scale = 1.0f / sqrtf((float)a.head_dim);
     p.B = kv->B; p.M = M; p.R = R;
     p.tokens = tokens; p.tok_stride = tok_stride; p.n_rows = n_rows;
