@@ -144,14 +144,14 @@ __device__ __forceinline__ int barriers_per_layer(const FwdParams &p) { return p
 __device__ __forceinline__ int attention_end(const FwdParams &p) { return overlap_mlp_out(p) ? 3 : 2; }  // barriers into the layer
 
 // GEMM number gi in execution order.  sequential: qkv, o, in, out; parallel: qkv, in, o, out.
-// Barrier count before layer l: 2 (set-up; embedding + first norm) + barriers_per_layer * l.
+// Barrier count before layer l: 1 (set-up, embedding and first norm) + barriers_per_layer * l.
 //   sequential layer: qkv | attention | o | norm2 | in | act | out | next norm   (8 barriers)
 //   parallel layer:   qkv, in | attention + act | o, out | next norms            (4 barriers)
 //   ... with few attention items: qkv, in | act | attention (some CTAs) and out (the others) | o | next norms   (5)
 __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi, const float *const *ltab = nullptr) {
     GemmDesc g;
     const int l = gi >> 2, e = gi & 3;
-    const int base = 2 + barriers_per_layer(p) * l;
+    const int base = 1 + barriers_per_layer(p) * l;
     if (l >= p.n_layers) {  // LM head
         g.tmW = &p.md->tm_lm; g.xop = p.op[OP_XN1];
         g.N = p.V; g.Kd = p.d; g.need = base; g.out = p.logits; g.ldo = p.V; g.bias = nullptr;
@@ -1934,18 +1934,18 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                 grid_zero(p.logits, p.R, p.V, p.V);
             }
         };
+        // Set-up, embedding and the first norm of a row all run on the CTA that owns the row, so only
+        // CTA-wide barriers separate them: one grid barrier in front of the first GEMM instead of two.
         setup_phase(p);
+        named_bar(2, kWorkThreads);  // the row's position and validity are read back by the embedding
+        embed_phase(p);
+        named_bar(2, kWorkThreads);  // the embedding rows are read back by the norm
+        norm_for_layer(0);
         bool go = grid_sync(p, sh, epoch);
-        if (go) {
-            if (threadIdx.x < 64) {  // lengths and rows of this pass (written by the set-up phase), for the attention items
-                const int b = threadIdx.x;
-                seq_tab[b] = b < p.B ? p.len[b] : 0;
-                seq_tab[64 + b] = b < p.B ? __ldcg(p.ri.n_eff + b) : 0;
-            }
-            embed_phase(p);
-            named_bar(2, kWorkThreads);  // the embedding rows are read back by the CTA that wrote them
-            norm_for_layer(0);
-            go = grid_sync(p, sh, epoch);
+        if (go && threadIdx.x < 64) {  // lengths and rows of this pass (written by the set-up of every row), for the
+            const int b = threadIdx.x;  // attention items, which run behind further grid barriers
+            seq_tab[b] = b < p.B ? p.len[b] : 0;
+            seq_tab[64 + b] = b < p.B ? __ldcg(p.ri.n_eff + b) : 0;
         }
         for (int l = 0; l < p.n_layers && go; ++l) {
             run_gemm<NT>(p, 4 * l + 0, smem);                       // qkv
