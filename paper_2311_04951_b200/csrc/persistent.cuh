@@ -129,6 +129,7 @@ struct GemmDesc {
     int need;  // grid barriers that must have completed before its operand exists
     int need_hi;  // ... before its tiles may use the ring slots shared with the attention scratch
     int kind;     // 0 qkv, 1 o, 2 in, 3 out, 4 LM head
+    unsigned wait_attn;  // attention CTAs that must have signalled before its operand exists (0: a grid barrier covers it)
     float *out;
     int ldo;
     const float *bias;
@@ -140,16 +141,18 @@ __device__ __forceinline__ int attention_ctas(const FwdParams &p) { return p.att
 // Parallel-residual blocks with at most half of the CTAs on attention: the MLP-out GEMM depends on the
 // activation, not on attention, so the CTAs without an attention item run it during the attention phase.
 __device__ __forceinline__ bool overlap_mlp_out(const FwdParams &p) { return p.overlap_out != 0; }
-__device__ __forceinline__ int barriers_per_layer(const FwdParams &p) { return p.parallel ? (overlap_mlp_out(p) ? 5 : 4) : 8; }
+__device__ __forceinline__ int barriers_per_layer(const FwdParams &p) { return p.parallel ? 4 : 8; }
 __device__ __forceinline__ int attention_end(const FwdParams &p) { return overlap_mlp_out(p) ? 3 : 2; }  // barriers into the layer
 
 // GEMM number gi in execution order.  sequential: qkv, o, in, out; parallel: qkv, in, o, out.
 // Barrier count before layer l: 1 (set-up, embedding and first norm) + barriers_per_layer * l.
 //   sequential layer: qkv | attention | o | norm2 | in | act | out | next norm   (8 barriers)
 //   parallel layer:   qkv, in | attention + act | o, out | next norms            (4 barriers)
-//   ... with few attention items: qkv, in | act | attention (some CTAs) and out (the others) | o | next norms   (5)
+//   ... with few attention items: qkv, in | act | attention (some CTAs); out, then - once every attention CTA has
+//       signalled - o (the others) | next norms   (4)
 __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi, const float *const *ltab = nullptr) {
     GemmDesc g;
+    g.wait_attn = 0;
     const int l = gi >> 2, e = gi & 3;
     const int base = 1 + barriers_per_layer(p) * l;
     if (l >= p.n_layers) {  // LM head
@@ -173,6 +176,7 @@ __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi, const 
             g.out = p.qkv; g.ldo = 3 * p.d; g.bias = ltab ? ltab[8 * l + 2] : ld->b_qkv;
         } else if (kind == 1) {
             g.xop = p.op[OP_AO]; g.N = p.d; g.Kd = p.d; g.need = base + 2;
+            if (overlap_mlp_out(p)) g.wait_attn = (unsigned)(l + 1) * (unsigned)attention_ctas(p);
             g.out = p.x; g.ldo = p.d; g.bias = ltab ? ltab[8 * l + 3] : ld->b_o;
         } else if (kind == 2) {
             g.xop = p.op[p.parallel ? OP_XN2 : OP_XN1]; g.N = p.d_in; g.Kd = p.d; g.need = p.parallel ? base : base + 4;
@@ -196,7 +200,7 @@ __device__ __forceinline__ void unit_range(const FwdParams &p, const GemmDesc &g
     const int N = (int)gridDim.x, i = (int)blockIdx.x;
     const int A = attention_ctas(p), bonus = p.stages - p.stages_lo;
     if (overlap_mlp_out(p)) {  // MLP-out runs beside attention on the CTAs without an item; everything else in equal shares
-        if (g.kind == 3) {
+        if (g.kind == 3 || g.kind == 1) {  // (the out-projection follows on the same CTAs: see attn_done)
             c0 = i < A ? 0 : (int)(total * (i - A) / (N - A));
             c1 = i < A ? 0 : (int)(total * (i - A + 1) / (N - A));
             return;
@@ -419,6 +423,18 @@ __device__ __forceinline__ void grid_arrive(const FwdParams &p, Shared *sh, int 
     named_bar(1, kWorkThreads);
     ++epoch;
     if (threadIdx.x == 0 && sh->abort == 0) red_release_add(p.gbar, 1u);
+}
+
+// Count of attention CTAs that have finished their items, over the layers of this pass (zeroed with the
+// barrier counter before the launch).  With few attention items in a parallel-residual block the CTAs
+// without an item run the MLP-out GEMM beside the attention and go straight on to the out-projection:
+// its operand issuer waits for this count instead of a grid barrier.
+__device__ __forceinline__ unsigned *attn_done(const FwdParams &p) { return p.gbar + 8; }
+__device__ __forceinline__ void attn_signal(const FwdParams &p, Shared *sh) {
+    fence_async_proxy();  // the attention output is read by other CTAs' bulk copies
+    __threadfence();
+    named_bar(1, kWorkThreads);
+    if (threadIdx.x == 0 && sh->abort == 0) red_release_add(attn_done(p), 1u);
 }
 
 // ---- non-GEMM phases (256 work threads) -------------------------------------------------------
@@ -1688,7 +1704,22 @@ __device__ __noinline__ void run_gemm(const FwdParams &p, int gi, uint8_t *smem)
                 __syncwarp();
             } else if (warp == kXWarp) {
                 // operand tiles of this GEMM (their phase has been released: this runs after its barrier)
-                if (lane == 0 && !sh->abort) {
+                bool ready = true;
+                if (lane == 0 && !sh->abort && g.wait_attn) {
+                    // the attention output is complete once every attention CTA of this layer has signalled
+                    const unsigned *cnt = attn_done(p);
+                    if (ld_acquire(cnt) < g.wait_attn) {
+                        const long long t0 = clock64();
+                        while (ld_acquire(cnt) < g.wait_attn) {
+                            if (sh->abort || clock64() - t0 > kWaitCycles) { ready = false; break; }
+                        }
+                    }
+                    if (!ready) {
+                        set_status(p.status, kTimeoutCode);
+                        sh->abort = 1;
+                    }
+                }
+                if (lane == 0 && ready && !sh->abort) {
                     fence_async_proxy();  // that phase's generic-proxy writes -> visible to the bulk copies
                     int kx = c0 % g.kchunks;
                     for (int c = c0; c < c1; ++c) {
@@ -1956,12 +1987,12 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                 if ((int)blockIdx.x < attention_ctas(p)) {
                     grid_arrive(p, sh, epoch);  // the activation is out; attention needs nothing from the others
                     attention_phase(p, l, attn_scratch, sh);
+                    attn_signal(p, sh);
                 } else {
                     if (!(go = grid_sync(p, sh, epoch))) break;
                     run_gemm<NT>(p, 4 * l + 2, smem);               // MLP out -> x, beside the attention items
+                    run_gemm<NT>(p, 4 * l + 3, smem);               // out-proj -> x, once the attention CTAs have signalled
                 }
-                if (!(go = grid_sync(p, sh, epoch))) break;
-                run_gemm<NT>(p, 4 * l + 3, smem);                   // out-proj -> x
                 if (!(go = grid_sync(p, sh, epoch))) break;
             } else if (p.parallel) {
                 attention_phase(p, l, attn_scratch, sh);
