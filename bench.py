@@ -31,7 +31,7 @@ METRIC = "generated tok/s, speculative vs autoregressive; verify-step HBM GB/s v
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one verify launch of forward_kernel from the ncu
 # capture summarised under profiles/ (taken on the kernel as it stands); other workloads: not captured
-NCU_TRAFFIC_PER_VERIFY_LAUNCH = {"neox-1.4b": 2.6699e9, "llama-7b-l4-ctx8k": 2.4913e9}
+NCU_TRAFFIC_PER_VERIFY_LAUNCH = {"neox-1.4b": 2.6736e9, "llama-7b-l4-ctx8k": 2.4925e9}
 
 # bench workloads: name -> (preset, batch, prompt, K, temperature)
 WORKLOADS = {

@@ -64,6 +64,16 @@ def test_forward_many_heads_one_split_of_many_chunks(mode):
     _forward_over_seeded_cache(synth.llama_like(1, 4096, 32, 512, 512), [1151, 127, 1152, 64, 300], 5, mode, scale=1.5)
 
 
+@pytest.mark.parametrize("mode", [2, 1])
+@pytest.mark.parametrize("lens,M", [([700, 90], 6), ([2100], 5), ([300, 1, 129], 2)])
+def test_parallel_residual_out_projection_behind_the_attention_count(lens, M, mode):
+    """Parallel-residual layers with few attention items: some CTAs run the attention items while the others
+    run the MLP-out GEMM and then the out-projection, whose operand copies wait for the count of finished
+    attention CTAs instead of a grid barrier.  Several layers (the count runs on from layer to layer),
+    several splits per head (the last split to finish merges before its CTA signals), both attention forms."""
+    _forward_over_seeded_cache(synth.neox_like(3, 256, 2, 512, 520), lens, M, mode)
+
+
 def _forward_over_seeded_cache(arch, lens, M, mode, scale=6.0):
     """Whole verification pass (single forward kernel) of a head-128 model over a seeded cache:
     logits of all rows and the appended cache rows against the oracle.  Exercises the tensor-core
