@@ -52,3 +52,68 @@ def test_verify_pass_at_the_1p4b_shape_matches_the_oracle():
     cache = kv.cache_view().float().cpu().numpy()[:, 0, :, :, :P + K + 1]
     r = oc.kv[:, :, :, :P + K + 1]
     assert (np.abs(cache - r) <= gu.LOGIT_RTOL * np.abs(r) + gu.LOGIT_ATOL).all()
+
+
+def test_7b_shape_pass_in_the_bench_configuration_properties():
+    """The 7B Llama shape at full width and depth (32 layers, d 4096, 32 heads x 128, SwiGLU 11008, vocab
+    32000), batch 1, context 2048, K = 4: the launch configuration of the verify sweep.  The oracle needs
+    minutes for a pass of this size, so the pass is checked through properties that hold at any size:
+    the five rows fed together give the logits and cache rows of the same rows fed one at a time (the
+    claim that lets one verification pass replace K + 1 decode steps), the probabilities are the softmax
+    of the logits (numpy, fp64), and the accept / resample decisions follow the oracle's rule on the
+    pass's own rows."""
+    import bench
+    arch = synth.PRESETS["llama-7b"]["target"]
+    K, T, ctx, S = 4, 1.0, 2048, 2048 + 64
+    dev = "cuda"
+    model = B.Model(arch, bench.random_weights_on_device(arch, 31, torch))   # bench.py's device-side N(0, 0.02) init
+    V = arch.vocab
+    g = torch.Generator(device=dev)
+    g.manual_seed(5)
+    fill = torch.randn((arch.n_layers, 1, 2, arch.n_heads, S, arch.head_dim), generator=g, device=dev) * 0.5
+
+    def fresh_kv():
+        kv = B.KV(model, 1, S)
+        kv.cache_view().copy_(fill)
+        B.kv_commit(kv, torch.tensor([ctx], dtype=torch.int32, device=dev))
+        assert kv.lengths().tolist() == [ctx]
+        return kv
+
+    rows_np = synth.gen_prompt(91, 1, K + 1, V)
+    q_np = synth.gen_dirichlet_rows(92, K, V).reshape(1, K, V)
+    u_np = synth.gen_uniforms(93, 0, 0, K + 1).reshape(1, K + 1)
+    n_acc = torch.zeros(1, dtype=torch.int32, device=dev)
+    nxt = torch.zeros(1, dtype=torch.int32, device=dev)
+    p_dbg = torch.zeros(1, K + 1, V, device=dev)
+    kv = fresh_kv()
+    ws = model.new_workspace(1, K + 1, S)
+    B.target_verify(model, kv, torch.from_numpy(rows_np).to(dev), K, torch.from_numpy(q_np).to(dev),
+                    torch.from_numpy(u_np).to(dev), T, n_acc, nxt, 1, p_dbg, ws)
+    together = B.last_logits(model, 1, K + 1, ws).cpu().numpy()[0]
+    p_gpu = p_dbg.cpu().numpy()[0]
+    assert kv.status() == 0
+    cache_together = kv.cache_view().float().cpu().numpy()[:, 0, :, :, ctx:ctx + K + 1]
+    assert np.abs(together).max() > 0.5                      # the comparison below is not about zeros
+    # probabilities = softmax of the logits
+    z = together.astype(np.float64) / T
+    e = np.exp(z - z.max(axis=1, keepdims=True))
+    assert np.abs(p_gpu - e / e.sum(axis=1, keepdims=True)).max() <= gu.P_ATOL
+    # decisions follow the rule on the pass's own rows
+    gu.check_decisions_on_own_rows(p_gpu, q_np[0], rows_np[0, 1:], u_np[0, :K], u_np[0, K],
+                                   int(n_acc.cpu()[0]), int(nxt.cpu()[0]))
+    # one row at a time
+    kv1 = fresh_kv()
+    ws1 = model.new_workspace(1, 1, S)
+    one = torch.ones(1, dtype=torch.int32, device=dev)
+    u1 = torch.full((1, 1), 0.5, device=dev)
+    for i in range(K + 1):
+        B.target_verify(model, kv1, torch.from_numpy(rows_np[:, i:i + 1].copy()).to(dev), 0, None, u1, T, n_acc, nxt, 1,
+                        None, ws1)
+        single = B.last_logits(model, 1, 1, ws1).cpu().numpy()[0, 0]
+        B.kv_commit(kv1, one)
+        gu.assert_logits_close(single, together[i])         # same math; fp32 reduction order and bf16 K/V flips only
+    assert kv1.status() == 0 and kv1.lengths().tolist() == [ctx + K + 1]
+    cache_single = kv1.cache_view().float().cpu().numpy()[:, 0, :, :, ctx:ctx + K + 1]
+    tol = gu.LOGIT_RTOL * np.abs(cache_single) + gu.LOGIT_ATOL
+    assert (np.abs(cache_together - cache_single) <= tol).all()
+    assert (cache_together == cache_single).mean() > 0.8
