@@ -184,6 +184,10 @@ int target_verify(ssd_model *target, ssd_kv *tkv, const int32_t *dev_rows, int K
  * keeps n_accepted + 1 as the last target_verify on this cache left it on the device.
  * Rejected rows are not erased: they lie beyond the length and are overwritten later
  * (Section "So, what's the problem?": no redundant calculation, no copy).
+ * n_keep[b] is at most the number of rows of that forward.  The host plans the attention splits of a
+ * pass from an upper bound of the lengths, which it advances by the rows of every forward and which
+ * kv_lengths makes exact again; a caller that makes a length jump in another way (a cache it filled
+ * itself, then a large n_keep) calls kv_lengths before the next forward.
  */
 int kv_commit(ssd_kv *kv, const int32_t *dev_n_keep, void *stream);
 

@@ -117,3 +117,57 @@ def test_7b_shape_pass_in_the_bench_configuration_properties():
     tol = gu.LOGIT_RTOL * np.abs(cache_single) + gu.LOGIT_ATOL
     assert (np.abs(cache_together - cache_single) <= tol).all()
     assert (cache_together == cache_single).mean() > 0.8
+
+
+def test_7b_shape_batch_of_eight_equals_single_sequences():
+    """The batched configuration at full size: 8 independent sequences x (K + 1 = 5) rows = 40 rows in one pass of
+    the 7B shape (the 40-row operand tiles and M = 128 MMAs, 256 (sequence, head) attention groups on 148 SMs),
+    with ragged cache lengths.  Sequences are independent, so a sequence's logits, decisions and appended
+    cache rows must be those of the same sequence run alone (the 8-row path checked above)."""
+    import bench
+    arch = synth.PRESETS["llama-7b"]["target"]
+    K, T, S, Bn = 4, 1.0, 2048 + 64, 8
+    lens = [2048, 1900, 2047, 1024, 2048, 129, 640, 2048]
+    dev = "cuda"
+    model = B.Model(arch, bench.random_weights_on_device(arch, 31, torch))
+    V = arch.vocab
+    g = torch.Generator(device=dev)
+    kv = B.KV(model, Bn, S)
+    view = kv.cache_view()                                   # [L, B, 2, H, S, Dh] bf16
+    for b in range(Bn):
+        g.manual_seed(100 + b)
+        view[:, b].copy_(torch.randn((arch.n_layers, 2, arch.n_heads, S, arch.head_dim), generator=g, device=dev) * 0.5)
+    B.kv_commit(kv, torch.tensor(lens, dtype=torch.int32, device=dev))
+    assert kv.lengths().tolist() == lens
+    rows_np = synth.gen_prompt(94, Bn, K + 1, V)
+    q_np = synth.gen_dirichlet_rows(95, Bn * K, V).reshape(Bn, K, V)
+    u_np = np.stack([synth.gen_uniforms(96, b, 0, K + 1) for b in range(Bn)])
+    n_acc = torch.zeros(Bn, dtype=torch.int32, device=dev)
+    nxt = torch.zeros(Bn, dtype=torch.int32, device=dev)
+    p_dbg = torch.zeros(Bn, K + 1, V, device=dev)
+    ws = model.new_workspace(Bn, K + 1, S)
+    B.target_verify(model, kv, torch.from_numpy(rows_np).to(dev), K, torch.from_numpy(q_np).to(dev),
+                    torch.from_numpy(u_np).to(dev), T, n_acc, nxt, 1, p_dbg, ws)
+    batched = B.last_logits(model, Bn, K + 1, ws).cpu().numpy()
+    assert kv.status() == 0 and kv.lengths().tolist() == lens
+    p_gpu, a_gpu, y_gpu = p_dbg.cpu().numpy(), n_acc.cpu().numpy(), nxt.cpu().numpy()
+    for b in range(Bn):
+        gu.check_decisions_on_own_rows(p_gpu[b], q_np[b], rows_np[b, 1:], u_np[b, :K], u_np[b, K], int(a_gpu[b]), int(y_gpu[b]))
+    for b in (1, 5, 7):                                       # sampled sequences, each alone on a cache of its own
+        kv1 = B.KV(model, 1, S)
+        kv1.cache_view()[:, 0].copy_(view[:, b])
+        # (the batched pass appended its rows behind lens[b]; the single pass overwrites them with its own)
+        B.kv_commit(kv1, torch.tensor([lens[b]], dtype=torch.int32, device=dev))
+        assert kv1.lengths().tolist() == [lens[b]]          # (also refreshes the host-side bound the splits are planned from)
+        ws1 = model.new_workspace(1, K + 1, S)
+        B.target_verify(model, kv1, torch.from_numpy(rows_np[b:b + 1].copy()).to(dev), K,
+                        torch.from_numpy(q_np[b:b + 1].copy()).to(dev), torch.from_numpy(u_np[b:b + 1].copy()).to(dev), T,
+                        n_acc[:1], nxt[:1], 1, None, ws1)
+        alone = B.last_logits(model, 1, K + 1, ws1).cpu().numpy()[0]
+        assert kv1.status() == 0
+        gu.assert_logits_close(batched[b], alone)
+        n0 = lens[b]
+        cb = view[:, b, :, :, n0:n0 + K + 1].float().cpu().numpy()
+        c1 = kv1.cache_view()[:, 0, :, :, n0:n0 + K + 1].float().cpu().numpy()
+        assert (np.abs(cb - c1) <= gu.LOGIT_RTOL * np.abs(c1) + gu.LOGIT_ATOL).all()
+        assert (cb == c1).mean() > 0.8
