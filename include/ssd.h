@@ -140,8 +140,8 @@ int kv_prefill(ssd_model *m, ssd_kv *kv, const int32_t *dev_tokens, const int32_
                void *dev_ws, size_t ws_bytes, void *stream);
 
 /*
- * One draft step (Section "Speculative Sampling": the draft model runs "for a short sequence
- * of calls").  Feeds n_in[b] (1..rows_in) rows per sequence -- the tokens the draft cache has
+ * One draft step (Section "Speculative Sampling": the small model is called a few times in a row to
+ * propose tokens).  Feeds n_in[b] (1..rows_in) rows per sequence -- the tokens the draft cache has
  * not seen yet -- commits them to the draft cache, turns the LAST fed row's logits into
  * q = softmax(logits / temperature), draws x~ = inverse-CDF(q, u[b]) and writes both.
  *   dev_tokens_in  int32, token j of sequence b at [b * tokens_stride + j], j < rows_in (1 or 2)
@@ -158,8 +158,8 @@ int draft_step(ssd_model *draft, ssd_kv *dkv, const int32_t *dev_tokens_in, int 
                size_t ws_bytes, void *stream);
 
 /*
- * The verification step (Section "Autoregressive vs Speculative Sampling": K draft tokens are
- * "evaluated in the target model together"; Figure 2).  One forward over K+1 rows per sequence
+ * The verification step (Section "Autoregressive vs Speculative Sampling": the target model scores
+ * all K draft tokens in one pass; Figure 2).  One forward over K+1 rows per sequence
  *   dev_rows[b, 0..K] = pending token, x~_1 .. x~_K                 (int32, row stride K+1)
  * at positions len[b] .. len[b]+K against the cache, giving p_1 .. p_{K+1} = softmax(logits / T);
  * then per sequence, left to right: accept x~_i iff u_i * q_i(x~_i) < p_i(x~_i) (i.e. with
@@ -184,14 +184,20 @@ int target_verify(ssd_model *target, ssd_kv *tkv, const int32_t *dev_rows, int K
  * keeps n_accepted + 1 as the last target_verify on this cache left it on the device.
  * Rejected rows are not erased: they lie beyond the length and are overwritten later
  * (Section "So, what's the problem?": no redundant calculation, no copy).
- * n_keep[b] is at most the number of rows of that forward.  The host plans the attention splits of a
- * pass from an upper bound of the lengths, which it advances by the rows of every forward and which
- * kv_lengths makes exact again; a caller that makes a length jump in another way (a cache it filled
- * itself, then a large n_keep) calls kv_lengths before the next forward.
+ * n_keep[b] is at most the number of rows of that forward.  A length that would exceed the cache's
+ * capacity is clamped to it and SSD_E_CAPACITY is recorded in the sticky status word.  The host plans the
+ * attention splits of a pass from an upper bound of the lengths, which the bookkeeping kernels keep close
+ * to the real lengths and kv_lengths makes exact; a caller that makes a length jump in another way (a cache
+ * it filled itself, then a large n_keep) calls kv_lengths before the next forward.
  */
 int kv_commit(ssd_kv *kv, const int32_t *dev_n_keep, void *stream);
 
-/* Cut sequences back: length[b] = min(length[b], dev_new_len[b]). */
+/* Cut sequences back: length[b] = min(length[b], dev_new_len[b]) (int32 [batch] on the device).  Rows beyond
+ * the new length are not erased; later passes overwrite them.  This is how rejected draft rows leave a cache
+ * and how a caller resynchronises a cache with a token sequence of its own choice: cut back, then feed the
+ * other tokens.  After a cut and a re-feed the cache equals the cache of a fresh prompt pass over the same
+ * tokens.  (Section "So, what's the problem?": the caches of both models are fixed up to the accepted
+ * prefix, and nothing that is still valid is computed again.) */
 int kv_rollback(ssd_kv *kv, const int32_t *dev_new_len, void *stream);
 
 /*
@@ -272,6 +278,17 @@ int ssd_last_logits(const ssd_model *m, int batch, int rows_per_seq, const void 
 int ssd_set_trace(int enable);
 int ssd_read_trace(const ssd_model *m, int batch, int rows_per_seq, const void *dev_ws, size_t ws_bytes,
                    uint64_t *host_out, int max_entries, int *n_out, void *stream);
+
+/* Failure detection.  Every device-side wait is bounded: a wait that takes work (a weight tile, an operand,
+ * a grid barrier, a count of finished attention items) gives up after `cycles` GPU clock cycles, records
+ * SSD_E_TIMEOUT in the cache's sticky status word, and its kernel stops taking work, waits for its own
+ * copies in flight (those drain waits keep the default bound), releases its tensor memory and returns, so
+ * the context stays usable.  0 restores the default of about two seconds; negative: SSD_E_ARG.
+ * ssd_wait_probe exercises that path without disturbing anything else: it queues a one-thread kernel that
+ * waits, with the configured bound, on a barrier nobody ever arrives at; after it has run,
+ * ssd_device_status(kv) reports SSD_E_TIMEOUT.  (No counterpart in the paper: housekeeping.) */
+int ssd_set_wait_limit(long long cycles);
+int ssd_wait_probe(ssd_kv *kv, void *stream);
 
 /* Number of kernels this library has launched in this process so far. */
 uint64_t ssd_launch_count(void);

@@ -4,7 +4,7 @@ The vocabulary-wide part of speculative sampling, step by step, in numpy:
 temperature softmax, inverse-CDF sampling, and the accept / reject / resample rule.
 
 The paper names the method (Section "Speculative Sampling", Figure 2: the target model
-"qualifies and accepts (or rejects)" K draft tokens, and samples one token itself when a
+passes or refuses each of the K draft tokens, and samples one token itself when a
 rejection occurs) and quotes its guarantee (Section "Autoregressive vs Speculative
 Sampling": the target distribution is recovered).  The rule that achieves the guarantee is
 the modified rejection sampling of the scheme the paper cites:

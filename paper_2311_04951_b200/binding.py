@@ -38,7 +38,7 @@ EXPORTS = ["ssd_model_create", "ssd_model_desc_bytes", "ssd_set_persistent", "ss
            "ssd_workspace_bytes", "kv_init", "kv_destroy", "kv_prefill", "draft_step", "target_verify",
            "kv_commit", "kv_rollback", "spec_advance", "kv_lengths", "ssd_device_status",
            "verify_from_logits", "verify_from_logits_noalloc", "verify_scratch_bytes", "attention_rows", "ssd_last_logits", "ssd_set_trace", "ssd_read_trace", "ssd_launch_count",
-           "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror"]
+           "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror", "ssd_set_wait_limit", "ssd_wait_probe"]
 
 
 def lib_path() -> str:
@@ -91,6 +91,8 @@ def load():
     L.ssd_launch_count.restype = ctypes.c_uint64
     L.ssd_gemm_profile.argtypes = [i32]
     L.ssd_gemm_profile_read.argtypes = [ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_double), i32]
+    L.ssd_set_wait_limit.argtypes = [ctypes.c_longlong]
+    L.ssd_wait_probe.argtypes = [vp, vp]
     L.ssd_strerror.argtypes = [i32]
     L.ssd_strerror.restype = ctypes.c_char_p
     _LIB = L
@@ -112,6 +114,12 @@ def _p(t: Optional[torch.Tensor]):
 
 def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def device_buffer(nbytes: int) -> torch.Tensor:
+    """Every device block this binding hands to the library (descriptor table, cache slab, workspace) comes
+    from here: uint8, 256-byte aligned.  Tests replace it to put guard bands around the blocks."""
+    return torch.empty(max(int(nbytes), 1), dtype=torch.uint8, device="cuda")
 
 
 def arch_struct(arch) -> SsdArch:
@@ -147,7 +155,7 @@ class Model:
         h = ctypes.c_void_p()
         a = arch_struct(arch)
         nd = int(L.ssd_model_desc_bytes(ctypes.byref(a)))
-        self.desc = torch.empty(max(nd, 1), dtype=torch.uint8, device="cuda") if nd else None
+        self.desc = device_buffer(nd) if nd else None
         _check(L.ssd_model_create(ctypes.byref(a), ptrs, n, _p(self.desc), nd, ctypes.byref(h)), "ssd_model_create")
         self.h = h
 
@@ -168,7 +176,7 @@ class Model:
         n = self.workspace_bytes(batch, rows_per_seq, max_len)
         if n == 0:
             raise SsdError(-3, "ssd_workspace_bytes")
-        return torch.empty(n, dtype=torch.uint8, device="cuda")
+        return device_buffer(n)
 
     def __del__(self):
         try:
@@ -185,7 +193,7 @@ class KV:
     def __init__(self, model: Model, batch: int, max_len: int):
         self.model, self.batch, self.max_len = model, batch, max_len
         n = model.kv_bytes(batch, max_len)
-        self.buf = torch.empty(n, dtype=torch.uint8, device="cuda")
+        self.buf = device_buffer(n)
         h = ctypes.c_void_p()
         _check(load().kv_init(model.h, batch, max_len, _p(self.buf), n, _stream(), ctypes.byref(h)), "kv_init")
         self.h = h
@@ -322,6 +330,17 @@ def read_trace(model: Model, batch: int, rows_per_seq: int, ws: torch.Tensor) ->
     _check(load().ssd_read_trace(model.h, batch, rows_per_seq, _p(ws), ws.numel(), out.ctypes.data_as(ctypes.c_void_p),
                                  1024, ctypes.byref(n), _stream()), "ssd_read_trace")
     return out[:n.value]
+
+
+def set_wait_limit(cycles: int) -> None:
+    """Bound (GPU clock cycles) of every device-side wait that takes work; 0 restores the default (~2 s)."""
+    _check(load().ssd_set_wait_limit(int(cycles)), "ssd_set_wait_limit")
+
+
+def wait_probe(kv: KV) -> None:
+    """Queue the failure-detection probe: a wait on a barrier nobody arrives at; it runs out after the
+    configured bound and leaves SSD_E_TIMEOUT in the cache's status word."""
+    _check(load().ssd_wait_probe(kv.h, _stream()), "ssd_wait_probe")
 
 
 def launch_count() -> int:

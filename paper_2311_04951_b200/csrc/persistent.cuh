@@ -120,6 +120,7 @@ struct alignas(64) FwdParams {
     int kv_rows_per_layer;   // B * 2 * H * S
     int attn_ctas;           // min(attention items, CTAs): set by the host together with the split plan
     int overlap_out;         // parallel-residual block and at most half of the CTAs on attention
+    long long wait_cycles;   // bound of every wait that takes work (see Shared::wait_limit)
 };
 
 struct GemmDesc {
@@ -344,6 +345,7 @@ struct alignas(16) Shared {
     volatile int abort;     // some wait in this CTA gave up
     volatile int go;        // snapshot of !abort taken inside the grid barrier: uniform for all work threads
     int flag;
+    long long wait_limit;   // cycles after which a wait that takes work gives up (the drain waits of the error path keep kWaitCycles)
     // for the tensor-core attention items (kept here so that they take no more arguments than the others):
     uint32_t tmem_base;     // base address of this CTA's tensor memory
     uint32_t attn_bar_off;  // byte offset from this block to the attention barriers, followed by their counts
@@ -364,7 +366,7 @@ __device__ __forceinline__ bool mbar_wait_or_abort(uint64_t *bar, uint32_t parit
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (sh->abort || clock64() - t0 > kWaitCycles) return false;
+        if (sh->abort || clock64() - t0 > sh->wait_limit) return false;
     }
     return true;
 }
@@ -374,7 +376,7 @@ __device__ __forceinline__ bool mbar_spin_or_abort(uint64_t *bar, uint32_t parit
     if (mbar_test_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_test_wait(bar, parity)) {
-        if (sh->abort || clock64() - t0 > kWaitCycles) return false;
+        if (sh->abort || clock64() - t0 > sh->wait_limit) return false;
     }
     return true;
 }
@@ -394,7 +396,7 @@ __device__ __forceinline__ bool grid_sync(const FwdParams &p, Shared *sh, int &e
             if (ld_acquire(p.gbar) < target) {
                 const long long t0 = clock64();
                 while (ld_acquire(p.gbar) < target) {
-                    if (clock64() - t0 > kWaitCycles) { ok = false; break; }
+                    if (clock64() - t0 > sh->wait_limit) { ok = false; break; }
                 }
             }
         }
@@ -773,6 +775,15 @@ __device__ __forceinline__ void merge_splits(const FwdParams &p, int r0, int h, 
             }
 }
 
+// Positions per split of a sequence that holds `total` positions after this pass: equal shares of whole
+// tiles, taken on the device from the sequence's own length.  The host fixes only the number of splits
+// (from an upper bound of the lengths), so ragged sequences are each cut evenly and a loose bound costs
+// nothing but an empty split.
+__device__ __forceinline__ int split_chunk(const FwdParams &p, int total, int tile) {
+    const int c = (max(total, 1) + p.n_split - 1) / p.n_split;
+    return (c + tile - 1) / tile * tile;
+}
+
 constexpr int kAttnRows = 16;  // query rows per item (one MMA row tile)
 constexpr int kAttnBufs = 3;   // K/V chunk buffers: two chunks (64 KB at head 128) in flight per SM
 __host__ __device__ inline size_t attn_scratch_bytes(int Dh) {
@@ -816,8 +827,9 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
     const int n_rows = staged_len(sh)[64 + b];
     const int len = staged_len(sh)[b];
     const int r0 = b * p.M, m_base = mt * kAttnRows;
-    const int p_begin = split * p.chunk;
-    const int p_end = min(p_begin + p.chunk, len + n_rows);
+    const int chunk = split_chunk(p, len + n_rows, kAttnTile);
+    const int p_begin = split * chunk;
+    const int p_end = min(p_begin + chunk, len + n_rows);
     const float sc = p.attn_scale * 1.4426950408889634f;  // scores in log2 units
 
     __nv_bfloat16 *kc = (__nv_bfloat16 *)(p.cache + (size_t)layer * p.layer_bytes) + ((size_t)(b * 2) * p.H + h) * p.S * Dh;
@@ -1232,8 +1244,9 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
     const int len = staged_len(sh)[b];
     const int r0 = b * p.M, m_base = mt * kAttnRows;
     const int rows_here = max(0, min(kAttnRows, p.M - m_base));
-    const int p_begin = split * p.chunk;
-    const int p_end = min(p_begin + p.chunk, len + n_rows);
+    const int chunk = split_chunk(p, len + n_rows, kTcChunk);
+    const int p_begin = split * chunk;
+    const int p_end = min(p_begin + chunk, len + n_rows);
     const int n_chunks = p_begin < p_end ? (p_end - p_begin + kTcChunk - 1) / kTcChunk : 0;
     const float sc = p.attn_scale * 1.4426950408889634f;  // scores in log2 units
     const uint32_t tS = tmem_base, tO = tmem_base + 64;  // scores of chunk c at tS + 32 (c & 1)
@@ -1711,7 +1724,7 @@ __device__ __noinline__ void run_gemm(const FwdParams &p, int gi, uint8_t *smem)
                     if (ld_acquire(cnt) < g.wait_attn) {
                         const long long t0 = clock64();
                         while (ld_acquire(cnt) < g.wait_attn) {
-                            if (sh->abort || clock64() - t0 > kWaitCycles) { ready = false; break; }
+                            if (sh->abort || clock64() - t0 > sh->wait_limit) { ready = false; break; }
                         }
                     }
                     if (!ready) {
@@ -1875,6 +1888,7 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
         sh->released = 0;
         sh->abort = 0;
         sh->go = 1;
+        sh->wait_limit = kp.wait_cycles > 0 ? kp.wait_cycles : kWaitCycles;
         sh->attn_bar_off = (uint32_t)((uint8_t *)abar - (uint8_t *)sh);
         sh->seq_off = (uint32_t)((uint8_t *)seq_tab - (uint8_t *)sh);
         sh->ltab_off = kp.n_layers <= kMaxStagedLayers ? (uint32_t)((uint8_t *)ltab - (uint8_t *)sh) : 0u;
@@ -1911,14 +1925,14 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                     if (s >= S1 && scratch_used && seen_release < dw.need_hi) {  // slot shared with the attention scratch
                         const long long t0 = clock64();
                         while ((seen_release = sh->released) < dw.need_hi) {
-                            if (sh->abort || clock64() - t0 > kWaitCycles) { failed = true; break; }
+                            if (sh->abort || clock64() - t0 > sh->wait_limit) { failed = true; break; }
                         }
                         if (failed) { rp.par ^= 1u << s; break; }  // nothing was issued into s
                     }
                     if (!mbar_test_wait(&empty[s], ph ^ 1u)) {
                         const long long t0 = clock64();
                         while (!mbar_test_wait(&empty[s], ph ^ 1u)) {
-                            if (sh->abort || clock64() - t0 > kWaitCycles) { failed = true; break; }
+                            if (sh->abort || clock64() - t0 > sh->wait_limit) { failed = true; break; }
                         }
                         if (failed) { rp.par ^= 1u << s; break; }  // nothing was issued into s
                     }

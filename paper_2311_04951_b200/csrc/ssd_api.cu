@@ -33,6 +33,7 @@ std::mutex g_mu;
 bool g_persistent = true;  // bf16 models: whole forward in one cooperative kernel
 int g_attn_mode = 0;       // 0: choose per pass; 1: warp-MMA attention items; 2: tensor-core items wherever they apply
 bool g_trace = false;       // stamp the global timer after every grid barrier of the forward kernel
+long long g_wait_cycles = 0;  // 0: the kernels' default bound (about two seconds) on every wait that takes work
 bool g_prof = false;
 std::vector<cudaEvent_t> g_prof_events;  // pairs
 size_t g_prof_used = 0;
@@ -174,9 +175,38 @@ struct ssd_kv {
     bool tm_rows_ok;
     int len_ub;   // host-side upper bound of the committed lengths
     int last_rows;  // rows the last forward left uncommitted (upper bound bookkeeping)
+    // The bound follows the device without a synchronisation: every kernel that changes the lengths writes
+    // (operation number << 32 | largest length) into this word of mapped host memory; the host adds what the
+    // operations queued behind that number can add at most (growth_at[n & 255] = total growth bound after op n).
+    unsigned long long *mailbox, *mailbox_dev;
+    unsigned op_seq;
+    long long growth_total;
+    long long growth_at[256];
 };
 
 namespace {
+
+// A length-changing operation is about to be queued: it may add up to `growth` positions to a sequence.
+unsigned kv_note_op(ssd_kv *kv, int growth) {
+    ++kv->op_seq;
+    kv->growth_total += growth;
+    kv->growth_at[kv->op_seq & 255] = kv->growth_total;
+    kv->len_ub += growth;
+    if (kv->len_ub > kv->S) kv->len_ub = kv->S;
+    return kv->op_seq;
+}
+// Upper bound of the committed lengths once everything queued so far has run.
+int kv_bound(ssd_kv *kv) {
+    if (kv->mailbox) {
+        const unsigned long long v = *reinterpret_cast<volatile unsigned long long *>(kv->mailbox);
+        const unsigned seq = (unsigned)(v >> 32);
+        if (seq != 0 && kv->op_seq - seq < 256u) {
+            const long long ub = (long long)(unsigned)(v & 0xffffffffu) + kv->growth_total - kv->growth_at[seq & 255];
+            kv->len_ub = ub > kv->S ? kv->S : (int)ub;
+        }
+    }
+    return kv->len_ub;
+}
 
 enum { T_TOK = 0, T_POS = 1, T_L0 = 2, PER_LAYER = 12 };
 enum { L_LN1G, L_LN1B, L_WQKV, L_BQKV, L_WO, L_BO, L_LN2G, L_LN2B, L_WIN, L_BIN, L_WOUT, L_BOUT };
@@ -409,7 +439,7 @@ int run_attention(const ssd_model *m, ssd_kv *kv, int layer, const float *q, int
     at.cache = kv->cache + (size_t)layer * kv->layer_bytes;
     at.len = kv->len;
     at.M = M; at.H = a.n_heads; at.Dh = a.head_dim; at.S = kv->S; at.d = a.d_model;
-    int ctx = kv->len_ub + M;
+    int ctx = kv_bound(kv) + M;
     if (ctx > kv->S) ctx = kv->S;
     plan_split(kv->B * a.n_heads, ctx, &at.chunk, &at.n_split);
     at.scale = 1.0f / sqrtf((float)a.head_dim);
@@ -449,12 +479,14 @@ int launch_forward_nt(FwdParams p, cudaStream_t st) {
     p.attn_smem_off = (int)(S1 * stage);
     p.bar_off = (int)align_up(S1 * stage + region2, 128);
     const size_t smem = 1024 + (size_t)p.bar_off + tail;
-    static bool attr = false;
-    if (!attr) {
+    static bool attr[64] = {false};  // the attribute belongs to the device's copy of the kernel
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SSD_E_CUDA;
+    if (!attr[dev]) {
         if (cudaFuncSetAttribute(forward_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) !=
             cudaSuccess)
             return SSD_E_CUDA;
-        attr = true;
+        attr[dev] = true;
     }
     void *args[] = {&p};
     if (cudaLaunchCooperativeKernel((void *)forward_kernel<NT>, dim3(g_num_sms), dim3(kPersistThreads), args, smem,
@@ -505,7 +537,7 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     p.x = w.x; p.qkv = w.qkv; p.t_in = w.t_in; p.logits = w.logits;
     p.part_m = w.part_m; p.part_l = w.part_l; p.part_o = w.part_o;
     p.gbar = w.sync; p.tickets = w.sync + 16;
-    int ctx = kv->len_ub + M;
+    int ctx = kv_bound(kv) + M;
     if (ctx > kv->S) ctx = kv->S;
     // Tensor-core attention items stream 128 positions per ~2 us but cost ~8 us more to start than the
     // warp-MMA items (64 positions per ~2 us): they pay off from about a thousand positions per split.
@@ -526,6 +558,7 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
         p.overlap_out = (a.parallel_residual && 2 * p.attn_ctas <= sms) ? 1 : 0;
     }
     p.want_logits = want_logits ? 1 : 0;
+    p.wait_cycles = g_wait_cycles;
     p.trace = (g_trace && 2 + barriers_needed(a) + 3 < kTraceSlots) ? w.trace : nullptr;
     CUDA_OK(cudaMemsetAsync(w.sync, 0, w.sync_bytes, st));
     cudaEvent_t prof_stop;
@@ -773,9 +806,26 @@ int kv_init(const ssd_model *m, int batch, int max_len, void *dev_buf, size_t by
     kv->layer_bytes = (size_t)batch * 2 * m->a.d_model * max_len * kv->esize;
     kv->len_ub = 0;
     kv->last_rows = 0;
+    kv->op_seq = 0;
+    kv->growth_total = 0;
+    memset(kv->growth_at, 0, sizeof(kv->growth_at));
+    kv->mailbox = kv->mailbox_dev = nullptr;
+    {   // eight bytes of mapped host memory (not device memory); without it the bound is only advanced
+        void *h = nullptr, *d = nullptr;
+        if (cudaHostAlloc(&h, sizeof(unsigned long long), cudaHostAllocMapped) == cudaSuccess) {
+            *reinterpret_cast<unsigned long long *>(h) = 0;
+            if (cudaHostGetDevicePointer(&d, h, 0) == cudaSuccess) {
+                kv->mailbox = (unsigned long long *)h;
+                kv->mailbox_dev = (unsigned long long *)d;
+            } else {
+                cudaFreeHost(h);
+            }
+        }
+        (void)cudaGetLastError();
+    }
     // Rows beyond a sequence's length are read (masked) by the chunked attention: they must hold finite numbers.
     if (cudaMemsetAsync(kv->cache, 0, kv->layer_bytes * m->a.n_layers, (cudaStream_t)stream) != cudaSuccess) {
-        delete kv;
+        kv_destroy(kv);
         return SSD_E_CUDA;
     }
     kv->tm_rows_ok = false;
@@ -785,14 +835,21 @@ int kv_init(const ssd_model *m, int batch, int max_len, void *dev_buf, size_t by
             kv->tm_rows_ok = make_map(&kv->tm_rows, kv->cache, (int)rows, 128, kTcChunk) == SSD_OK;
     }
     if (cudaMemsetAsync(dev_buf, 0, kv_header_bytes(batch), (cudaStream_t)stream) != cudaSuccess) {
-        delete kv;
+        kv_destroy(kv);
         return SSD_E_CUDA;
     }
     *out = kv;
     return SSD_OK;
 }
 
-void kv_destroy(ssd_kv *kv) { delete kv; }
+void kv_destroy(ssd_kv *kv) {
+    if (kv && kv->mailbox) {
+        // the word may still be written by queued kernels: wait for the device before it goes away
+        cudaDeviceSynchronize();
+        cudaFreeHost(kv->mailbox);
+    }
+    delete kv;
+}
 
 static bool same_cache_shape(const ssd_model *m, const ssd_kv *kv) {
     return m->a.n_layers == kv->a.n_layers && m->a.d_model == kv->a.d_model && m->a.n_heads == kv->a.n_heads &&
@@ -803,7 +860,7 @@ int kv_prefill(ssd_model *m, ssd_kv *kv, const int32_t *dev_tokens, const int32_
                void *dev_ws, size_t ws_bytes, void *stream) {
     if (!m || !kv || !dev_tokens || !dev_n_tokens || max_tokens < 0) return SSD_E_ARG;
     if (!same_cache_shape(m, kv)) return SSD_E_ARG;
-    if (kv->len_ub + max_tokens > kv->S) return SSD_E_CAPACITY;
+    if (kv_bound(kv) + max_tokens > kv->S) return SSD_E_CAPACITY;
     cudaStream_t st = (cudaStream_t)stream;
     int C = kMaxRows / kv->B;
     if (C > 8) C = 8;
@@ -815,9 +872,8 @@ int kv_prefill(ssd_model *m, ssd_kv *kv, const int32_t *dev_tokens, const int32_
     for (int c = 0; c < chunks; ++c) {
         LAUNCH(prefill_rows_kernel, ceil_div(kv->B, 64), 64, 0, st, dev_n_tokens, c, C, w.n_rows_tmp, kv->B);
         if ((rc = forward(m, kv, dev_tokens + (size_t)c * C, max_tokens, C, w.n_rows_tmp, false, w, st))) return rc;
-        LAUNCH(kv_commit_rows_kernel, ceil_div(kv->B, 64), 64, 0, st, kv->len, w.ri.n_eff, kv->B);
-        kv->len_ub += C;
-        if (kv->len_ub > kv->S) kv->len_ub = kv->S;
+        const unsigned seq = kv_note_op(kv, C);
+        LAUNCH(kv_commit_rows_kernel, 1, 64, 0, st, kv->len, w.ri.n_eff, kv->B, kv->mailbox_dev, seq);
     }
     return SSD_OK;
 }
@@ -840,9 +896,8 @@ int draft_step(ssd_model *draft, ssd_kv *dkv, const int32_t *dev_tokens_in, int 
     t.token_out = dev_token_out; t.token_stride = token_out_stride;
     t.q_out = dev_q_out; t.q_stride = q_stride;
     LAUNCH(draft_tail_kernel, dkv->B * kTailCluster, kTailThreads, 0, st, t);
-    LAUNCH(kv_commit_rows_kernel, ceil_div(dkv->B, 64), 64, 0, st, dkv->len, w.ri.n_eff, dkv->B);
-    dkv->len_ub += rows_in;
-    if (dkv->len_ub > dkv->S) dkv->len_ub = dkv->S;
+    const unsigned seq = kv_note_op(dkv, rows_in);
+    LAUNCH(kv_commit_rows_kernel, 1, 64, 0, st, dkv->len, w.ri.n_eff, dkv->B, dkv->mailbox_dev, seq);
     return SSD_OK;
 }
 
@@ -897,15 +952,16 @@ int target_verify(ssd_model *target, ssd_kv *tkv, const int32_t *dev_rows, int K
 int kv_commit(ssd_kv *kv, const int32_t *dev_n_keep, void *stream) {
     if (!kv) return SSD_E_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    LAUNCH(kv_commit_kernel, ceil_div(kv->B, 64), 64, 0, st, kv->len, dev_n_keep ? dev_n_keep : kv->keep, kv->B);
-    kv->len_ub += kv->last_rows > 0 ? kv->last_rows : 1;
-    if (kv->len_ub > kv->S) kv->len_ub = kv->S;
+    const unsigned seq = kv_note_op(kv, kv->last_rows > 0 ? kv->last_rows : 1);
+    LAUNCH(kv_commit_kernel, 1, 64, 0, st, kv->len, dev_n_keep ? dev_n_keep : kv->keep, kv->B, kv->S, kv->status,
+           kv->mailbox_dev, seq);
     return SSD_OK;
 }
 
 int kv_rollback(ssd_kv *kv, const int32_t *dev_new_len, void *stream) {
     if (!kv || !dev_new_len) return SSD_E_ARG;
-    LAUNCH(kv_rollback_kernel, ceil_div(kv->B, 64), 64, 0, (cudaStream_t)stream, kv->len, dev_new_len, kv->B);
+    const unsigned seq = kv_note_op(kv, 0);
+    LAUNCH(kv_rollback_kernel, 1, 64, 0, (cudaStream_t)stream, kv->len, dev_new_len, kv->B, kv->mailbox_dev, seq);
     return SSD_OK;
 }
 
@@ -920,9 +976,11 @@ int spec_advance(ssd_kv *tkv, ssd_kv *dkv, int32_t *dev_rows, int K, const int32
     a.n_accepted = dev_n_accepted; a.next_token = dev_next_token; a.next_stride = next_token_stride;
     a.out_tokens = dev_out_tokens; a.out_cap = out_cap; a.out_count = dev_out_count;
     a.draft_in = dev_draft_in; a.draft_n_in = dev_draft_n_in;
-    LAUNCH(spec_advance_kernel, ceil_div(tkv->B, 64), 64, 0, (cudaStream_t)stream, a);
-    tkv->len_ub += K + 1;
-    if (tkv->len_ub > tkv->S) tkv->len_ub = tkv->S;
+    a.t_mailbox = tkv->mailbox_dev;
+    a.t_seq = kv_note_op(tkv, K + 1);
+    a.d_mailbox = dkv ? dkv->mailbox_dev : nullptr;
+    a.d_seq = dkv ? kv_note_op(dkv, 0) : 0u;  // the draft cache is only cut back here
+    LAUNCH(spec_advance_kernel, 1, 64, 0, (cudaStream_t)stream, a);
     return SSD_OK;
 }
 
@@ -1021,6 +1079,29 @@ int verify_from_logits_noalloc(const float *dev_logits, int batch, int K, int vo
 }
 
 uint64_t ssd_launch_count(void) { return g_launches.load(); }
+
+int ssd_set_wait_limit(long long cycles) {
+    if (cycles < 0) return SSD_E_ARG;
+    g_wait_cycles = cycles;
+    return SSD_OK;
+}
+
+// One thread waits, through the same bounded-wait helper the other kernels use, on a barrier that nobody
+// arrives at; the wait runs out and the kernel records the time-out and returns.
+__global__ void wait_probe_kernel(int32_t *status, long long limit) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait_limit(&bar, 0, limit)) set_status(status, kTimeoutCode);
+    }
+}
+
+int ssd_wait_probe(ssd_kv *kv, void *stream) {
+    if (!kv) return SSD_E_ARG;
+    LAUNCH(wait_probe_kernel, 1, 32, 0, (cudaStream_t)stream, kv->status, g_wait_cycles > 0 ? g_wait_cycles : kWaitCycles);
+    return SSD_OK;
+}
 
 int ssd_set_trace(int enable) {
     g_trace = enable != 0;

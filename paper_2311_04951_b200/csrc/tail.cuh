@@ -1,7 +1,7 @@
 // Vocabulary-wide tail of a step: temperature softmax statistics, the accept / reject scan,
 // residual renormalise-and-resample or bonus draw, and the draft's "sample from q, export q".
-// (Section "Speculative Sampling", Figure 2: the target "qualifies and accepts (or rejects)" the
-// draft tokens and generates one token itself.)  No host round-trip: everything a decision
+// (Section "Speculative Sampling", Figure 2: the target model passes or refuses each draft token in
+// turn and generates one token itself.)  No host round-trip: everything a decision
 // needs stays on the device; reductions use warp shuffles, prefix sums run in fp64.
 //
 // One row of the vocabulary is worked on by a thread-block cluster of kTailCluster CTAs (one SM alone
@@ -324,17 +324,58 @@ __global__ void __cluster_dims__(kTailCluster, 1, 1) __launch_bounds__(kTailThre
 }
 
 // ---------------- cache length bookkeeping ----------------
-__global__ void kv_commit_kernel(int32_t *len, const int32_t *n_keep, int B) {
-    int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b < B) len[b] += max(0, n_keep[b]);
+// Every kernel that changes the committed lengths runs as ONE block of 64 threads (at most 64 sequences)
+// and afterwards reports the largest length to the host through a word of mapped host memory, tagged with
+// the host's sequence number of the operation: (seq << 32) | max length.  The host plans attention splits
+// from an upper bound of the lengths; with this word the bound follows the real lengths without a
+// synchronisation (it adds what the operations queued behind `seq` can add at most).
+__device__ __forceinline__ void report_max_len(int my_len, unsigned long long *mailbox, unsigned seq) {
+    __shared__ int s_max[2];
+    int v = my_len;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x == 0 && mailbox) {
+        const unsigned m = (unsigned)max(s_max[0], s_max[1]);
+        *reinterpret_cast<volatile unsigned long long *>(mailbox) = ((unsigned long long)seq << 32) | m;
+    }
 }
-__global__ void kv_commit_rows_kernel(int32_t *len, const int32_t *n_eff, int B) {
-    int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b < B) len[b] += n_eff[b];
+// Keep n_keep[b] more rows.  A length that would pass the capacity S is clamped and recorded as
+// SSD_E_CAPACITY in the sticky status word: rows that no forward wrote must not become context.
+__global__ void kv_commit_kernel(int32_t *len, const int32_t *n_keep, int B, int S, int32_t *status,
+                                 unsigned long long *mailbox, unsigned seq) {
+    const int b = threadIdx.x;
+    int v = 0;
+    if (b < B) {
+        v = len[b] + max(0, n_keep[b]);
+        if (v > S) {
+            v = S;
+            set_status(status, -3);
+        }
+        len[b] = v;
+    }
+    report_max_len(v, mailbox, seq);
 }
-__global__ void kv_rollback_kernel(int32_t *len, const int32_t *new_len, int B) {
-    int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b < B) len[b] = max(0, min(len[b], new_len[b]));
+__global__ void kv_commit_rows_kernel(int32_t *len, const int32_t *n_eff, int B, unsigned long long *mailbox,
+                                      unsigned seq) {
+    const int b = threadIdx.x;
+    int v = 0;
+    if (b < B) {
+        v = len[b] + n_eff[b];   // n_eff is what the forward's set-up found to fit
+        len[b] = v;
+    }
+    report_max_len(v, mailbox, seq);
+}
+__global__ void kv_rollback_kernel(int32_t *len, const int32_t *new_len, int B, unsigned long long *mailbox,
+                                   unsigned seq) {
+    const int b = threadIdx.x;
+    int v = 0;
+    if (b < B) {
+        v = max(0, min(len[b], new_len[b]));
+        len[b] = v;
+    }
+    report_max_len(v, mailbox, seq);
 }
 // chunk c of a prompt pass: rows fed per sequence = clamp(n_tokens - c*C, 0, C)
 __global__ void prefill_rows_kernel(const int32_t *n_tokens, int chunk, int C, int32_t *n_rows, int B) {
@@ -350,11 +391,11 @@ struct AdvanceArgs {
     int next_stride;
     int32_t *out_tokens; int out_cap; int32_t *out_count;
     int32_t *draft_in, *draft_n_in;
+    unsigned long long *t_mailbox, *d_mailbox;  // see report_max_len
+    unsigned t_seq, d_seq;
 };
 
-__global__ void spec_advance_kernel(AdvanceArgs a) {
-    const int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= a.B) return;
+__device__ __forceinline__ void spec_advance_one(const AdvanceArgs &a, int b, int &t_new, int &d_new) {
     const int K = a.K;
     int acc = max(0, min(a.n_accepted[b], K));
     const int y = a.next_token[(size_t)b * a.next_stride];
@@ -380,9 +421,21 @@ __global__ void spec_advance_kernel(AdvanceArgs a) {
             a.draft_n_in[b] = 1;
         }
     }
-    a.tlen[b] += acc + 1;
-    if (a.dlen) a.dlen[b] = min(a.dlen[b], K > 0 ? min(n + acc, n + K - 1) : n + acc);
+    t_new = a.tlen[b] + acc + 1;
+    a.tlen[b] = t_new;
+    if (a.dlen) {
+        d_new = min(a.dlen[b], K > 0 ? min(n + acc, n + K - 1) : n + acc);
+        a.dlen[b] = d_new;
+    }
     row[0] = y;
+}
+__global__ void spec_advance_kernel(AdvanceArgs a) {  // one block of 64 threads
+    const int b = threadIdx.x;
+    int t_new = 0, d_new = 0;
+    if (b < a.B) spec_advance_one(a, b, t_new, d_new);
+    report_max_len(t_new, a.t_mailbox, a.t_seq);
+    __syncthreads();  // the exchange slots are reused
+    report_max_len(d_new, a.d_mailbox, a.d_seq);
 }
 
 }  // namespace ssd

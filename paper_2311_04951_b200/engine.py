@@ -28,7 +28,11 @@ class Engine:
         self.tkv = B.KV(target, batch, max_len)
         self.ws_t = target.new_workspace(batch, K + 1, max_len)
         self.rows = torch.zeros(batch, K + 1, dtype=torch.int32, device=dev)
-        self.n_acc = torch.zeros(batch, dtype=torch.int32, device=dev)
+        # accepted counts of the last `log_cap` iterations, one row each: target_verify writes row it % log_cap
+        # (a pointer, not a copy), so acceptance statistics can be read after a run without touching the loop
+        self.log_cap = max(1, out_cap // (K + 1) + 1)
+        self.n_acc_log = torch.zeros(self.log_cap, batch, dtype=torch.int32, device=dev)
+        self.it = 0
         self.next_tok = torch.zeros(batch, dtype=torch.int32, device=dev)
         self.out_cap = out_cap
         self.out_tokens = torch.zeros(batch, out_cap, dtype=torch.int32, device=dev)
@@ -45,6 +49,24 @@ class Engine:
         else:
             self.dkv = None
             self.q = None
+
+    @property
+    def n_acc(self) -> torch.Tensor:
+        """int32 [batch]: where the current iteration's accepted counts are written and read."""
+        return self.n_acc_log[self.it % self.log_cap]
+
+    def refresh_bounds(self) -> None:
+        """Make the host-side length bounds (from which attention splits are planned) exact; synchronises."""
+        self.tkv.lengths()
+        if self.dkv is not None:
+            self.dkv.lengths()
+
+    def copy_cache_from(self, other: "Engine") -> None:
+        """Take over the target cache contents, lengths and pending tokens of an engine of the same shape."""
+        assert self.tkv.buf.numel() == other.tkv.buf.numel() and self.batch == other.batch
+        self.tkv.buf.copy_(other.tkv.buf)
+        self.rows[:, 0] = other.rows[:, 0]
+        self.tkv.lengths()
 
     # ---- prompt pass (functional, untimed) ----
     def prefill(self, prompts: torch.Tensor) -> None:
@@ -80,6 +102,7 @@ class Engine:
         B.spec_advance(self.tkv, self.dkv, self.rows, self.K, self.n_acc, self.next_tok, 1, self.out_tokens,
                        self.out_cap, self.out_count, self.draft_in if self.dkv is not None else None,
                        self.draft_n_in if self.dkv is not None else None)
+        self.it += 1
 
     def ar_step(self, u: torch.Tensor, p_debug: Optional[torch.Tensor] = None) -> None:
         """Plain autoregressive decode step (Eq. 1): one row per sequence, token drawn with u [batch, 1]."""

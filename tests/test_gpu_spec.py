@@ -30,8 +30,8 @@ def test_tiny_config_full_trajectory():
     ref = ospec.speculative_generate(otgt, odrf, prompt[0], n_new, K, T, lambda it: synth.gen_uniforms(su, 0, it, 2 * K + 1),
                                      256, keep_trace=True)
     eng = engine.Engine(tgt, drf, 1, 256, K, T, 128)
-    synced, n = gu.lockstep(eng, synth, prompt[0], ref["iterations"], K, su, ref["trace"])
-    assert synced == n == ref["iterations"]
+    res = gu.lockstep(eng, synth, prompt[0], ref["iterations"], K, su, ref["trace"])
+    assert res["identical"] == res["iterations"] == ref["iterations"] and res["excused"] == 0
     toks = eng.out_tokens.cpu().numpy()[0, :n_new].tolist()
     assert toks == ref["tokens"]
     assert eng.tkv.status() == 0 and eng.dkv.status() == 0
@@ -58,15 +58,22 @@ def test_lockstep_trajectories_per_family(name, arch, scale, K, T):
     ref = ospec.speculative_generate(otgt, odrf, prompt[0], n_new, K, T, lambda it: synth.gen_uniforms(23, 0, it, 2 * K + 1),
                                      160, keep_trace=True)
     eng = engine.Engine(tgt, drf, 1, 160, K, T, 128)
-    synced, n = gu.lockstep(eng, synth, prompt[0], ref["iterations"], K, 23, ref["trace"],
-                            peaky=bool(arch.dtype) and scale > 1.0)
-    assert eng.tkv.status() == 0
+    res = gu.lockstep(eng, synth, prompt[0], ref["iterations"], K, 23, ref["trace"],
+                      peaky=bool(arch.dtype) and scale > 1.0)
+    assert eng.tkv.status() == 0 and eng.dkv.status() == 0
     accepted = sum(t["a"] for t in ref["trace"])
     assert 0 < accepted < K * len(ref["trace"])          # both outcomes occur
+    # every iteration was compared (an excusable difference is followed by a resync to the oracle's tokens):
+    # identical + excused == all, and nothing else passes lockstep's assertions
+    assert res["iterations"] == ref["iterations"] == res["identical"] + res["excused"]
+    print(f"{name}: {res['excused']} excused iteration(s) of {res['iterations']} ({res['decisions']} decisions)")
     if arch.dtype == 0:
-        assert synced == n
+        assert res["excused"] == 0
     else:
-        assert synced >= min(n, 4)                        # bf16: in step until a near-threshold decision
+        assert res["excused"] <= max(2, res["iterations"] // 4)   # near-threshold decisions are rare
+    # the engine's output list is the oracle's token sequence
+    n_out = int(eng.out_count.cpu()[0])
+    assert eng.out_tokens.cpu().numpy()[0, :n_out].tolist() == ref["all_tokens"][len(prompt[0]):]
 
 
 def test_greedy_speculative_equals_greedy_autoregressive_on_gpu():

@@ -44,3 +44,31 @@ def test_single_process_aggregation_is_identity():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.aggregate_replicas(None, [5, 6], [1.5, 2.5], "cpu") == [5, 6, 1.5, 2.5]
+
+
+def test_gpus_flag_spawns_replicas_through_the_launcher():
+    """`python bench.py --gpus 2 ...` with no launcher around it starts two ranks of itself under
+    torch.distributed.run (rendezvous on 127.0.0.1).  On a machine without GPUs the arm that can run is
+    the reference arm (the CPU oracle): rank 0 works and prints the line, rank 1 exits 0 without work, and
+    the line reports the world size the launcher made."""
+    import json
+    import subprocess
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference", "--workload", "tiny",
+           "--steps", "2", "--warmup", "0"]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=600, env=env, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1, out.stdout
+    rec = json.loads(lines[0])
+    assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["value"] > 0
+    assert rec["config"]["workload"] == "tiny" and rec["cpu_baseline"]["kind"] == "oracle"
+
+
+def test_replica_command_is_the_documented_launch_line():
+    sys.path.insert(0, ROOT)
+    import argparse
+    import bench
+    cmd = bench.replica_command(argparse.Namespace(gpus=4), ["--gpus", "4", "--steps", "3"], 29500)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=4" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[-4:] == ["--gpus", "4", "--steps", "3"]
