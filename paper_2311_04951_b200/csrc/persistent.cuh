@@ -425,6 +425,11 @@ __device__ __forceinline__ void grid_arrive(const FwdParams &p, Shared *sh, int 
     named_bar(1, kWorkThreads);
     ++epoch;
     if (threadIdx.x == 0 && sh->abort == 0) red_release_add(p.gbar, 1u);
+    if (p.trace && blockIdx.x == 0 && threadIdx.x == 0) {  // (the stamp of a barrier this CTA does not wait at: its arrival)
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+        p.trace[epoch] = t;
+    }
 }
 
 // Count of attention CTAs that have finished their items, over the layers of this pass (zeroed with the
