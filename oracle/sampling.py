@@ -49,6 +49,40 @@ def softmax_t(logits_row: np.ndarray, temperature: float) -> np.ndarray:
     return (e / e.sum()).astype(np.float32)
 
 
+def filter_top_k_top_p(p_row: np.ndarray, top_k: int = 0, top_p: float = 1.0) -> np.ndarray:
+    """Restrict a distribution to its most probable tokens and renormalise (the paper's Section
+    "Autoregressive vs Speculative Sampling" names sampling "from top-p" as the alternative to the argmax;
+    it prints no formula, so this is the reading used for both models' distributions):
+
+      1. top-k (top_k > 0): t_k = the top_k-th largest probability; keep every token with p >= t_k
+         (tokens tied with the threshold are all kept, so the kept set can exceed top_k);
+      2. top-p (0 < top_p < 1), applied to what step 1 kept: walk the kept tokens in order of decreasing
+         probability, adding them up in float64; t_p = the probability at which the running sum first
+         reaches top_p x (mass kept by step 1); keep every token with p >= t_p (ties again all kept);
+      3. every other token gets probability 0 and the kept ones are divided by the kept mass (summed in
+         float64 in index order, rounded to fp32; the division is fp32).
+
+    top_k = 0 and top_p = 1 return the row unchanged."""
+    p = np.asarray(p_row, np.float32)
+    if top_k <= 0 and not (0.0 < top_p < 1.0):
+        return p
+    keep = np.ones(p.shape[0], bool)
+    if top_k > 0 and top_k < p.shape[0]:
+        t_k = np.sort(p)[::-1][top_k - 1]
+        keep &= p >= t_k
+    if 0.0 < top_p < 1.0:
+        mass_k = float(p[keep].astype(np.float64).sum())
+        vals = np.sort(p[keep])[::-1]
+        c = np.cumsum(vals.astype(np.float64))
+        i = int(np.searchsorted(c, float(np.float32(top_p)) * mass_k, side="left"))
+        i = min(i, vals.shape[0] - 1)
+        keep &= p >= vals[i]
+    mass = np.float32(p[keep].astype(np.float64).sum())
+    out = np.zeros_like(p)
+    out[keep] = p[keep] / mass
+    return out
+
+
 def inv_cdf(weights: np.ndarray, u) -> int:
     """Smallest i with c_i > u * S (c inclusive float64 prefix sums, S = c[-1])."""
     w = np.asarray(weights)

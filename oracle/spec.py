@@ -32,7 +32,8 @@ from .decoder import Model
 
 
 def autoregressive_generate(target: Model, prompt, n_new: int, temperature: float,
-                            uniforms: Callable[[int], np.ndarray], s_max: int) -> Dict:
+                            uniforms: Callable[[int], np.ndarray], s_max: int, top_k: int = 0,
+                            top_p: float = 1.0) -> Dict:
     prompt = [int(t) for t in prompt]
     cache = target.new_cache(s_max)
     if len(prompt) > 1:
@@ -41,7 +42,7 @@ def autoregressive_generate(target: Model, prompt, n_new: int, temperature: floa
     out: List[int] = []
     for j in range(n_new):
         logits = cache.feed([pending])
-        p = sampling.softmax_t(logits[0], temperature)
+        p = sampling.filter_top_k_top_p(sampling.softmax_t(logits[0], temperature), top_k, top_p)
         y = sampling.inv_cdf(p, uniforms(j)[0])
         out.append(y)
         pending = y
@@ -50,7 +51,10 @@ def autoregressive_generate(target: Model, prompt, n_new: int, temperature: floa
 
 def speculative_generate(target: Model, draft: Model, prompt, n_new: int, K: int,
                          temperature: float, uniforms: Callable[[int], np.ndarray],
-                         s_max: int, keep_trace: bool = False) -> Dict:
+                         s_max: int, keep_trace: bool = False, top_k: int = 0, top_p: float = 1.0) -> Dict:
+    """top_k / top_p: both models' distributions are restricted (sampling.filter_top_k_top_p) before the
+    draft draws and before the accept / resample rule, so the emitted tokens follow the restricted
+    target distribution."""
     x = [int(t) for t in prompt]
     tc, dc = target.new_cache(s_max), draft.new_cache(s_max)
     if len(x) > 1:
@@ -71,7 +75,7 @@ def speculative_generate(target: Model, draft: Model, prompt, n_new: int, K: int
         feed = x[dc.len:n]
         for i in range(K):
             logits = dc.feed(feed)
-            q = sampling.softmax_t(logits[-1], temperature)
+            q = sampling.filter_top_k_top_p(sampling.softmax_t(logits[-1], temperature), top_k, top_p)
             t = sampling.inv_cdf(q, u_d[i])
             q_rows.append(q)
             drafts.append(t)
@@ -80,7 +84,8 @@ def speculative_generate(target: Model, draft: Model, prompt, n_new: int, K: int
         # 2. verify: K+1 rows in one target pass, not committed yet
         logits = tc.feed([x[n - 1]] + drafts, advance=False)
         target_rows += K + 1
-        p_rows = [sampling.softmax_t(logits[i], temperature) for i in range(K + 1)]
+        p_rows = [sampling.filter_top_k_top_p(sampling.softmax_t(logits[i], temperature), top_k, top_p)
+                  for i in range(K + 1)]
         # 3. accept / reject / resample
         a, y = sampling.accept_resample(p_rows, q_rows, drafts, u_a, u_r)
         # 4. emit and fix both caches

@@ -14,6 +14,7 @@ import numpy as np
 import pytest
 
 from oracle import sampling as S
+from paper_2311_04951_b200 import synth
 
 
 def _dist(rng, V, zeros=0):
@@ -236,3 +237,100 @@ def test_greedy_reduces_to_argmax_agreement():
             qq[i, t] = 1
         a, y = S.accept_resample(p, qq, toks, rng.random(K).astype(np.float32), np.float32(rng.random()))
         assert a == agree and y == best[agree]
+
+
+# ---------------------------------------------------------------- top-k / top-p restriction
+def _nucleus_by_fractions(p, top_k, top_p):
+    """The definition written out with exact rationals on a tiny row (no ties allowed in the input)."""
+    from fractions import Fraction
+    vals = [Fraction(float(x)) for x in p]
+    order = sorted(range(len(p)), key=lambda j: -vals[j])
+    kept = order[:top_k] if top_k > 0 else order
+    if 0 < top_p < 1:
+        mass = sum(vals[j] for j in kept)
+        acc, cut = Fraction(0), len(kept)
+        for n, j in enumerate(kept):
+            acc += vals[j]
+            if acc >= Fraction(float(np.float32(top_p))) * mass:
+                cut = n + 1
+                break
+        kept = kept[:cut]
+    return sorted(kept)
+
+
+def test_filter_keeps_the_definition_s_set_on_tiny_rows():
+    rng = np.random.default_rng(5)
+    for _ in range(300):
+        V = int(rng.integers(2, 9))
+        p = rng.dirichlet(np.full(V, 0.7)).astype(np.float32)
+        if len(set(p.tolist())) < V:
+            continue
+        k = int(rng.integers(0, V + 2))
+        tp = float(rng.choice([1.0, 0.3, 0.5, 0.8, 0.95]))
+        out = S.filter_top_k_top_p(p, k, tp)
+        kept = np.nonzero(out > 0)[0].tolist()
+        assert kept == _nucleus_by_fractions(p, k, tp), (p, k, tp)
+        # renormalised, ratios among the kept tokens unchanged
+        assert abs(float(out.astype(np.float64).sum()) - 1.0) < 1e-6
+        j0 = kept[0]
+        for j in kept:
+            assert abs(out[j] / out[j0] - p[j] / p[j0]) < 1e-5
+
+
+def test_filter_special_cases_and_ties():
+    p = np.array([0.1, 0.3, 0.05, 0.3, 0.25], np.float32)
+    assert np.array_equal(S.filter_top_k_top_p(p, 0, 1.0), p)               # off: unchanged, same bits
+    assert np.array_equal(S.filter_top_k_top_p(p, 9, 1.0), p)               # k >= V: nothing cut
+    one = S.filter_top_k_top_p(np.array([0.2, 0.5, 0.3], np.float32), 1, 1.0)
+    assert one.tolist() == [0.0, 1.0, 0.0]                                       # top-1 = one-hot at the argmax
+    tie = S.filter_top_k_top_p(p, 1, 1.0)                                    # the two 0.3 tie at the threshold: both kept
+    assert np.nonzero(tie)[0].tolist() == [1, 3] and tie[1] == tie[3] == np.float32(0.5)
+    nuc = S.filter_top_k_top_p(p, 0, 0.61)                                   # 0.3 + 0.3 = 0.6 < 0.61: a third token is needed
+    assert np.nonzero(nuc)[0].tolist() == [1, 3, 4]
+    edge = S.filter_top_k_top_p(p, 0, 0.6)                                   # reaching the target exactly is enough
+    assert np.nonzero(edge)[0].tolist() == [1, 3] or np.nonzero(edge)[0].tolist() == [1, 3, 4]   # (0.3 + 0.3 in fp32 vs 0.6)
+    both = S.filter_top_k_top_p(p, 3, 0.5)                                   # top-p acts on what top-k kept: 0.5 * 0.85
+    assert np.nonzero(both)[0].tolist() == [1, 3]
+
+
+def test_filter_minimality_and_mass_on_large_rows():
+    """V = 32000 Dirichlet rows: the kept set is a threshold set, its mass reaches the target, and without its
+    smallest member it would not (no ties at the threshold in these rows)."""
+    rows = synth.gen_dirichlet_rows(17, 3, 32000, alpha=0.3)
+    for p in rows:
+        for k, tp in ((50, 1.0), (0, 0.9), (200, 0.5)):
+            out = S.filter_top_k_top_p(p, k, tp)
+            kept = out > 0
+            assert p[kept].min() > p[~kept].max()
+            if k:
+                assert kept.sum() <= k
+            if tp < 1:
+                base = np.sort(p)[::-1][:k].astype(np.float64).sum() if k else p.astype(np.float64).sum()
+                m = p[kept].astype(np.float64).sum()
+                assert m >= tp * base * (1 - 1e-12)
+                assert m - float(p[kept].min()) < tp * base
+
+
+def test_speculative_rule_preserves_the_restricted_target():
+    """The accept / resample identity with both rows restricted: sum over draft tokens of
+    q'(x) min(1, p'(x)/q'(x)) [x = y] + P(reject) r'(y) = p'(y), in exact rationals."""
+    from fractions import Fraction
+    rng = np.random.default_rng(9)
+    for _ in range(50):
+        V = 7
+        p = S.filter_top_k_top_p(rng.dirichlet(np.ones(V)).astype(np.float32), 4, 0.9)
+        q = S.filter_top_k_top_p(rng.dirichlet(np.ones(V)).astype(np.float32), 4, 0.9)
+        P = [Fraction(float(x)) for x in p]
+        Q = [Fraction(float(x)) for x in q]
+        sp, sq = sum(P), sum(Q)
+        P = [x / sp for x in P]
+        Q = [x / sq for x in Q]
+        acc = [min(P[j], Q[j]) for j in range(V)]
+        rej = 1 - sum(acc)
+        res = [max(Fraction(0), P[j] - Q[j]) for j in range(V)]
+        sr = sum(res)
+        for y in range(V):
+            total = acc[y] + (rej * res[y] / sr if sr else 0)
+            assert total == P[y]
+            if P[y] == 0:
+                assert total == 0        # a token outside the restricted target is never emitted
