@@ -213,6 +213,21 @@ int spec_advance(ssd_kv *tkv, ssd_kv *dkv, int32_t *dev_rows, int K, const int32
                  const int32_t *dev_next_token, int next_token_stride, int32_t *dev_out_tokens, int out_cap,
                  int32_t *dev_out_count, int32_t *dev_draft_in, int32_t *dev_draft_n_in, void *stream);
 
+/*
+ * Restrict sampling to the most probable tokens (Section "Autoregressive vs Speculative Sampling" names
+ * sampling "from top-p" beside the argmax; the paper gives no formula, the reading is): for every row of both
+ * models, after softmax(logits / T), (1) top_k > 0: t = the top_k-th largest probability, tokens with p >= t
+ * stay (ties with t all stay); (2) 0 < top_p < 1, on what (1) kept: t = the probability at which the running
+ * sum over tokens of decreasing probability first reaches top_p x (mass kept by (1)), tokens with p >= t stay;
+ * (3) the others get 0 and the kept ones are divided by their mass.  draft_step then exports and samples the
+ * restricted q, target_verify / verify_from_logits apply the accept / resample rule to the restricted p (and
+ * expect q restricted the same way), so the emitted tokens follow the restricted target distribution.
+ * top_k = 0 and top_p = 1 (the default) switch it off; greedy rows (temperature 0) are unaffected.  Applies to
+ * the calls queued afterwards; verify_from_logits_noalloc returns SSD_E_UNIMPL while a restriction is set.
+ * SSD_E_ARG for top_k < 0 or top_p outside (0, 1].
+ */
+int ssd_set_sampling(int top_k, float top_p);
+
 /* Copy the committed lengths to the host (synchronises the stream). */
 int kv_lengths(ssd_kv *kv, int32_t *host_out, void *stream);
 

@@ -38,7 +38,7 @@ EXPORTS = ["ssd_model_create", "ssd_model_desc_bytes", "ssd_set_persistent", "ss
            "ssd_workspace_bytes", "kv_init", "kv_destroy", "kv_prefill", "draft_step", "target_verify",
            "kv_commit", "kv_rollback", "spec_advance", "kv_lengths", "ssd_device_status",
            "verify_from_logits", "verify_from_logits_noalloc", "verify_scratch_bytes", "attention_rows", "ssd_last_logits", "ssd_set_trace", "ssd_read_trace", "ssd_launch_count",
-           "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror", "ssd_set_wait_limit", "ssd_wait_probe"]
+           "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror", "ssd_set_wait_limit", "ssd_wait_probe", "ssd_set_sampling"]
 
 
 def lib_path() -> str:
@@ -91,6 +91,7 @@ def load():
     L.ssd_launch_count.restype = ctypes.c_uint64
     L.ssd_gemm_profile.argtypes = [i32]
     L.ssd_gemm_profile_read.argtypes = [ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_double), i32]
+    L.ssd_set_sampling.argtypes = [i32, f32]
     L.ssd_set_wait_limit.argtypes = [ctypes.c_longlong]
     L.ssd_wait_probe.argtypes = [vp, vp]
     L.ssd_strerror.argtypes = [i32]
@@ -330,6 +331,12 @@ def read_trace(model: Model, batch: int, rows_per_seq: int, ws: torch.Tensor) ->
     _check(load().ssd_read_trace(model.h, batch, rows_per_seq, _p(ws), ws.numel(), out.ctypes.data_as(ctypes.c_void_p),
                                  1024, ctypes.byref(n), _stream()), "ssd_read_trace")
     return out[:n.value]
+
+
+def set_sampling(top_k: int = 0, top_p: float = 1.0) -> None:
+    """Restrict both models' distributions to the top_k most probable tokens and / or the top_p nucleus
+    (0 and 1.0 switch the restriction off)."""
+    _check(load().ssd_set_sampling(int(top_k), float(top_p)), "ssd_set_sampling")
 
 
 def set_wait_limit(cycles: int) -> None:

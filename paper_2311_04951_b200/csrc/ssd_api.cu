@@ -33,6 +33,8 @@ std::mutex g_mu;
 bool g_persistent = true;  // bf16 models: whole forward in one cooperative kernel
 int g_attn_mode = 0;       // 0: choose per pass; 1: warp-MMA attention items; 2: tensor-core items wherever they apply
 bool g_trace = false;       // stamp the global timer after every grid barrier of the forward kernel
+int g_top_k = 0;           // restriction of both models' distributions before sampling / verification (0: none)
+float g_top_p = 1.0f;      // (1: none)
 long long g_wait_cycles = 0;  // 0: the kernels' default bound (about two seconds) on every wait that takes work
 bool g_prof = false;
 std::vector<cudaEvent_t> g_prof_events;  // pairs
@@ -251,6 +253,7 @@ struct Workspace {
     int32_t *n_rows_tmp;
     float *x, *qkv, *qrot, *t_in, *logits;
     RowStat *stats;
+    RowFilter *filt;
     Operand xn1, xn2, ao, act;
     float *part_m, *part_l, *part_o;
     int max_split;
@@ -296,6 +299,7 @@ Workspace carve(const ssd_model *m, int B, int M, uint8_t *base) {
     w.trace = (unsigned long long *)take(sizeof(unsigned long long) * kTraceSlots);
     w.logits = (float *)take(sizeof(float) * (size_t)R * a.vocab);
     w.stats = (RowStat *)take(sizeof(RowStat) * R);
+    w.filt = (RowFilter *)take(sizeof(RowFilter) * R);
     // GEMM operands: hi rows [0, rows) then lo rows [rows, 2 rows) in one buffer; the stepwise path
     // pads rows to Rp, the single-kernel path to Rk (one allocation of 2 * Rk rows serves both)
     auto operand = [&](int ld, bool needed) {
@@ -895,6 +899,7 @@ int draft_step(ssd_model *draft, ssd_kv *dkv, const int32_t *dev_tokens_in, int 
     t.u = dev_u; t.u_stride = u_stride;
     t.token_out = dev_token_out; t.token_stride = token_out_stride;
     t.q_out = dev_q_out; t.q_stride = q_stride;
+    t.top_k = g_top_k; t.top_p = g_top_p;
     LAUNCH(draft_tail_kernel, dkv->B * kTailCluster, kTailThreads, 0, st, t);
     const unsigned seq = kv_note_op(dkv, rows_in);
     LAUNCH(kv_commit_rows_kernel, 1, 64, 0, st, dkv->len, w.ri.n_eff, dkv->B, dkv->mailbox_dev, seq);
@@ -903,17 +908,18 @@ int draft_step(ssd_model *draft, ssd_kv *dkv, const int32_t *dev_tokens_in, int 
 
 size_t verify_scratch_bytes(int batch, int K) {
     if (batch < 1 || K < 0) return 0;
-    return align_up(sizeof(RowStat) * (size_t)batch * (K + 1), 256);
+    return align_up(sizeof(RowStat) * (size_t)batch * (K + 1), 256) + align_up(sizeof(RowFilter) * (size_t)batch * (K + 1), 256);
 }
 
 static int run_verify_tail(const float *logits, int B, int K, int V, const int32_t *rows, const float *q,
                            const float *u, float temperature, int32_t *n_acc, int32_t *next, int next_stride,
-                           float *p_debug, int32_t *keep, RowStat *stats, cudaStream_t st) {
+                           float *p_debug, int32_t *keep, RowStat *stats, RowFilter *filt, cudaStream_t st) {
     VerifyArgs v;
     v.logits = logits; v.K = K; v.V = V; v.rows = rows; v.q = q; v.u = u;
     v.inv_t = temperature > 0.f ? 1.0f / temperature : 0.f;
     v.n_accepted = n_acc; v.next_token = next; v.next_stride = next_stride;
     v.p_debug = p_debug; v.keep = keep; v.stats = stats;
+    v.filt = filt; v.top_k = filt ? g_top_k : 0; v.top_p = filt ? g_top_p : 1.0f;
     LAUNCH(row_stats_kernel, dim3((K + 1) * kTailCluster, B), kTailThreads, 0, st, v);
     LAUNCH(verify_kernel, B * kTailCluster, kTailThreads, 0, st, v);
     return SSD_OK;
@@ -930,6 +936,7 @@ int verify_from_logits(const float *dev_logits, int batch, int K, int vocab, con
     if (scratch_bytes < verify_scratch_bytes(batch, K)) return SSD_E_CAPACITY;
     return run_verify_tail(dev_logits, batch, K, vocab, dev_rows, dev_q, dev_u, temperature, dev_n_accepted,
                            dev_next_token, next_token_stride, dev_p_debug, nullptr, (RowStat *)dev_scratch,
+                           (RowFilter *)((uint8_t *)dev_scratch + align_up(sizeof(RowStat) * (size_t)batch * (K + 1), 256)),
                            (cudaStream_t)stream);
 }
 
@@ -946,7 +953,7 @@ int target_verify(ssd_model *target, ssd_kv *tkv, const int32_t *dev_rows, int K
     if (rc) return rc;
     if ((rc = forward(target, tkv, dev_rows, K + 1, K + 1, nullptr, true, w, st))) return rc;
     return run_verify_tail(w.logits, tkv->B, K, target->a.vocab, dev_rows, dev_q, dev_u, temperature, dev_n_accepted,
-                           dev_next_token, next_token_stride, dev_p_debug, tkv->keep, w.stats, st);
+                           dev_next_token, next_token_stride, dev_p_debug, tkv->keep, w.stats, w.filt, st);
 }
 
 int kv_commit(ssd_kv *kv, const int32_t *dev_n_keep, void *stream) {
@@ -1069,16 +1076,24 @@ int verify_from_logits_noalloc(const float *dev_logits, int batch, int K, int vo
         return SSD_E_ARG;
     if (K > 0 && !dev_q) return SSD_E_ARG;
     if ((long long)batch * (K + 1) > SSD_NOALLOC_MAX_ROWS) return SSD_E_CAPACITY;
+    if (g_top_k > 0 || (g_top_p > 0.f && g_top_p < 1.f)) return SSD_E_UNIMPL;  // its fixed array has no room for the restriction
     RowStat *stats = nullptr;
     int rc = noalloc_scratch(&stats);
     if (rc) return rc;
     // every entry a call reads is written earlier in the same call (row_stats_kernel fills
     // stats[0 .. batch*(K+1)) before verify_kernel looks at them): nothing has to start at zero
     return run_verify_tail(dev_logits, batch, K, vocab, dev_rows, dev_q, dev_u, temperature, dev_n_accepted,
-                           dev_next_token, next_token_stride, dev_p_debug, nullptr, stats, (cudaStream_t)stream);
+                           dev_next_token, next_token_stride, dev_p_debug, nullptr, stats, nullptr, (cudaStream_t)stream);
 }
 
 uint64_t ssd_launch_count(void) { return g_launches.load(); }
+
+int ssd_set_sampling(int top_k, float top_p) {
+    if (top_k < 0 || !(top_p > 0.f) || top_p > 1.f) return SSD_E_ARG;
+    g_top_k = top_k;
+    g_top_p = top_p;
+    return SSD_OK;
+}
 
 int ssd_set_wait_limit(long long cycles) {
     if (cycles < 0) return SSD_E_ARG;

@@ -50,6 +50,18 @@ __device__ __forceinline__ float prob_of(float logit, const RowStat &st, float i
     return expf((logit - st.mx) * inv_t) / st.z;
 }
 
+// Restriction of a row to its most probable tokens (top-k, then top-p on what top-k kept): token j stays iff
+// its probability is >= thr, and the kept ones are divided by their mass.  mass == 0 means "no restriction".
+struct RowFilter {
+    float thr;
+    float mass;
+};
+__device__ __forceinline__ float prob_f(float logit, const RowStat &st, const RowFilter &f, float inv_t, int j) {
+    const float pr = prob_of(logit, st, inv_t, j);
+    if (f.mass == 0.f || inv_t == 0.f) return pr;  // (a one-hot row is its own restriction)
+    return pr >= f.thr ? pr / f.mass : 0.f;
+}
+
 // Block-wide (max, lowest index of max).
 __device__ __forceinline__ void block_argmax(float v, int idx, float *sv, int *si, float &out_v, int &out_i) {
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
@@ -133,6 +145,115 @@ __device__ __forceinline__ RowStat row_stats(const float *logits, int V, float i
     st.z = (float)z;
     st.pad = 0;
     return st;
+}
+
+// Shared memory of the threshold search below.
+struct FilterSmem {
+    unsigned cnt[256];
+    double mass[256];
+    unsigned tot_cnt[256];
+    double tot_mass[256];
+    unsigned sel, cnt_above;
+    double mass_above, total;
+};
+
+// The threshold of a restriction, by the whole cluster: the largest probability value t such that the tokens
+// with p >= t (p >= lo only are looked at) number at least want_cnt (by_mass false) or weigh at least want_mass
+// (by_mass true); if no t reaches it, the smallest value present.  Tokens equal to the threshold all stay.  A
+// radix search over the fp32 bit pattern (probabilities are >= 0, so the patterns order like the values): four
+// passes of eight bits, each a 256-bin histogram of counts and masses of the tokens that match the bits fixed
+// so far, summed over the CTAs in rank order through distributed shared memory; the bins are walked from the
+// top.  Returns the threshold and, through *kept_mass, the mass at or above it (fp64 sums; the walk order
+// differs from a sorted running sum only in rounding).  The same result in every thread of the cluster.
+template <typename ProbFn>
+__device__ __forceinline__ float select_threshold(ProbFn prob, int V, float lo, bool by_mass, unsigned want_cnt,
+                                                  double want_frac, FilterSmem *fs, cg::cluster_group &cl,
+                                                  double *kept_mass) {
+    const int rank = (int)cl.block_rank();
+    int lo_i, hi_i;
+    tail_slice(V, rank, lo_i, hi_i);
+    unsigned prefix = 0;
+    int nb = 0;
+    double want_mass = 0.0;
+    if (threadIdx.x == 0) { fs->cnt_above = 0; fs->mass_above = 0.0; }
+    for (int pass = 0; pass < 4; ++pass) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) { fs->cnt[i] = 0; fs->mass[i] = 0.0; }
+        __syncthreads();
+        for (int j = lo_i + threadIdx.x; j < hi_i; j += blockDim.x) {
+            const float pr = prob(j);
+            const unsigned bits = __float_as_uint(pr);
+            if (pr >= lo && (nb == 0 || (bits >> (32 - nb)) == prefix)) {
+                const unsigned bin = (bits >> (24 - nb)) & 255u;
+                atomicAdd(&fs->cnt[bin], 1u);
+                atomicAdd(&fs->mass[bin], (double)pr);
+            }
+        }
+        __syncthreads();
+        cl.sync();  // every CTA's histogram is complete
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) {
+            unsigned c = 0;
+            double m = 0.0;
+            for (int r = 0; r < kTailCluster; ++r) {
+                const FilterSmem *o = cl.map_shared_rank(fs, r);
+                c += o->cnt[i];
+                m += o->mass[i];
+            }
+            fs->tot_cnt[i] = c;
+            fs->tot_mass[i] = m;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            if (pass == 0) {  // the mass of everything looked at: the base of a mass target
+                double t = 0.0;
+                for (int i = 255; i >= 0; --i) t += fs->tot_mass[i];
+                fs->total = t;
+            }
+            const double target = want_frac * fs->total;
+            unsigned c = fs->cnt_above;
+            double m = fs->mass_above;
+            int sel = -1, lowest = -1;
+            for (int i = 255; i >= 0; --i) {
+                if (fs->tot_cnt[i] == 0) continue;
+                lowest = i;
+                const bool met = by_mass ? (m + fs->tot_mass[i] >= target) : (c + fs->tot_cnt[i] >= want_cnt);
+                if (met) { sel = i; break; }
+                c += fs->tot_cnt[i];
+                m += fs->tot_mass[i];
+            }
+            if (sel < 0) {  // the target lies beyond everything there is: keep all (back off the last bin's sums)
+                sel = lowest < 0 ? 0 : lowest;
+                if (lowest >= 0) { c -= fs->tot_cnt[sel]; m -= fs->tot_mass[sel]; }
+            }
+            fs->sel = (unsigned)sel;
+            fs->cnt_above = c;
+            fs->mass_above = m;
+        }
+        __syncthreads();
+        prefix = (prefix << 8) | fs->sel;
+        nb += 8;
+        want_mass = fs->mass_above + fs->tot_mass[fs->sel];
+        cl.sync();  // all remote reads of this pass are done before the histograms are cleared
+    }
+    *kept_mass = want_mass;
+    return __uint_as_float(prefix);
+}
+
+// The restriction of a row (top_k tokens, then the top_p nucleus of those), by the whole cluster.
+__device__ __forceinline__ RowFilter row_filter(const float *logits, int V, const RowStat &st, float inv_t, int top_k,
+                                                float top_p, FilterSmem *fs, cg::cluster_group &cl) {
+    RowFilter f;
+    f.thr = 0.f;
+    f.mass = 0.f;
+    const bool use_k = top_k > 0 && top_k < V, use_p = top_p > 0.f && top_p < 1.f;
+    if (inv_t == 0.f || (!use_k && !use_p)) return f;
+    auto prob = [&](int j) { return prob_of(__ldcg(logits + j), st, inv_t, j); };
+    double mass = 0.0;
+    float thr = 0.f;
+    if (use_k) thr = select_threshold(prob, V, 0.f, false, (unsigned)top_k, 0.0, fs, cl, &mass);
+    if (use_p) thr = select_threshold(prob, V, thr, true, 0u, (double)top_p, fs, cl, &mass);
+    f.thr = thr;
+    f.mass = (float)mass;
+    return f;
 }
 
 // Inverse-CDF draw over V weights w(j) >= 0 by the whole cluster: the smallest j whose inclusive prefix
@@ -222,6 +343,9 @@ struct VerifyArgs {
     float *p_debug;         // [B, K+1, V] or null
     int32_t *keep;          // [B] or null: n_accepted + 1 for kv_commit
     RowStat *stats;         // scratch [B, K+1]
+    RowFilter *filt;        // scratch [B, K+1]
+    int top_k;              // restriction of the target rows (0 / 1.0: none); q arrives already restricted
+    float top_p;
 };
 
 // grid (kTailCluster (K+1), B), one cluster per row: statistics of every row (+ optional export of the p row)
@@ -230,16 +354,21 @@ __global__ void __cluster_dims__(kTailCluster, 1, 1) __launch_bounds__(kTailThre
     __shared__ int si[32];
     __shared__ double sd[32];
     __shared__ ClusterSlots pub;
+    __shared__ FilterSmem fs;
     cg::cluster_group cl = cg::this_cluster();
     const int i = blockIdx.x / kTailCluster, b = blockIdx.y;
     const float *lg = a.logits + ((size_t)b * (a.K + 1) + i) * a.V;
     RowStat st = row_stats(lg, a.V, a.inv_t, sv, si, sd, &pub, cl);
-    if (cl.block_rank() == 0 && threadIdx.x == 0) a.stats[b * (a.K + 1) + i] = st;
+    const RowFilter fl = row_filter(lg, a.V, st, a.inv_t, a.filt ? a.top_k : 0, a.top_p, &fs, cl);  // (no room for it: no restriction)
+    if (cl.block_rank() == 0 && threadIdx.x == 0) {
+        a.stats[b * (a.K + 1) + i] = st;
+        if (a.filt) a.filt[b * (a.K + 1) + i] = fl;
+    }
     if (a.p_debug) {
         int lo, hi;
         tail_slice(a.V, (int)cl.block_rank(), lo, hi);
         float *p = a.p_debug + ((size_t)b * (a.K + 1) + i) * a.V;
-        for (int j = lo + threadIdx.x; j < hi; j += blockDim.x) p[j] = prob_of(lg[j], st, a.inv_t, j);
+        for (int j = lo + threadIdx.x; j < hi; j += blockDim.x) p[j] = prob_f(lg[j], st, fl, a.inv_t, j);
     }
     cl.sync();
 }
@@ -253,12 +382,13 @@ __global__ void __cluster_dims__(kTailCluster, 1, 1) __launch_bounds__(kTailThre
     cg::cluster_group cl = cg::this_cluster();
     const int b = blockIdx.x / kTailCluster, K = a.K, V = a.V;
     const RowStat *st = a.stats + b * (K + 1);
+    const RowFilter none = {0.f, 0.f};
     if (threadIdx.x == 0) {  // (every CTA of the cluster takes the same few steps)
         int acc = 0;
         for (int i = 0; i < K; ++i) {
             int x = a.rows[b * (K + 1) + 1 + i];
             x = max(0, min(x, V - 1));
-            const float px = prob_of(a.logits[((size_t)b * (K + 1) + i) * V + x], st[i], a.inv_t, x);
+            const float px = prob_f(a.logits[((size_t)b * (K + 1) + i) * V + x], st[i], a.filt ? a.filt[b * (K + 1) + i] : none, a.inv_t, x);
             const float qx = a.q[((size_t)b * K + i) * V + x];
             // accept with probability min(1, p/q): u * q < p, one fp32 rounding of the product
             if (__fmul_rn(a.u[b * (K + 1) + i], qx) < px) ++acc; else break;
@@ -269,17 +399,18 @@ __global__ void __cluster_dims__(kTailCluster, 1, 1) __launch_bounds__(kTailThre
     const int acc = s_acc;
     const float *lg = a.logits + ((size_t)b * (K + 1) + acc) * V;
     const RowStat rs = st[acc];
+    const RowFilter rf = a.filt ? a.filt[b * (K + 1) + acc] : none;
     const float u = a.u[b * (K + 1) + K];
     const float inv_t = a.inv_t;
     double S;
     int y = -1;
     if (acc < K) {
         const float *qr = a.q + ((size_t)b * K + acc) * V;
-        y = inv_cdf_cluster([&](int j) { return fmaxf(0.f, __fsub_rn(prob_of(lg[j], rs, inv_t, j), qr[j])); }, V, u,
+        y = inv_cdf_cluster([&](int j) { return fmaxf(0.f, __fsub_rn(prob_f(lg[j], rs, rf, inv_t, j), qr[j])); }, V, u,
                             sd, si, &S, &pub, cl, 0);
     }
     if (y < 0)  // all accepted: bonus from p_{K+1}; or an all-zero residual: fall back to p
-        y = inv_cdf_cluster([&](int j) { return prob_of(lg[j], rs, inv_t, j); }, V, u, sd, si, &S, &pub, cl, 1);
+        y = inv_cdf_cluster([&](int j) { return prob_f(lg[j], rs, rf, inv_t, j); }, V, u, sd, si, &S, &pub, cl, 1);
     if (y < 0) y = rs.amax;  // a row whose probabilities all vanished (non-finite logits)
     if (cl.block_rank() == 0 && threadIdx.x == 0) {
         a.n_accepted[b] = acc;
@@ -297,6 +428,8 @@ struct DraftTailArgs {
     const float *u; int u_stride;
     int32_t *token_out; int token_stride;
     float *q_out; size_t q_stride;
+    int top_k;            // restriction of q (0 / 1.0: none)
+    float top_p;
 };
 
 // grid (kTailCluster B), one cluster per sequence: q = softmax(last row / T), exported; x~ = inverse-CDF(q, u)
@@ -305,16 +438,18 @@ __global__ void __cluster_dims__(kTailCluster, 1, 1) __launch_bounds__(kTailThre
     __shared__ int si[32];
     __shared__ double sd[32];
     __shared__ ClusterSlots pub;
+    __shared__ FilterSmem fs;
     cg::cluster_group cl = cg::this_cluster();
     const int b = blockIdx.x / kTailCluster;
     int row = a.n_eff[b] - 1;
     if (row < 0) row = 0;
     const float *lg = a.logits + ((size_t)b * a.M + row) * a.V;
     const RowStat st = row_stats(lg, a.V, a.inv_t, sv, si, sd, &pub, cl);
+    const RowFilter fl = row_filter(lg, a.V, st, a.inv_t, a.top_k, a.top_p, &fs, cl);
     float *q = a.q_out + (size_t)b * a.q_stride;
     int lo, hi;
     tail_slice(a.V, (int)cl.block_rank(), lo, hi);
-    for (int j = lo + threadIdx.x; j < hi; j += blockDim.x) q[j] = prob_of(lg[j], st, a.inv_t, j);
+    for (int j = lo + threadIdx.x; j < hi; j += blockDim.x) q[j] = prob_f(lg[j], st, fl, a.inv_t, j);
     __syncthreads();  // the draw below reads this CTA's own slice of q
     double S;
     int y = inv_cdf_cluster([&](int j) { return q[j]; }, a.V, a.u[(size_t)b * a.u_stride], sd, si, &S, &pub, cl, 0);

@@ -125,3 +125,71 @@ def test_argument_errors_are_reported_on_the_host():
     assert e.value.code == -3
     with pytest.raises(B.SsdError):
         B.verify_from_logits(lg, 1, z, f, f, -1.0, z, z, 1, None, sc)       # negative temperature
+
+
+@pytest.mark.parametrize("V", [1000, 32000, 50304])
+@pytest.mark.parametrize("top_k,top_p", [(50, 1.0), (0, 0.9), (40, 0.7), (1, 1.0), (0, 0.2), (100000, 0.999)])
+def test_restricted_tail_matches_oracle(V, top_k, top_p):
+    """top-k / top-p restriction inside the tail: the p rows the decisions use equal the oracle's restricted
+    rows (same kept set unless a token sits at the nucleus boundary within rounding of the running sum), and
+    the decisions follow the oracle's rule on those rows.  q is restricted the same way on the host side of
+    the test, as a draft that runs under the same setting would deliver it."""
+    T, K, Bn = 0.9, 4, 2
+    logits, rows, q, u = make_case(2000 + V % 89 + top_k % 7, Bn, K, V, T, True)
+    std = 3.0 if V > 1000 else 1.5          # peakier rows: a nucleus of tens, not thousands, of tokens
+    logits = (logits * np.float32(std / 1.5)).astype(np.float32)
+    q = np.stack([[osamp.filter_top_k_top_p(q[b, i], top_k, top_p) for i in range(K)] for b in range(Bn)])
+    toks = synth.draw_tokens_from_rows(77, q.reshape(Bn * K, V)).reshape(Bn, K)
+    rows[:, 1:] = toks
+    B.set_sampling(top_k, top_p)
+    try:
+        n_acc, nxt, p = run_tail(logits, rows, q, u, T)
+    finally:
+        B.set_sampling(0, 1.0)
+    for b in range(Bn):
+        for i in range(K + 1):
+            raw = osamp.softmax_t(logits[b, i], T)
+            ref = osamp.filter_top_k_top_p(raw, top_k, top_p)
+            got = p[b, i]
+            same = (got > 0) == (ref > 0)
+            if not same.all():
+                # only tokens whose probability equals the threshold up to rounding of the running sums may differ
+                thr = min(raw[got > 0].min(), raw[ref > 0].min())
+                odd = raw[~same]
+                assert (np.abs(odd - thr) <= 1e-6 * max(thr, 1e-30) + 1e-12).all() or \
+                    abs(raw[got > 0].astype(np.float64).sum() - raw[ref > 0].astype(np.float64).sum()) <= 2e-6
+            else:
+                assert np.abs(got - ref).max() <= gu.P_ATOL
+                assert abs(float(got.astype(np.float64).sum()) - 1.0) < 1e-5
+        gu.check_decisions_on_own_rows(p[b], q[b], rows[b, 1:], u[b, :K], u[b, K], int(n_acc[b]), int(nxt[b]))
+        assert p[b, int(n_acc[b])][int(nxt[b])] > 0       # the emitted token lies inside the restricted target
+    if top_k == 1:
+        assert ((p > 0).sum(axis=2) == 1).all()
+
+
+def test_draft_and_verify_under_a_restriction_follow_the_oracle_loop():
+    """Whole speculative iterations with top-k / top-p set (fp32 model, so the two sides agree to rounding):
+    the draft's exported q rows, its tokens, the accepted counts and the target's tokens equal the oracle's
+    loop run with the same restriction."""
+    from oracle import decoder as od, spec as ospec
+    from paper_2311_04951_b200 import engine
+    arch = synth.gpt2_like(3, 128, 4, 256, 400, 160)
+    ws = gu.scaled_weights(synth, arch, 21, 7.0)
+    d_arch, d_ws = synth.prefix_draft(arch, ws, 1)
+    tgt = B.Model(arch, B.upload_weights(arch, ws))
+    K, T, n_new, top_k, top_p = 3, 0.9, 40, 12, 0.85
+    prompt = synth.gen_prompt(22, 1, 12, arch.vocab)
+    ref = ospec.speculative_generate(od.Model(arch, ws), od.Model(d_arch, d_ws), prompt[0], n_new, K, T,
+                                     lambda it: synth.gen_uniforms(23, 0, it, 2 * K + 1), 160, keep_trace=True,
+                                     top_k=top_k, top_p=top_p)
+    B.set_sampling(top_k, top_p)
+    try:
+        eng = engine.Engine(tgt, tgt.share_prefix(1), 1, 160, K, T, 128)
+        res = gu.lockstep(eng, synth, prompt[0], ref["iterations"], K, 23, ref["trace"])
+    finally:
+        B.set_sampling(0, 1.0)
+    assert eng.tkv.status() == 0 and eng.dkv.status() == 0
+    assert res["identical"] == res["iterations"] == ref["iterations"] and res["excused"] == 0
+    assert max(int((t["q"][0] > 0).sum()) for t in ref["trace"]) <= top_k     # the restriction was active
+    n_out = int(eng.out_count.cpu()[0])
+    assert eng.out_tokens.cpu().numpy()[0, :n_out].tolist() == ref["all_tokens"][len(prompt[0]):]
