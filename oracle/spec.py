@@ -51,10 +51,14 @@ def autoregressive_generate(target: Model, prompt, n_new: int, temperature: floa
 
 def speculative_generate(target: Model, draft: Model, prompt, n_new: int, K: int,
                          temperature: float, uniforms: Callable[[int], np.ndarray],
-                         s_max: int, keep_trace: bool = False, top_k: int = 0, top_p: float = 1.0) -> Dict:
+                         s_max: int, keep_trace: bool = False, top_k: int = 0, top_p: float = 1.0,
+                         k_of: Callable[[int, List[int]], int] = None) -> Dict:
     """top_k / top_p: both models' distributions are restricted (sampling.filter_top_k_top_p) before the
     draft draws and before the accept / resample rule, so the emitted tokens follow the restricted
-    target distribution."""
+    target distribution.
+    k_of: optional schedule of the number of draft tokens: iteration `it` drafts k_of(it, accepted so far)
+    tokens (1 <= k <= K).  The block of uniforms keeps the layout of K: draft draws u[0:k], accept tests
+    u[K:K+k], the target's draw u[2K]."""
     x = [int(t) for t in prompt]
     tc, dc = target.new_cache(s_max), draft.new_cache(s_max)
     if len(x) > 1:
@@ -67,7 +71,11 @@ def speculative_generate(target: Model, draft: Model, prompt, n_new: int, K: int
         n = len(x)
         u = np.asarray(uniforms(it), np.float32)
         assert u.shape[0] == 2 * K + 1
-        u_d, u_a, u_r = u[:K], u[K:2 * K], u[2 * K]
+        Kmax = K
+        if k_of is not None:
+            K = int(k_of(it, accepted))
+            assert 1 <= K <= Kmax
+        u_d, u_a, u_r = u[:K], u[Kmax:Kmax + K], u[2 * Kmax]
         assert tc.len == n - 1 and dc.len in (n - 1, n - 2)
         # 1. draft K tokens
         catchups.append(n - dc.len)
@@ -95,8 +103,9 @@ def speculative_generate(target: Model, draft: Model, prompt, n_new: int, K: int
         dc.rollback(min(n + a, n + K - 1))
         accepted.append(a)
         if keep_trace:
-            trace.append(dict(n=n, drafts=list(drafts), a=a, y=y, u=u.copy(),
+            trace.append(dict(n=n, drafts=list(drafts), a=a, y=y, u=u.copy(), k=K,
                               p=np.stack(p_rows), q=np.stack(q_rows), logits=logits.copy()))
+        K = Kmax
         it += 1
     return {"tokens": x[n0:n0 + n_new], "all_tokens": x, "accepted": accepted, "iterations": it,
             "target_rows": target_rows, "catchups": catchups, "trace": trace,

@@ -18,16 +18,52 @@ import torch
 from . import binding as B
 
 
+def expected_tokens(alpha: float, k: int) -> float:
+    """Tokens emitted per iteration with k draft tokens when each is accepted independently with
+    probability alpha: 1 + alpha + ... + alpha^k."""
+    return float(k + 1) if alpha >= 1.0 else (1.0 - alpha ** (k + 1)) / (1.0 - alpha)
+
+
+class AdaptiveK:
+    """Number of draft tokens per iteration from the running acceptance rate (Section "Speculative
+    Sampling": drafting pays off while the draft's tokens keep being accepted).  The rate is estimated as
+    accepted / tested over the iterations reported so far (exponentially forgotten), and the next k maximises
+    tokens per unit of time, expected_tokens(alpha, k) / (1 + k * cost), where cost = time of a draft step /
+    time of a verification pass.  Host-side policy only: no arithmetic of the method."""
+
+    def __init__(self, k_max: int, cost: float, k_min: int = 1, forget: float = 0.9, alpha0: float = 0.5):
+        assert 1 <= k_min <= k_max and cost >= 0.0 and 0.0 <= forget <= 1.0
+        self.k_max, self.k_min, self.cost, self.forget = k_max, k_min, float(cost), float(forget)
+        self.acc, self.tested = alpha0, 1.0          # one pseudo-observation at alpha0
+
+    @property
+    def alpha(self) -> float:
+        return self.acc / self.tested if self.tested > 0 else 0.0
+
+    def update(self, accepted, k: int) -> None:
+        """accepted: the iteration's accepted counts (one per sequence) with k draft tokens each."""
+        for a in accepted:
+            a = int(a)
+            self.acc = self.forget * self.acc + a
+            self.tested = self.forget * self.tested + min(a + 1, k)   # the tests up to and including the first refusal
+
+    def choose(self) -> int:
+        a = self.alpha
+        return max(range(self.k_min, self.k_max + 1), key=lambda k: (expected_tokens(a, k) / (1.0 + k * self.cost), -k))
+
+
 class Engine:
     def __init__(self, target: B.Model, draft: Optional[B.Model], batch: int, max_len: int, K: int,
                  temperature: float, out_cap: int):
         self.target, self.draft = target, draft
         self.batch, self.max_len, self.K, self.T = batch, max_len, K, float(temperature)
+        self.K_max = K
         V = target.arch.vocab
         dev = "cuda"
         self.tkv = B.KV(target, batch, max_len)
         self.ws_t = target.new_workspace(batch, K + 1, max_len)
         self.rows = torch.zeros(batch, K + 1, dtype=torch.int32, device=dev)
+        self._rows_of = {K: self.rows}    # row blocks of iterations that draft fewer than K tokens (stride k + 1)
         # accepted counts of the last `log_cap` iterations, one row each: target_verify writes row it % log_cap
         # (a pointer, not a copy), so acceptance statistics can be read after a run without touching the loop
         self.log_cap = max(1, out_cap // (K + 1) + 1)
@@ -43,7 +79,8 @@ class Engine:
             self.dkv = B.KV(draft, batch, max_len)
             self.ws_d = draft.new_workspace(batch, 2, max_len)
             self.ws_pre_d = draft.new_workspace(batch, self.chunk, max_len)
-            self.q = torch.zeros(batch, K, V, dtype=torch.float32, device=dev)
+            self.q_full = torch.zeros(batch * K * V, dtype=torch.float32, device=dev)
+            self.q = self.q_full.view(batch, K, V)
             self.draft_in = torch.zeros(batch, 2, dtype=torch.int32, device=dev)
             self.draft_n_in = torch.ones(batch, dtype=torch.int32, device=dev)
         else:
@@ -85,15 +122,29 @@ class Engine:
             self.draft_n_in.fill_(1)
         self.out_count.zero_()
 
-    # ---- one iteration; u_draft [batch, K], u_verify [batch, K+1] fp32 on the device ----
+    def set_k(self, k: int) -> None:
+        """Draft k <= K tokens in the following iterations: the row block and the q block become [batch, k + 1]
+        and [batch, k, V] (views of the buffers sized for K); the pending token moves along."""
+        assert 1 <= k <= self.K_max and self.dkv is not None
+        if k == self.K:
+            return
+        if k not in self._rows_of:
+            self._rows_of[k] = torch.zeros(self.batch, k + 1, dtype=torch.int32, device=self.rows.device)
+        new = self._rows_of[k]
+        new[:, 0] = self.rows[:, 0]
+        self.rows, self.K = new, k
+        self.q = self.q_full[:self.batch * k * self.target.arch.vocab].view(self.batch, k, self.target.arch.vocab)
+
+    # ---- one iteration; u_draft [batch, >= K] (row stride = its width), u_verify [batch, K+1] contiguous, on the device ----
     def spec_iteration(self, u_draft: torch.Tensor, u_verify: torch.Tensor, p_debug: Optional[torch.Tensor] = None):
         K, V = self.K, self.target.arch.vocab
+        us = u_draft.stride(0)
         for i in range(K):
             if i == 0:
                 tok_in, stride, rows_in, n_in = self.draft_in, 2, 2, self.draft_n_in
             else:
                 tok_in, stride, rows_in, n_in = self.rows[:, i:], K + 1, 1, None
-            B.draft_step(self.draft, self.dkv, tok_in, stride, rows_in, n_in, self.T, u_draft[:, i:], K,
+            B.draft_step(self.draft, self.dkv, tok_in, stride, rows_in, n_in, self.T, u_draft[:, i:], us,
                          self.rows[:, i + 1:], K + 1, self.q[:, i], K * V, self.ws_d)
         B.target_verify(self.target, self.tkv, self.rows, K, self.q, u_verify, self.T, self.n_acc, self.next_tok, 1,
                         p_debug, self.ws_t)
@@ -113,9 +164,14 @@ class Engine:
 
     # ---- whole generations ----
     def generate(self, prompts: np.ndarray, n_new: int, uniforms: Callable[[int, int], np.ndarray],
-                 check_every: int = 4, max_iters: Optional[int] = None) -> Dict:
+                 check_every: int = 4, max_iters: Optional[int] = None, policy: Optional[AdaptiveK] = None) -> Dict:
         """uniforms(seq, iteration) -> fp32 [2K+1] (speculative) or [>=1] (autoregressive, K == 0).
-        Runs until every sequence has >= n_new tokens; the host only polls the counters."""
+        Runs until every sequence has >= n_new tokens; the host only polls the counters.
+        With a policy, the number of draft tokens follows it from iteration to iteration (the accepted counts
+        are read back every iteration); the block of uniforms keeps the layout of the largest K: draft draws
+        u[0:k], accept tests u[K:K+k], the target's draw u[2K]."""
+        if policy is not None:
+            return self._generate_adaptive(prompts, n_new, uniforms, policy, max_iters)
         dev = "cuda"
         K = self.K
         self.prefill(torch.from_numpy(np.ascontiguousarray(prompts, np.int32)).to(dev))
@@ -140,3 +196,28 @@ class Engine:
         toks = self.out_tokens.cpu().numpy()
         return {"tokens": [toks[b, :min(n_new, counts[b])].tolist() for b in range(self.batch)],
                 "counts": counts, "iterations": iters, "status": self.tkv.status()}
+
+    def _generate_adaptive(self, prompts, n_new, uniforms, policy: AdaptiveK, max_iters) -> Dict:
+        dev = "cuda"
+        Km = self.K_max
+        self.prefill(torch.from_numpy(np.ascontiguousarray(prompts, np.int32)).to(dev))
+        iters, ks = 0, []
+        limit = max_iters if max_iters is not None else n_new
+        while iters < limit:
+            k = policy.choose()
+            self.set_k(k)
+            u = np.stack([uniforms(s, iters) for s in range(self.batch)]).astype(np.float32)
+            ud = torch.from_numpy(u[:, :k].copy()).to(dev)
+            uv = torch.from_numpy(np.concatenate([u[:, Km:Km + k], u[:, 2 * Km:2 * Km + 1]], axis=1).copy()).to(dev)
+            self.spec_iteration(ud, uv)
+            acc = self.n_acc.cpu().numpy()
+            self.advance()
+            policy.update(acc, k)
+            ks.append(k)
+            iters += 1
+            if int(self.out_count.min().item()) >= n_new:
+                break
+        counts = self.out_count.cpu().numpy()
+        toks = self.out_tokens.cpu().numpy()
+        return {"tokens": [toks[b, :min(n_new, counts[b])].tolist() for b in range(self.batch)],
+                "counts": counts, "iterations": iters, "status": self.tkv.status(), "ks": ks}

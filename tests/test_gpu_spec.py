@@ -126,3 +126,22 @@ def test_autoregressive_sampling_matches_oracle():
     out = engine.Engine(tgt, None, 1, 96, 0, 0.7, 64).generate(prompt, 30, uni)
     ref = ospec.autoregressive_generate(otgt, prompt[0], 30, 0.7, lambda it: uni(0, it), 96)["tokens"]
     assert out["tokens"][0] == ref
+
+
+def test_adaptive_k_generation_matches_the_oracle_run_with_the_same_schedule():
+    """The number of draft tokens follows the running acceptance rate (host policy); the oracle's loop,
+    given the schedule the engine used, must emit the same tokens (fp32 model: every decision identical)."""
+    arch = synth.gpt2_like(3, 128, 4, 256, 400, 200)
+    (tgt, drf), (otgt, odrf) = build_pair(arch, 61, 7.0, 1)
+    Kmax, T, n_new = 6, 0.9, 48
+    prompt = synth.gen_prompt(62, 1, 10, arch.vocab)
+    uni = lambda s, it: synth.gen_uniforms(63, s, it, 2 * Kmax + 1)
+    pol = engine.AdaptiveK(k_max=Kmax, cost=0.15, forget=0.8)
+    eng = engine.Engine(tgt, drf, 1, 200, Kmax, T, 128)
+    out = eng.generate(prompt, n_new, uni, policy=pol)
+    assert out["status"] == 0 and len(set(out["ks"])) > 1            # the policy really moved K
+    ks = out["ks"]
+    ref = ospec.speculative_generate(otgt, odrf, prompt[0], n_new, Kmax, T, lambda it: uni(0, it), 200,
+                                     k_of=lambda it, acc: ks[it] if it < len(ks) else ks[-1])
+    assert out["tokens"][0] == ref["tokens"]
+    assert ref["iterations"] == out["iterations"]
