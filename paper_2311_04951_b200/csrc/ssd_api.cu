@@ -25,6 +25,7 @@ namespace {
 
 std::atomic<uint64_t> g_launches{0};
 int g_num_sms = 0;
+int g_l2_window = 0;  // bytes of L2 that may hold persisting lines (0: the device has none / the limit could not be set)
 bool g_attr_done = false;
 std::mutex g_mu;
 
@@ -135,6 +136,16 @@ int init_device_once() {
     int dev = 0;
     CUDA_OK(cudaGetDevice(&dev));
     CUDA_OK(cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev));
+    {   // room in L2 for persisting lines (a limit of this process's context, gone with it)
+        int max_persist = 0, max_window = 0;
+        cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev);
+        cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, dev);
+        size_t want = 32u << 20;
+        if ((size_t)max_persist < want) want = (size_t)max_persist;
+        if (want > 0 && cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) == cudaSuccess)
+            g_l2_window = (int)(want < (size_t)max_window ? want : (size_t)max_window);
+        (void)cudaGetLastError();
+    }
     int rc = 0;
     rc |= set_smem(gemm_bf16_kernel<1>, gemm_smem<1>());
     rc |= set_smem(gemm_bf16_kernel<2>, gemm_smem<2>());
@@ -461,7 +472,7 @@ int run_attention(const ssd_model *m, ssd_kv *kv, int layer, const float *q, int
 inline int barriers_needed(const ssd_arch &a) { return (a.parallel_residual ? 5 : 8) * a.n_layers; }  // upper bound
 
 template <int NT>
-int launch_forward_nt(FwdParams p, cudaStream_t st) {
+int launch_forward_nt(FwdParams p, const void *ws_base, size_t ws_bytes, cudaStream_t st) {
     constexpr size_t stage = kWTileBytesP + 2 * NT * 8 * kTileK * 2;
     size_t attn = align_up(attn_scratch_bytes(p.Dh), 128);
     if (p.attn_tc && attn < (size_t)kTcScratchBytes) attn = kTcScratchBytes;
@@ -493,21 +504,44 @@ int launch_forward_nt(FwdParams p, cudaStream_t st) {
         attr[dev] = true;
     }
     void *args[] = {&p};
-    if (cudaLaunchCooperativeKernel((void *)forward_kernel<NT>, dim3(g_num_sms), dim3(kPersistThreads), args, smem,
-                                    st) != cudaSuccess)
-        return SSD_E_CUDA;
+    // The workspace (residual stream, GEMM outputs and operands: a few MB that every phase re-reads and that the
+    // GEMMs reduce into) is marked persisting in L2 for this launch, so that the weight stream does not push it
+    // out between the phase that writes a buffer and the phase that reads it.
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(g_num_sms);
+    cfg.blockDim = dim3(kPersistThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attrs[2];
+    int na = 0;
+    attrs[na].id = cudaLaunchAttributeCooperative;
+    attrs[na].val.cooperative = 1;
+    ++na;
+    if (g_l2_window > 0 && ws_base && ws_bytes > 0) {
+        attrs[na].id = cudaLaunchAttributeAccessPolicyWindow;
+        attrs[na].val.accessPolicyWindow.base_ptr = const_cast<void *>(ws_base);
+        attrs[na].val.accessPolicyWindow.num_bytes = ws_bytes < (size_t)g_l2_window ? ws_bytes : (size_t)g_l2_window;
+        attrs[na].val.accessPolicyWindow.hitRatio = 1.0f;
+        attrs[na].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+        attrs[na].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+        ++na;
+    }
+    cfg.attrs = attrs;
+    cfg.numAttrs = na;
+    if (cudaLaunchKernelExC(&cfg, (const void *)forward_kernel<NT>, args) != cudaSuccess) return SSD_E_CUDA;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return SSD_OK;
 }
 
-int launch_forward_rows(const FwdParams &p, int rows_k, cudaStream_t st) {
+int launch_forward_rows(const FwdParams &p, int rows_k, const void *ws_base, size_t ws_bytes, cudaStream_t st) {
     switch (rows_k / 8) {
-        case 1: return launch_forward_nt<1>(p, st);
-        case 2: return launch_forward_nt<2>(p, st);
-        case 3: return launch_forward_nt<3>(p, st);
-        case 4: return launch_forward_nt<4>(p, st);
-        case 5: return launch_forward_nt<5>(p, st);
-        case 8: return launch_forward_nt<8>(p, st);
+        case 1: return launch_forward_nt<1>(p, ws_base, ws_bytes, st);
+        case 2: return launch_forward_nt<2>(p, ws_base, ws_bytes, st);
+        case 3: return launch_forward_nt<3>(p, ws_base, ws_bytes, st);
+        case 4: return launch_forward_nt<4>(p, ws_base, ws_bytes, st);
+        case 5: return launch_forward_nt<5>(p, ws_base, ws_bytes, st);
+        case 8: return launch_forward_nt<8>(p, ws_base, ws_bytes, st);
         default: break;
     }
     return SSD_E_CAPACITY;
@@ -567,7 +601,7 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     CUDA_OK(cudaMemsetAsync(w.sync, 0, w.sync_bytes, st));
     cudaEvent_t prof_stop;
     if (prof_begin(st, &prof_stop)) return SSD_E_CUDA;
-    int rc = launch_forward_rows(p, Rk, st);
+    int rc = launch_forward_rows(p, Rk, w.ri.seq, w.bytes, st);
     if (!rc && prof_end(st, prof_stop)) return SSD_E_CUDA;
     if (rc) return rc;
     kv->last_rows = M;
