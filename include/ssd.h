@@ -158,6 +158,24 @@ int draft_step(ssd_model *draft, ssd_kv *dkv, const int32_t *dev_tokens_in, int 
                size_t ws_bytes, void *stream);
 
 /*
+ * The draft loop of an iteration - n_steps draft steps - as one call (Section "Speculative Sampling": the draft
+ * model proposes a short run of tokens before the target looks at them; Section "So, what's the problem?": the
+ * draft keeps a cache of its own, which this call advances by every row it feeds).  Step 0 is draft_step's
+ * (rows_in catch-up rows, n_in of them per sequence); step s > 0 feeds the token step s - 1 drew.  Step s reads
+ * its uniform at dev_u[b * u_stride + s], writes its token to dev_tokens_out[b * token_out_stride + s] and its
+ * q row to dev_q_out + b * q_stride + s * vocab (element strides; q_stride >= n_steps * vocab): with
+ * token_out_stride = K + 1 and q_stride = K * vocab these are columns 1.. of target_verify's row block and its
+ * q block.  bf16 models run all steps in ONE launch of the forward kernel, which ends every step itself (q, draw,
+ * commit spread over the grid) and goes on without returning to the host, its weight stream running on across
+ * the steps; other models, and any call made while a sampling restriction is set, run the same steps as
+ * separate draft_step calls.  1 <= n_steps <= SSD_MAX_ROWS_PER_SEQ; results as n_steps calls of draft_step.
+ */
+int draft_steps(ssd_model *draft, ssd_kv *dkv, int n_steps, const int32_t *dev_tokens_in, int tokens_stride,
+                int rows_in, const int32_t *dev_n_in, float temperature, const float *dev_u, int u_stride,
+                int32_t *dev_tokens_out, int token_out_stride, float *dev_q_out, size_t q_stride, void *dev_ws,
+                size_t ws_bytes, void *stream);
+
+/*
  * The verification step (Section "Autoregressive vs Speculative Sampling": the target model scores
  * all K draft tokens in one pass; Figure 2).  One forward over K+1 rows per sequence
  *   dev_rows[b, 0..K] = pending token, x~_1 .. x~_K                 (int32, row stride K+1)

@@ -38,7 +38,7 @@ EXPORTS = ["ssd_model_create", "ssd_model_desc_bytes", "ssd_set_persistent", "ss
            "ssd_workspace_bytes", "kv_init", "kv_destroy", "kv_prefill", "draft_step", "target_verify",
            "kv_commit", "kv_rollback", "spec_advance", "kv_lengths", "ssd_device_status",
            "verify_from_logits", "verify_from_logits_noalloc", "verify_scratch_bytes", "attention_rows", "ssd_last_logits", "ssd_set_trace", "ssd_read_trace", "ssd_launch_count",
-           "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror", "ssd_set_wait_limit", "ssd_wait_probe", "ssd_set_sampling"]
+           "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror", "ssd_set_wait_limit", "ssd_wait_probe", "ssd_set_sampling", "draft_steps"]
 
 
 def lib_path() -> str:
@@ -74,6 +74,7 @@ def load():
     L.kv_destroy.restype = None
     L.kv_prefill.argtypes = [vp, vp, vp, vp, i32, vp, sz, vp]
     L.draft_step.argtypes = [vp, vp, vp, i32, i32, vp, f32, vp, i32, vp, i32, vp, sz, vp, sz, vp]
+    L.draft_steps.argtypes = [vp, vp, i32, vp, i32, i32, vp, f32, vp, i32, vp, i32, vp, sz, vp, sz, vp]
     L.target_verify.argtypes = [vp, vp, vp, i32, vp, vp, f32, vp, vp, i32, vp, vp, sz, vp]
     L.kv_commit.argtypes = [vp, vp, vp]
     L.kv_rollback.argtypes = [vp, vp, vp]
@@ -238,6 +239,17 @@ def draft_step(draft: Model, dkv: KV, tokens_in: torch.Tensor, tokens_stride: in
     _check(load().draft_step(draft.h, dkv.h, _p(tokens_in), tokens_stride, rows_in, _p(n_in), temperature, _p(u),
                              u_stride, _p(token_out), token_out_stride, _p(q_out), q_stride, _p(ws), ws.numel(),
                              _stream()), "draft_step")
+
+
+def draft_steps(draft: Model, dkv: KV, n_steps: int, tokens_in: torch.Tensor, tokens_stride: int, rows_in: int,
+                n_in: Optional[torch.Tensor], temperature: float, u: torch.Tensor, u_stride: int,
+                tokens_out: torch.Tensor, token_out_stride: int, q_out: torch.Tensor, q_stride: int,
+                ws: torch.Tensor) -> None:
+    """n_steps draft steps in one call (one launch for bf16 models): step s draws with u[b * u_stride + s] and
+    writes tokens_out[b * token_out_stride + s] and the q row at q_out + b * q_stride + s * vocab."""
+    _check(load().draft_steps(draft.h, dkv.h, n_steps, _p(tokens_in), tokens_stride, rows_in, _p(n_in), temperature,
+                              _p(u), u_stride, _p(tokens_out), token_out_stride, _p(q_out), q_stride, _p(ws),
+                              ws.numel(), _stream()), "draft_steps")
 
 
 def target_verify(target: Model, tkv: KV, rows: torch.Tensor, K: int, q: Optional[torch.Tensor], u: torch.Tensor,

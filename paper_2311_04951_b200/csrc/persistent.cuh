@@ -121,6 +121,20 @@ struct alignas(64) FwdParams {
     int attn_ctas;           // min(attention items, CTAs): set by the host together with the split plan
     int overlap_out;         // parallel-residual block and at most half of the CTAs on attention
     long long wait_cycles;   // bound of every wait that takes work (see Shared::wait_limit)
+    // Several draft steps in one launch (n_steps >= 1; the draft loop of a speculative iteration).  With tail == 1
+    // every step ends inside the kernel: the logits of each sequence's last fed row become q = softmax(logits / T),
+    // a token is drawn from q with the step's uniform, both are written out, the fed rows are committed, and the
+    // next step feeds that token (one row per sequence).  cur_step is kept by the kernel in its copy of this block.
+    int n_steps, tail, cur_step;
+    float inv_t;                                   // 1 / T; 0 = greedy
+    const float *u;     int u_stride;              // uniform of sequence b at step s: u[b * u_stride + s]
+    int32_t *tok_out;   int tok_out_stride;        // token of step s: tok_out[b * tok_out_stride + s]
+    float *q_out;       size_t q_stride;           // q row of step s: q_out + b * q_stride + s * V
+    int32_t *len_rw;                               // the committed lengths, advanced after every step
+    float *tp_m, *tp_s; int32_t *tp_a;             // per (sequence, CTA): max, sum of exp relative to it, argmax of the CTA's slice
+    double *tp_mass;                               // per (sequence, CTA): mass of q in the CTA's slice
+    int32_t *tail_hit;                             // [n_steps][B][2]: smallest index past u S (INT_MAX: none) / largest index with q > 0
+    unsigned long long *mailbox; unsigned mb_seq;  // the largest length, reported to the host at the end
 };
 
 struct GemmDesc {
@@ -151,11 +165,17 @@ __device__ __forceinline__ int attention_end(const FwdParams &p) { return overla
 //   parallel layer:   qkv, in | attention + act | o, out | next norms            (4 barriers)
 //   ... with few attention items: qkv, in | act | attention (some CTAs); out, then - once every attention CTA has
 //       signalled - o (the others) | next norms   (4)
-__device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi, const float *const *ltab = nullptr) {
+// Grid barriers of one step of a launch: the head, the layers', and five around the phases of the in-kernel tail.
+__device__ __forceinline__ int step_barriers(const FwdParams &p) { return 1 + barriers_per_layer(p) * p.n_layers + (p.tail ? 5 : 0); }
+constexpr int kStepShift = 12;  // a GEMM is named (step << kStepShift) | number within the forward
+
+__device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi_step, const float *const *ltab = nullptr) {
     GemmDesc g;
     g.wait_attn = 0;
+    const int step = gi_step >> kStepShift, gi = gi_step & ((1 << kStepShift) - 1);
+    const int sb = step * step_barriers(p);  // barriers before this step
     const int l = gi >> 2, e = gi & 3;
-    const int base = 1 + barriers_per_layer(p) * l;
+    const int base = sb + 1 + barriers_per_layer(p) * l;
     if (l >= p.n_layers) {  // LM head
         g.tmW = &p.md->tm_lm; g.xop = p.op[OP_XN1];
         g.N = p.V; g.Kd = p.d; g.need = base; g.out = p.logits; g.ldo = p.V; g.bias = nullptr;
@@ -170,14 +190,14 @@ __device__ __forceinline__ GemmDesc gemm_desc(const FwdParams &p, int gi, const 
         g.kind = kind;
         // the attention phase of layer l ends at barrier base + 2; qkv precedes it (previous layer's counts)
         // (so does the MLP input GEMM of a parallel-residual block)
-        g.need_hi = (kind == 0 || (kind == 2 && p.parallel)) ? (l == 0 ? 0 : base - barriers_per_layer(p) + attention_end(p))
+        g.need_hi = (kind == 0 || (kind == 2 && p.parallel)) ? (l == 0 ? sb : base - barriers_per_layer(p) + attention_end(p))
                                                              : base + attention_end(p);
         if (kind == 0) {
             g.xop = p.op[OP_XN1]; g.N = 3 * p.d; g.Kd = p.d; g.need = base;
             g.out = p.qkv; g.ldo = 3 * p.d; g.bias = ltab ? ltab[8 * l + 2] : ld->b_qkv;
         } else if (kind == 1) {
             g.xop = p.op[OP_AO]; g.N = p.d; g.Kd = p.d; g.need = base + 2;
-            if (overlap_mlp_out(p)) g.wait_attn = (unsigned)(l + 1) * (unsigned)attention_ctas(p);
+            if (overlap_mlp_out(p)) g.wait_attn = (unsigned)(step * p.n_layers + l + 1) * (unsigned)attention_ctas(p);
             g.out = p.x; g.ldo = p.d; g.bias = ltab ? ltab[8 * l + 3] : ld->b_o;
         } else if (kind == 2) {
             g.xop = p.op[p.parallel ? OP_XN2 : OP_XN1]; g.N = p.d_in; g.Kd = p.d; g.need = p.parallel ? base : base + 4;
@@ -639,9 +659,9 @@ __device__ __noinline__ void setup_phase(const FwdParams &p) {
     const int half = p.rotary_dim / 2;
     for (int r = blockIdx.x; r < p.R; r += gridDim.x) {
         const int b = r / p.M, j = r % p.M;
-        int n = p.n_rows ? p.n_rows[b] : p.M;
+        int n = p.cur_step > 0 ? 1 : (p.n_rows ? p.n_rows[b] : p.M);
         n = max(0, min(n, p.M));
-        const int len = p.len[b];
+        const int len = __ldcg(p.len + b);  // (advanced between the steps of a draft loop)
         const bool fits = len + n <= p.S && (p.pos_limit == 0 || len + n <= p.pos_limit);
         if (!fits) {
             n = 0;
@@ -669,7 +689,9 @@ __device__ __noinline__ void setup_phase(const FwdParams &p) {
 __device__ __noinline__ void embed_phase(const FwdParams &p) {
     for (int r = blockIdx.x; r < p.R; r += gridDim.x) {
         const int b = r / p.M, j = r % p.M;
-        int tok = __ldcg(p.ri.valid + r) ? p.tokens[(size_t)b * p.tok_stride + j] : 0;
+        int tok = 0;
+        if (__ldcg(p.ri.valid + r))
+            tok = p.cur_step > 0 ? __ldcg(p.tok_out + (size_t)b * p.tok_out_stride + p.cur_step - 1) : p.tokens[(size_t)b * p.tok_stride + j];
         tok = max(0, min(tok, p.V - 1));
         const int pos = __ldcg(p.ri.pos + r);
         for (int i = threadIdx.x; i < p.d; i += kWorkThreads) {
@@ -1823,6 +1845,161 @@ __device__ __noinline__ void run_gemm(const FwdParams &p, int gi, uint8_t *smem)
             save_state();
 }
 
+// ---- the vocabulary-wide tail of a draft step, inside the kernel ---------------------------------
+// After the LM head of a draft step every sequence's last fed row of logits is turned into q = softmax(row / T),
+// exported, and sampled by inverse CDF with the step's uniform - the work of draft_tail_kernel, spread over the
+// whole grid so that the kernel can go on to the next step without returning to the host.  CTA c owns the slice
+// [c * per, (c + 1) * per) of the vocabulary; inside a CTA warp w works on sequences w, w + 8, ... with warp
+// shuffles only.  Three phases, a grid barrier behind each:
+//   1. per (sequence, CTA): max, argmax and sum of exp relative to that max over the slice;
+//   2. every CTA combines the partials of all CTAs into (max, argmax, Z), writes its slice of q and the slice's
+//      mass (fp64, index order: lane l holds a contiguous piece of the slice);
+//   3. every CTA takes the prefix of the slice masses in CTA order; the lanes whose piece can hold the first
+//      index with c_j > u S walk it and post the index (atomic minimum); the largest index with q > 0 is
+//      posted too (the fallback when rounding leaves no index past u S);
+// then CTA 0 writes the tokens and commits the rows fed in this step.
+__device__ __forceinline__ int tail_per(const FwdParams &p) { return (((p.V + (int)gridDim.x - 1) / (int)gridDim.x) + 3) & ~3; }
+__device__ __forceinline__ const float *tail_row(const FwdParams &p, int b) {
+    int row = __ldcg(p.ri.n_eff + b) - 1;
+    if (row < 0) row = 0;
+    return p.logits + ((size_t)b * p.M + row) * p.V;
+}
+
+__device__ __noinline__ void tail_partial(const FwdParams &p) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, G = (int)gridDim.x;
+    const int per = tail_per(p), lo = min(p.V, (int)blockIdx.x * per), hi = min(p.V, lo + per);
+    for (int b = warp; b < p.B; b += kConsumerWarps) {
+        const float *lg = tail_row(p, b);
+        float mx = -INFINITY;
+        int am = 0x7fffffff;
+        for (int j = lo + lane; j < hi; j += 32) {
+            const float l = __ldcg(lg + j);
+            if (l > mx) { mx = l; am = j; }  // ascending per lane: the first maximum
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, mx, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, am, o);
+            if (ov > mx || (ov == mx && oi < am)) { mx = ov; am = oi; }
+        }
+        float sum = 0.f;
+        if (p.inv_t != 0.f && mx > -INFINITY)
+            for (int j = lo + lane; j < hi; j += 32) sum += expf((__ldcg(lg + j) - mx) * p.inv_t);
+        sum = warp_sum(sum);
+        if (lane == 0) {
+            p.tp_m[(size_t)b * G + blockIdx.x] = mx;
+            p.tp_s[(size_t)b * G + blockIdx.x] = sum;
+            p.tp_a[(size_t)b * G + blockIdx.x] = am;
+        }
+    }
+}
+
+// (max, argmax - lowest index among the maxima -, Z) of a sequence's row from the CTAs' partials; the same in every lane
+__device__ __forceinline__ void tail_stats(const FwdParams &p, int b, float &mx, int &am, float &z) {
+    const int lane = threadIdx.x & 31, G = (int)gridDim.x;
+    mx = -INFINITY;
+    am = 0x7fffffff;
+    for (int c = lane; c < G; c += 32) {
+        const float v = __ldcg(p.tp_m + (size_t)b * G + c);
+        const int i = __ldcg(p.tp_a + (size_t)b * G + c);
+        if (v > mx || (v == mx && i < am)) { mx = v; am = i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, mx, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, am, o);
+        if (ov > mx || (ov == mx && oi < am)) { mx = ov; am = oi; }
+    }
+    double zz = 0.0;
+    if (p.inv_t != 0.f)
+        for (int c = lane; c < G; c += 32) {
+            const float m = __ldcg(p.tp_m + (size_t)b * G + c);
+            if (m > -INFINITY) zz += (double)__ldcg(p.tp_s + (size_t)b * G + c) * (double)expf((m - mx) * p.inv_t);
+        }
+    zz = warp_sum(zz);
+    z = (float)zz;
+}
+__device__ __forceinline__ float tail_prob(float logit, float mx, int am, float z, float inv_t, int j) {
+    if (inv_t == 0.f) return j == am ? 1.f : 0.f;
+    return expf((logit - mx) * inv_t) / z;
+}
+
+__device__ __noinline__ void tail_q(const FwdParams &p) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, G = (int)gridDim.x;
+    const int per = tail_per(p), lo = min(p.V, (int)blockIdx.x * per), hi = min(p.V, lo + per);
+    const int seg = (hi - lo + 31) / 32, j0 = min(hi, lo + lane * seg), j1 = min(hi, j0 + seg);
+    for (int b = warp; b < p.B; b += kConsumerWarps) {
+        const float *lg = tail_row(p, b);
+        float mx, z;
+        int am;
+        tail_stats(p, b, mx, am, z);
+        float *q = p.q_out + (size_t)b * p.q_stride + (size_t)p.cur_step * p.V;
+        double local = 0.0;
+        for (int j = j0; j < j1; ++j) {
+            const float w = tail_prob(__ldcg(lg + j), mx, am, z, p.inv_t, j);
+            q[j] = w;
+            local += (double)w;
+        }
+        local = warp_sum(local);  // (a sum of at most 32 pieces: the order does not matter at fp64 for a decision that
+        if (lane == 0) p.tp_mass[(size_t)b * G + blockIdx.x] = local;  //  is excused within 1e-6 S of a step anyway)
+    }
+}
+
+__device__ __noinline__ void tail_draw(const FwdParams &p) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, G = (int)gridDim.x;
+    const int per = tail_per(p), lo = min(p.V, (int)blockIdx.x * per), hi = min(p.V, lo + per);
+    const int seg = (hi - lo + 31) / 32, j0 = min(hi, lo + lane * seg), j1 = min(hi, j0 + seg);
+    for (int b = warp; b < p.B; b += kConsumerWarps) {
+        // prefix of the slice masses in CTA order (every lane walks all of them: G loads that overlap)
+        double off = 0.0, S = 0.0;
+        for (int c = 0; c < G; ++c) {
+            const double t = __ldcg(p.tp_mass + (size_t)b * G + c);
+            if (c < (int)blockIdx.x) off += t;
+            S += t;
+        }
+        const float *q = p.q_out + (size_t)b * p.q_stride + (size_t)p.cur_step * p.V;
+        double local = 0.0;
+        int last_pos = -1;
+        for (int j = j0; j < j1; ++j) {
+            const float w = q[j];  // written by this very lane in the phase before
+            local += (double)w;
+            if (w > 0.f) last_pos = j;
+        }
+        double incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        const double target = (double)__ldcg(p.u + (size_t)b * p.u_stride + p.cur_step) * S;
+        double run = off + (incl - local);
+        int hit = 0x7fffffff;
+        if (S > 0.0 && (run + local > target || run > target)) {
+            for (int j = j0; j < j1; ++j) {
+                const float w = q[j];
+                run += (double)w;
+                if (w > 0.f && run > target) { hit = j; break; }  // a zero-weight index is never drawn
+            }
+        }
+        int32_t *slot = p.tail_hit + ((size_t)p.cur_step * p.B + b) * 2;
+        if (hit != 0x7fffffff) atomicMin(slot, hit);
+        if (last_pos >= 0) atomicMax(slot + 1, last_pos);
+    }
+}
+
+// CTA 0: the tokens of this step, and the rows it fed become part of the cache
+__device__ __noinline__ void tail_commit(const FwdParams &p) {
+    if (blockIdx.x != 0) return;
+    for (int b = threadIdx.x; b < p.B; b += kWorkThreads) {
+        const int32_t *slot = p.tail_hit + ((size_t)p.cur_step * p.B + b) * 2;
+        const int hit = __ldcg(slot), last = __ldcg(slot + 1);
+        int tok = hit != 0x7fffffff ? hit : last;
+        if (tok < 0) tok = max(0, min(__ldcg(p.tp_a + (size_t)b * gridDim.x), p.V - 1));  // a row without any probability
+        p.tok_out[(size_t)b * p.tok_out_stride + p.cur_step] = tok;
+        p.len_rw[b] = __ldcg(p.len_rw + b) + __ldcg(p.ri.n_eff + b);
+    }
+}
+
 // ---- the kernel -----------------------------------------------------------------------------
 // NT = padded rows / 8
 template <int NT>
@@ -1918,7 +2095,8 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             // a CTA that never runs an attention item (fewer items than CTAs) never uses the scratch: its
             // upper slots take weights at any time
             const bool scratch_used = (int)blockIdx.x < p.B * p.H * p.n_split * ((p.M + kAttnRows - 1) / kAttnRows);
-            for (int gw = 0; gw < NG && !failed; ++gw) {
+            for (int gws = 0; gws < NG * p.n_steps && !failed; ++gws) {
+                const int gw = ((gws / NG) << kStepShift) | (gws % NG);
                 const GemmDesc dw = gemm_desc(p, gw);
                 int c0, c1;
                 unit_range(p, dw, c0, c1);
@@ -1984,63 +2162,89 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
                 grid_zero(p.logits, p.R, p.V, p.V);
             }
         };
-        // Set-up, embedding and the first norm of a row all run on the CTA that owns the row, so only
-        // CTA-wide barriers separate them: one grid barrier in front of the first GEMM instead of two.
-        setup_phase(p);
-        named_bar(2, kWorkThreads);  // the row's position and validity are read back by the embedding
-        embed_phase(p);
-        named_bar(2, kWorkThreads);  // the embedding rows are read back by the norm
-        norm_for_layer(0);
-        bool go = grid_sync(p, sh, epoch);
-        if (go && threadIdx.x < 64) {  // lengths and rows of this pass (written by the set-up of every row), for the
-            const int b = threadIdx.x;  // attention items, which run behind further grid barriers
-            seq_tab[b] = b < p.B ? p.len[b] : 0;
-            seq_tab[64 + b] = b < p.B ? __ldcg(p.ri.n_eff + b) : 0;
-        }
-        for (int l = 0; l < p.n_layers && go; ++l) {
-            run_gemm<NT>(p, 4 * l + 0, smem);                       // qkv
-            if (p.parallel) run_gemm<NT>(p, 4 * l + 1, smem);       // MLP in (same block input)
-            if (!(go = grid_sync(p, sh, epoch))) break;
-            if (overlap_mlp_out(p)) {
-                act_phase(p);
-                if ((int)blockIdx.x < attention_ctas(p)) {
-                    grid_arrive(p, sh, epoch);  // the activation is out; attention needs nothing from the others
-                    attention_phase(p, l, attn_scratch, sh);
-                    attn_signal(p, sh);
-                } else {
+        if (p.tail && blockIdx.x == 0)  // the draws' meeting places: smallest hit index / largest index with weight
+            for (int i = threadIdx.x; i < p.n_steps * p.B * 2; i += kWorkThreads) p.tail_hit[i] = (i & 1) ? -1 : 0x7fffffff;
+        bool go = true;
+        for (int step = 0; step < p.n_steps && go; ++step) {
+            const int gs = step << kStepShift;
+            if (step > 0) {  // the rows of this step: one per sequence, the token the step before drew
+                if (threadIdx.x == 0) psm->cur_step = step;
+                named_bar(2, kWorkThreads);
+            }
+            // Set-up, embedding and the first norm of a row all run on the CTA that owns the row, so only
+            // CTA-wide barriers separate them: one grid barrier in front of the first GEMM instead of two.
+            setup_phase(p);
+            named_bar(2, kWorkThreads);  // the row's position and validity are read back by the embedding
+            embed_phase(p);
+            named_bar(2, kWorkThreads);  // the embedding rows are read back by the norm
+            norm_for_layer(0);
+            go = grid_sync(p, sh, epoch);
+            if (go && threadIdx.x < 64) {  // lengths and rows of this pass (written by the set-up of every row), for the
+                const int b = threadIdx.x;  // attention items, which run behind further grid barriers
+                seq_tab[b] = b < p.B ? __ldcg(p.len + b) : 0;
+                seq_tab[64 + b] = b < p.B ? __ldcg(p.ri.n_eff + b) : 0;
+            }
+            for (int l = 0; l < p.n_layers && go; ++l) {
+                run_gemm<NT>(p, gs | (4 * l + 0), smem);                  // qkv
+                if (p.parallel) run_gemm<NT>(p, gs | (4 * l + 1), smem);       // MLP in (same block input)
+                if (!(go = grid_sync(p, sh, epoch))) break;
+                if (overlap_mlp_out(p)) {
+                    act_phase(p);
+                    if ((int)blockIdx.x < attention_ctas(p)) {
+                        grid_arrive(p, sh, epoch);  // the activation is out; attention needs nothing from the others
+                        attention_phase(p, l, attn_scratch, sh);
+                        attn_signal(p, sh);
+                    } else {
+                        if (!(go = grid_sync(p, sh, epoch))) break;
+                        run_gemm<NT>(p, gs | (4 * l + 2), smem);               // MLP out -> x, beside the attention items
+                        run_gemm<NT>(p, gs | (4 * l + 3), smem);               // out-proj -> x, once the attention CTAs have signalled
+                    }
                     if (!(go = grid_sync(p, sh, epoch))) break;
-                    run_gemm<NT>(p, 4 * l + 2, smem);               // MLP out -> x, beside the attention items
-                    run_gemm<NT>(p, 4 * l + 3, smem);               // out-proj -> x, once the attention CTAs have signalled
+                } else if (p.parallel) {
+                    attention_phase(p, l, attn_scratch, sh);
+                    act_phase(p);
+                    if (!(go = grid_sync(p, sh, epoch))) break;
+                    run_gemm<NT>(p, gs | (4 * l + 2), smem);                   // out-proj -> x
+                    run_gemm<NT>(p, gs | (4 * l + 3), smem);                   // MLP out  -> x
+                    if (!(go = grid_sync(p, sh, epoch))) break;
+                } else {
+                    attention_phase(p, l, attn_scratch, sh);
+                    if (!(go = grid_sync(p, sh, epoch))) break;
+                    run_gemm<NT>(p, gs | (4 * l + 1), smem);                   // out-proj -> x
+                    if (!(go = grid_sync(p, sh, epoch))) break;
+                    const float *const *lt = staged_ltab(sh);
+                    const LayerDesc *ld = layer_desc(p.md, l);
+                    norm_phase(p, lt ? lt[8 * l + 4] : ld->ln2_g, lt ? lt[8 * l + 5] : ld->ln2_b, OP_XN1, nullptr, nullptr, 0, red);
+                    grid_zero(p.t_in, p.R, p.d_in, p.d_in);
+                    if (!(go = grid_sync(p, sh, epoch))) break;
+                    run_gemm<NT>(p, gs | (4 * l + 2), smem);                   // MLP in
+                    if (!(go = grid_sync(p, sh, epoch))) break;
+                    act_phase(p);
+                    if (!(go = grid_sync(p, sh, epoch))) break;
+                    run_gemm<NT>(p, gs | (4 * l + 3), smem);                   // MLP out -> x
+                    if (!(go = grid_sync(p, sh, epoch))) break;
                 }
-                if (!(go = grid_sync(p, sh, epoch))) break;
-            } else if (p.parallel) {
-                attention_phase(p, l, attn_scratch, sh);
-                act_phase(p);
-                if (!(go = grid_sync(p, sh, epoch))) break;
-                run_gemm<NT>(p, 4 * l + 2, smem);                   // out-proj -> x
-                run_gemm<NT>(p, 4 * l + 3, smem);                   // MLP out  -> x
-                if (!(go = grid_sync(p, sh, epoch))) break;
-            } else {
-                attention_phase(p, l, attn_scratch, sh);
-                if (!(go = grid_sync(p, sh, epoch))) break;
-                run_gemm<NT>(p, 4 * l + 1, smem);                   // out-proj -> x
-                if (!(go = grid_sync(p, sh, epoch))) break;
-                const float *const *lt = staged_ltab(sh);
-                const LayerDesc *ld = layer_desc(p.md, l);
-                norm_phase(p, lt ? lt[8 * l + 4] : ld->ln2_g, lt ? lt[8 * l + 5] : ld->ln2_b, OP_XN1, nullptr, nullptr, 0, red);
-                grid_zero(p.t_in, p.R, p.d_in, p.d_in);
-                if (!(go = grid_sync(p, sh, epoch))) break;
-                run_gemm<NT>(p, 4 * l + 2, smem);                   // MLP in
-                if (!(go = grid_sync(p, sh, epoch))) break;
-                act_phase(p);
-                if (!(go = grid_sync(p, sh, epoch))) break;
-                run_gemm<NT>(p, 4 * l + 3, smem);                   // MLP out -> x
+                norm_for_layer(l + 1);
                 if (!(go = grid_sync(p, sh, epoch))) break;
             }
-            norm_for_layer(l + 1);
-            if (!(go = grid_sync(p, sh, epoch))) break;
+            if (go && p.want_logits) run_gemm<NT>(p, gs | (4 * p.n_layers), smem);
+            if (go && p.tail) {  // q, the draw and the commit of this step (see tail_partial)
+                if (!(go = grid_sync(p, sh, epoch))) break;
+                tail_partial(p);
+                if (!(go = grid_sync(p, sh, epoch))) break;
+                tail_q(p);
+                if (!(go = grid_sync(p, sh, epoch))) break;
+                tail_draw(p);
+                if (!(go = grid_sync(p, sh, epoch))) break;
+                tail_commit(p);
+                if (!(go = grid_sync(p, sh, epoch))) break;
+            }
         }
-        if (go && p.want_logits) run_gemm<NT>(p, 4 * p.n_layers, smem);
+        if (go && p.tail && p.mailbox && blockIdx.x == 0 && threadIdx.x == 0) {  // the host's length bound follows (see report_max_len)
+            int m = 0;
+            for (int b = 0; b < p.B; ++b) m = max(m, __ldcg(p.len_rw + b));
+            *reinterpret_cast<volatile unsigned long long *>(p.mailbox) = ((unsigned long long)p.mb_seq << 32) | (unsigned)m;
+        }
         if (p.trace && blockIdx.x == 0 && threadIdx.x == 0) {
             unsigned long long t;
             asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));

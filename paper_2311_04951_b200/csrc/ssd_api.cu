@@ -265,6 +265,10 @@ struct Workspace {
     float *x, *qkv, *qrot, *t_in, *logits;
     RowStat *stats;
     RowFilter *filt;
+    // in-kernel tail of a draft loop: per (sequence, CTA) partials and the draws' meeting places
+    float *tp_m, *tp_s;
+    int32_t *tp_a, *tail_hit;
+    double *tp_mass;
     Operand xn1, xn2, ao, act;
     float *part_m, *part_l, *part_o;
     int max_split;
@@ -277,6 +281,20 @@ struct Workspace {
 };
 
 constexpr int kMaxSplit = 32;
+constexpr int kMaxCtas = 256;  // upper bound of the forward kernel's grid (one CTA per SM)
+
+// A draft loop: n_steps forwards in one launch, each ended inside the kernel (q, draw, commit).
+struct DraftLoop {
+    int n_steps;
+    float inv_t;
+    const float *u;
+    int u_stride;
+    int32_t *tok_out;
+    int tok_out_stride;
+    float *q_out;
+    size_t q_stride;
+    unsigned mb_seq;
+};
 constexpr int kTraceSlots = 1024;
 
 // Carve (or just size, base == nullptr) the workspace for B sequences x M rows.
@@ -311,6 +329,11 @@ Workspace carve(const ssd_model *m, int B, int M, uint8_t *base) {
     w.logits = (float *)take(sizeof(float) * (size_t)R * a.vocab);
     w.stats = (RowStat *)take(sizeof(RowStat) * R);
     w.filt = (RowFilter *)take(sizeof(RowFilter) * R);
+    w.tp_m = (float *)take(sizeof(float) * (size_t)B * kMaxCtas);
+    w.tp_s = (float *)take(sizeof(float) * (size_t)B * kMaxCtas);
+    w.tp_a = (int32_t *)take(sizeof(int32_t) * (size_t)B * kMaxCtas);
+    w.tp_mass = (double *)take(sizeof(double) * (size_t)B * kMaxCtas);
+    w.tail_hit = (int32_t *)take(sizeof(int32_t) * (size_t)kMaxRowsPerSeq * B * 2);
     // GEMM operands: hi rows [0, rows) then lo rows [rows, 2 rows) in one buffer; the stepwise path
     // pads rows to Rp, the single-kernel path to Rk (one allocation of 2 * Rk rows serves both)
     auto operand = [&](int ld, bool needed) {
@@ -549,7 +572,7 @@ int launch_forward_rows(const FwdParams &p, int rows_k, const void *ws_base, siz
 
 // The whole forward as one cooperative launch (bf16 models).
 int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int M, const int32_t *n_rows,
-                       bool want_logits, const Workspace &w, cudaStream_t st) {
+                       bool want_logits, const Workspace &w, cudaStream_t st, const DraftLoop *dl = nullptr) {
     const ssd_arch &a = m->a;
     FwdParams p;
     memset(&p, 0, sizeof(p));
@@ -597,7 +620,18 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     }
     p.want_logits = want_logits ? 1 : 0;
     p.wait_cycles = g_wait_cycles;
-    p.trace = (g_trace && 2 + barriers_needed(a) + 3 < kTraceSlots) ? w.trace : nullptr;
+    p.n_steps = 1;
+    if (dl) {
+        if (g_num_sms > kMaxCtas) return SSD_E_CAPACITY;
+        p.n_steps = dl->n_steps; p.tail = 1; p.inv_t = dl->inv_t;
+        p.u = dl->u; p.u_stride = dl->u_stride;
+        p.tok_out = dl->tok_out; p.tok_out_stride = dl->tok_out_stride;
+        p.q_out = dl->q_out; p.q_stride = dl->q_stride;
+        p.len_rw = kv->len;
+        p.tp_m = w.tp_m; p.tp_s = w.tp_s; p.tp_a = w.tp_a; p.tp_mass = w.tp_mass; p.tail_hit = w.tail_hit;
+        p.mailbox = kv->mailbox_dev; p.mb_seq = dl->mb_seq;
+    }
+    p.trace = (g_trace && 2 + p.n_steps * (barriers_needed(a) + 6) + 3 < kTraceSlots) ? w.trace : nullptr;
     CUDA_OK(cudaMemsetAsync(w.sync, 0, w.sync_bytes, st));
     cudaEvent_t prof_stop;
     if (prof_begin(st, &prof_stop)) return SSD_E_CUDA;
@@ -610,12 +644,16 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
 
 // One decoder forward over B x M rows against the cache.  Appends (does not commit) the rows'
 // keys/values; leaves logits in w.logits when want_logits.
+bool single_kernel_path(const ssd_model *m) {
+    const ssd_arch &a = m->a;
+    return a.dtype == 1 && g_persistent && m->dev_desc && a.head_dim % 16 == 0 &&
+           (a.pos == 0 || a.rotary_dim % 16 == 0);  // the MMA attention tiles heads by 16 and rotary halves by 8
+}
+
 int forward(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int M, const int32_t *n_rows,
             bool want_logits, const Workspace &w, cudaStream_t st) {
     const ssd_arch &a = m->a;
-    if (a.dtype == 1 && g_persistent && m->dev_desc && a.head_dim % 16 == 0 &&
-        (a.pos == 0 || a.rotary_dim % 16 == 0))  // the MMA attention tiles heads by 16 and rotary halves by 8
-        return forward_persistent(m, kv, tokens, tok_stride, M, n_rows, want_logits, w, st);
+    if (single_kernel_path(m)) return forward_persistent(m, kv, tokens, tok_stride, M, n_rows, want_logits, w, st);
     const int B = kv->B, R = B * M, d = a.d_model, F = a.d_ff;
     GemmCall gc{m, st, R, (R + 7) / 8 * 8};
     int rc = run_setup(m, kv, M, n_rows, w, st);
@@ -938,6 +976,44 @@ int draft_step(ssd_model *draft, ssd_kv *dkv, const int32_t *dev_tokens_in, int 
     const unsigned seq = kv_note_op(dkv, rows_in);
     LAUNCH(kv_commit_rows_kernel, 1, 64, 0, st, dkv->len, w.ri.n_eff, dkv->B, dkv->mailbox_dev, seq);
     return SSD_OK;
+}
+
+int draft_steps(ssd_model *draft, ssd_kv *dkv, int n_steps, const int32_t *dev_tokens_in, int tokens_stride, int rows_in,
+                const int32_t *dev_n_in, float temperature, const float *dev_u, int u_stride, int32_t *dev_tokens_out,
+                int token_out_stride, float *dev_q_out, size_t q_stride, void *dev_ws, size_t ws_bytes, void *stream) {
+    if (!draft || !dkv || !dev_tokens_in || !dev_u || !dev_tokens_out || !dev_q_out) return SSD_E_ARG;
+    if (n_steps < 1 || n_steps > kMaxRowsPerSeq || rows_in < 1 || rows_in > 2 || tokens_stride < rows_in ||
+        temperature < 0.f || token_out_stride < n_steps || u_stride < n_steps ||
+        q_stride < (size_t)n_steps * (size_t)draft->a.vocab)
+        return SSD_E_ARG;
+    if (!same_cache_shape(draft, dkv)) return SSD_E_ARG;
+    const bool restricted = g_top_k > 0 || (g_top_p > 0.f && g_top_p < 1.f);
+    if (!single_kernel_path(draft) || restricted) {
+        // the same steps, one call each (fp32 models, head dimensions the single kernel does not cover, or a
+        // sampling restriction, whose threshold search lives in the stand-alone tail kernel)
+        for (int s = 0; s < n_steps; ++s) {
+            const int rc = s == 0 ? draft_step(draft, dkv, dev_tokens_in, tokens_stride, rows_in, dev_n_in, temperature, dev_u,
+                                               u_stride, dev_tokens_out, token_out_stride, dev_q_out, q_stride, dev_ws,
+                                               ws_bytes, stream)
+                                  : draft_step(draft, dkv, dev_tokens_out + (s - 1), token_out_stride, 1, nullptr, temperature,
+                                               dev_u + s, u_stride, dev_tokens_out + s, token_out_stride,
+                                               dev_q_out + (size_t)s * draft->a.vocab, q_stride, dev_ws, ws_bytes, stream);
+            if (rc) return rc;
+        }
+        return SSD_OK;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    Workspace w;
+    int rc = check_ws(draft, dkv->B, rows_in, dev_ws, ws_bytes, &w);
+    if (rc) return rc;
+    DraftLoop dl;
+    dl.n_steps = n_steps;
+    dl.inv_t = temperature > 0.f ? 1.0f / temperature : 0.f;
+    dl.u = dev_u; dl.u_stride = u_stride;
+    dl.tok_out = dev_tokens_out; dl.tok_out_stride = token_out_stride;
+    dl.q_out = dev_q_out; dl.q_stride = q_stride;
+    dl.mb_seq = kv_note_op(dkv, rows_in + n_steps - 1);
+    return forward_persistent(draft, dkv, dev_tokens_in, tokens_stride, rows_in, dev_n_in, true, w, st, &dl);
 }
 
 size_t verify_scratch_bytes(int batch, int K) {

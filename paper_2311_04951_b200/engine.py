@@ -58,6 +58,7 @@ class Engine:
         self.target, self.draft = target, draft
         self.batch, self.max_len, self.K, self.T = batch, max_len, K, float(temperature)
         self.K_max = K
+        self.fused_draft = True   # draft loop as one draft_steps call (False: one draft_step call per token)
         V = target.arch.vocab
         dev = "cuda"
         self.tkv = B.KV(target, batch, max_len)
@@ -139,7 +140,10 @@ class Engine:
     def spec_iteration(self, u_draft: torch.Tensor, u_verify: torch.Tensor, p_debug: Optional[torch.Tensor] = None):
         K, V = self.K, self.target.arch.vocab
         us = u_draft.stride(0)
-        for i in range(K):
+        if self.fused_draft:  # the K draft steps as one call: tokens into columns 1.. of the row block, q rows into the q block
+            B.draft_steps(self.draft, self.dkv, K, self.draft_in, 2, 2, self.draft_n_in, self.T, u_draft, us,
+                          self.rows[:, 1:], K + 1, self.q, K * V, self.ws_d)
+        for i in range(0 if self.fused_draft else K):
             if i == 0:
                 tok_in, stride, rows_in, n_in = self.draft_in, 2, 2, self.draft_n_in
             else:
