@@ -300,6 +300,44 @@ def run_ours(args, rank, world):
     fwd_bytes = prof_steps * (verify_step_bytes(arch, Bn, K, p_lens) + K * draft_step_bytes)
     fwd_gbs = fwd_bytes / (fwd_ms * 1e-3) / 1e9 if fwd_ms > 0 else 0.0
 
+    # ---------------- the draft loop alone: one draft_step call per token, and all K steps in one launch ----------------
+    def time_draft(fused, reps):
+        d_eng = engine.Engine(target, draft, Bn, max_len, K, T, 8)
+        d_eng.copy_cache_from(eng)
+        d_eng.dkv.buf.copy_(eng.dkv.buf)
+        d_eng.draft_in.copy_(eng.draft_in)
+        d_eng.draft_n_in.fill_(1)
+        len0 = torch.from_numpy(d_eng.dkv.lengths()).cuda()
+        d_eng.fused_draft = fused
+        us = ud[0].stride(0)
+
+        def loop():
+            if fused:
+                B.draft_steps(draft, d_eng.dkv, K, d_eng.draft_in, 2, 2, d_eng.draft_n_in, T, ud[0], us,
+                              d_eng.rows[:, 1:], K + 1, d_eng.q, K * arch.vocab, d_eng.ws_d)
+            else:
+                for i in range(K):
+                    if i == 0:
+                        B.draft_step(draft, d_eng.dkv, d_eng.draft_in, 2, 2, d_eng.draft_n_in, T, ud[0], us,
+                                     d_eng.rows[:, 1:], K + 1, d_eng.q[:, 0], K * arch.vocab, d_eng.ws_d)
+                    else:
+                        B.draft_step(draft, d_eng.dkv, d_eng.rows[:, i:], K + 1, 1, None, T, ud[0][:, i:], us,
+                                     d_eng.rows[:, i + 1:], K + 1, d_eng.q[:, i], K * arch.vocab, d_eng.ws_d)
+            B.kv_rollback(d_eng.dkv, len0)     # the same context every time
+        for _ in range(2):
+            loop()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            loop()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps / K
+
+    draft_ms = {"per_token_calls_ms_per_step": time_draft(False, 5), "one_launch_ms_per_step": time_draft(True, 5),
+                "algorithmic_bytes_per_step": verify_step_bytes(draft.arch, Bn, 0, eng.dkv.lengths()) - Bn * 4}
+
     # ---------------- verification pass alone, and one-row decode, on the same cache ----------------
     def time_verify(k, reps, e):
         q = eng.q[:, :max(k, 1)].contiguous() if k else None
@@ -424,6 +462,7 @@ def run_ours(args, rank, world):
                         "tokens_per_iter": spec_tokens / (steps * Bn), "alpha": alpha,
                         "tokens_per_iter_closed_form": expected_tokens_per_iteration(alpha, K)},
         "autoregressive": {"tok_s": ar_tps, "ms_per_token": ar_ms / steps},
+        "draft_loop": draft_ms,
         "verify": {"ms": verify_ms, "rows": Bn * (K + 1), "bytes": v_bytes, "gbs": v_bytes / verify_ms / 1e6,
                    "frac_of_peak": v_bytes / verify_ms / 1e6 / peak,
                    "frac_of_8tbs": v_bytes / verify_ms / 1e6 / NOMINAL_HBM_GBS,

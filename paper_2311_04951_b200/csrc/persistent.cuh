@@ -1859,33 +1859,46 @@ __device__ __noinline__ void run_gemm(const FwdParams &p, int gi, uint8_t *smem)
 //      posted too (the fallback when rounding leaves no index past u S);
 // then CTA 0 writes the tokens and commits the rows fed in this step.
 __device__ __forceinline__ int tail_per(const FwdParams &p) { return (((p.V + (int)gridDim.x - 1) / (int)gridDim.x) + 3) & ~3; }
-__device__ __forceinline__ const float *tail_row(const FwdParams &p, int b) {
-    int row = __ldcg(p.ri.n_eff + b) - 1;
+__device__ __forceinline__ const float *tail_row(const FwdParams &p, const Shared *sh, int b) {
+    int row = (b < 64 ? staged_len(sh)[64 + b] : __ldcg(p.ri.n_eff + b)) - 1;  // (staged behind the step's first barrier)
     if (row < 0) row = 0;
     return p.logits + ((size_t)b * p.M + row) * p.V;
 }
 
-__device__ __noinline__ void tail_partial(const FwdParams &p) {
+// (All loops below fetch eight elements before they use the first: a load from L2 costs about a microsecond
+// under the weight stream, and a slice is only a few hundred elements.)
+__device__ __noinline__ void tail_partial(const FwdParams &p, const Shared *sh) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, G = (int)gridDim.x;
     const int per = tail_per(p), lo = min(p.V, (int)blockIdx.x * per), hi = min(p.V, lo + per);
     for (int b = warp; b < p.B; b += kConsumerWarps) {
-        const float *lg = tail_row(p, b);
-        float mx = -INFINITY;
+        const float *lg = tail_row(p, sh, b);
+        // running (max, argmax, sum of exp relative to the max) per lane, then over the warp
+        float mx = -INFINITY, sum = 0.f;
         int am = 0x7fffffff;
-        for (int j = lo + lane; j < hi; j += 32) {
-            const float l = __ldcg(lg + j);
-            if (l > mx) { mx = l; am = j; }  // ascending per lane: the first maximum
+        for (int jb = lo + lane; jb < hi; jb += 256) {
+            float l[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) l[u] = jb + 32 * u < hi ? __ldcg(lg + jb + 32 * u) : -INFINITY;
+            float m8 = mx;
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (l[u] > m8) { m8 = l[u]; am = jb + 32 * u; }  // ascending per lane: the first maximum
+            if (p.inv_t != 0.f && m8 > -INFINITY) {
+                sum *= expf((mx - m8) * p.inv_t);  // 0 while nothing has been summed
+#pragma unroll
+                for (int u = 0; u < 8; ++u) sum += expf((l[u] - m8) * p.inv_t);  // exp(-inf) = 0
+            }
+            mx = m8;
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, mx, o);
+            const float ov = __shfl_xor_sync(0xffffffffu, mx, o), os = __shfl_xor_sync(0xffffffffu, sum, o);
             const int oi = __shfl_xor_sync(0xffffffffu, am, o);
-            if (ov > mx || (ov == mx && oi < am)) { mx = ov; am = oi; }
+            const float m2 = fmaxf(mx, ov);
+            if (m2 > -INFINITY) sum = sum * expf((mx - m2) * p.inv_t) + os * expf((ov - m2) * p.inv_t);
+            if (ov > mx || (ov == mx && oi < am)) am = oi;
+            mx = m2;
         }
-        float sum = 0.f;
-        if (p.inv_t != 0.f && mx > -INFINITY)
-            for (int j = lo + lane; j < hi; j += 32) sum += expf((__ldcg(lg + j) - mx) * p.inv_t);
-        sum = warp_sum(sum);
         if (lane == 0) {
             p.tp_m[(size_t)b * G + blockIdx.x] = mx;
             p.tp_s[(size_t)b * G + blockIdx.x] = sum;
@@ -1897,13 +1910,20 @@ __device__ __noinline__ void tail_partial(const FwdParams &p) {
 // (max, argmax - lowest index among the maxima -, Z) of a sequence's row from the CTAs' partials; the same in every lane
 __device__ __forceinline__ void tail_stats(const FwdParams &p, int b, float &mx, int &am, float &z) {
     const int lane = threadIdx.x & 31, G = (int)gridDim.x;
+    float pm[8], ps[8];
+    int pa[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {  // (grids of up to 256 CTAs)
+        const int c = lane + 32 * k;
+        pm[k] = c < G ? __ldcg(p.tp_m + (size_t)b * G + c) : -INFINITY;
+        ps[k] = c < G ? __ldcg(p.tp_s + (size_t)b * G + c) : 0.f;
+        pa[k] = c < G ? __ldcg(p.tp_a + (size_t)b * G + c) : 0x7fffffff;
+    }
     mx = -INFINITY;
     am = 0x7fffffff;
-    for (int c = lane; c < G; c += 32) {
-        const float v = __ldcg(p.tp_m + (size_t)b * G + c);
-        const int i = __ldcg(p.tp_a + (size_t)b * G + c);
-        if (v > mx || (v == mx && i < am)) { mx = v; am = i; }
-    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+        if (pm[k] > mx || (pm[k] == mx && pa[k] < am)) { mx = pm[k]; am = pa[k]; }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         const float ov = __shfl_xor_sync(0xffffffffu, mx, o);
@@ -1911,11 +1931,11 @@ __device__ __forceinline__ void tail_stats(const FwdParams &p, int b, float &mx,
         if (ov > mx || (ov == mx && oi < am)) { mx = ov; am = oi; }
     }
     double zz = 0.0;
-    if (p.inv_t != 0.f)
-        for (int c = lane; c < G; c += 32) {
-            const float m = __ldcg(p.tp_m + (size_t)b * G + c);
-            if (m > -INFINITY) zz += (double)__ldcg(p.tp_s + (size_t)b * G + c) * (double)expf((m - mx) * p.inv_t);
-        }
+    if (p.inv_t != 0.f) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (pm[k] > -INFINITY) zz += (double)ps[k] * (double)expf((pm[k] - mx) * p.inv_t);
+    }
     zz = warp_sum(zz);
     z = (float)zz;
 }
@@ -1924,21 +1944,32 @@ __device__ __forceinline__ float tail_prob(float logit, float mx, int am, float 
     return expf((logit - mx) * inv_t) / z;
 }
 
-__device__ __noinline__ void tail_q(const FwdParams &p) {
+__device__ __noinline__ void tail_q(const FwdParams &p, const Shared *sh) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, G = (int)gridDim.x;
     const int per = tail_per(p), lo = min(p.V, (int)blockIdx.x * per), hi = min(p.V, lo + per);
     const int seg = (hi - lo + 31) / 32, j0 = min(hi, lo + lane * seg), j1 = min(hi, j0 + seg);
     for (int b = warp; b < p.B; b += kConsumerWarps) {
-        const float *lg = tail_row(p, b);
+        const float *lg = tail_row(p, sh, b);
+        float l[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) l[u] = j0 + u < j1 ? __ldcg(lg + j0 + u) : 0.f;  // (under the partials' latency)
         float mx, z;
         int am;
         tail_stats(p, b, mx, am, z);
         float *q = p.q_out + (size_t)b * p.q_stride + (size_t)p.cur_step * p.V;
         double local = 0.0;
-        for (int j = j0; j < j1; ++j) {
-            const float w = tail_prob(__ldcg(lg + j), mx, am, z, p.inv_t, j);
-            q[j] = w;
-            local += (double)w;
+        for (int jb = j0; jb < j1; jb += 8) {
+            if (jb > j0) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) l[u] = jb + u < j1 ? __ldcg(lg + jb + u) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (jb + u < j1) {
+                    const float w = tail_prob(l[u], mx, am, z, p.inv_t, jb + u);
+                    q[jb + u] = w;
+                    local += (double)w;
+                }
         }
         local = warp_sum(local);  // (a sum of at most 32 pieces: the order does not matter at fp64 for a decision that
         if (lane == 0) p.tp_mass[(size_t)b * G + blockIdx.x] = local;  //  is excused within 1e-6 S of a step anyway)
@@ -1950,20 +1981,32 @@ __device__ __noinline__ void tail_draw(const FwdParams &p) {
     const int per = tail_per(p), lo = min(p.V, (int)blockIdx.x * per), hi = min(p.V, lo + per);
     const int seg = (hi - lo + 31) / 32, j0 = min(hi, lo + lane * seg), j1 = min(hi, j0 + seg);
     for (int b = warp; b < p.B; b += kConsumerWarps) {
-        // prefix of the slice masses in CTA order (every lane walks all of them: G loads that overlap)
+        // total and this CTA's offset from the slice masses (lane l takes CTAs l, l + 32, ...; fp64)
         double off = 0.0, S = 0.0;
-        for (int c = 0; c < G; ++c) {
-            const double t = __ldcg(p.tp_mass + (size_t)b * G + c);
-            if (c < (int)blockIdx.x) off += t;
-            S += t;
+        {
+            double t[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) t[k] = lane + 32 * k < G ? __ldcg(p.tp_mass + (size_t)b * G + lane + 32 * k) : 0.0;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                S += t[k];
+                if (lane + 32 * k < (int)blockIdx.x) off += t[k];
+            }
+            S = warp_sum(S);
+            off = warp_sum(off);
         }
         const float *q = p.q_out + (size_t)b * p.q_stride + (size_t)p.cur_step * p.V;
         double local = 0.0;
         int last_pos = -1;
-        for (int j = j0; j < j1; ++j) {
-            const float w = q[j];  // written by this very lane in the phase before
-            local += (double)w;
-            if (w > 0.f) last_pos = j;
+        for (int jb = j0; jb < j1; jb += 8) {
+            float w[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) w[u] = jb + u < j1 ? __ldcg(q + jb + u) : 0.f;  // written by this very lane in the phase before
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                local += (double)w[u];
+                if (w[u] > 0.f) last_pos = jb + u;
+            }
         }
         double incl = local;
 #pragma unroll
@@ -1976,14 +2019,20 @@ __device__ __noinline__ void tail_draw(const FwdParams &p) {
         int hit = 0x7fffffff;
         if (S > 0.0 && (run + local > target || run > target)) {
             for (int j = j0; j < j1; ++j) {
-                const float w = q[j];
+                const float w = __ldcg(q + j);
                 run += (double)w;
                 if (w > 0.f && run > target) { hit = j; break; }  // a zero-weight index is never drawn
             }
         }
+        // one atomic per warp, not per lane: thousands of atomics on one word would serialise in L2
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            hit = min(hit, __shfl_xor_sync(0xffffffffu, hit, o));
+            last_pos = max(last_pos, __shfl_xor_sync(0xffffffffu, last_pos, o));
+        }
         int32_t *slot = p.tail_hit + ((size_t)p.cur_step * p.B + b) * 2;
-        if (hit != 0x7fffffff) atomicMin(slot, hit);
-        if (last_pos >= 0) atomicMax(slot + 1, last_pos);
+        if (lane == 0 && hit != 0x7fffffff) atomicMin(slot, hit);
+        if (lane == 0 && last_pos >= 0) atomicMax(slot + 1, last_pos);
     }
 }
 
@@ -2230,9 +2279,9 @@ __global__ void __launch_bounds__(kPersistThreads, 1) forward_kernel(const __gri
             if (go && p.want_logits) run_gemm<NT>(p, gs | (4 * p.n_layers), smem);
             if (go && p.tail) {  // q, the draw and the commit of this step (see tail_partial)
                 if (!(go = grid_sync(p, sh, epoch))) break;
-                tail_partial(p);
+                tail_partial(p, sh);
                 if (!(go = grid_sync(p, sh, epoch))) break;
-                tail_q(p);
+                tail_q(p, sh);
                 if (!(go = grid_sync(p, sh, epoch))) break;
                 tail_draw(p);
                 if (!(go = grid_sync(p, sh, epoch))) break;

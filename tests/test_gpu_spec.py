@@ -58,6 +58,7 @@ def test_lockstep_trajectories_per_family(name, arch, scale, K, T):
     ref = ospec.speculative_generate(otgt, odrf, prompt[0], n_new, K, T, lambda it: synth.gen_uniforms(23, 0, it, 2 * K + 1),
                                      160, keep_trace=True)
     eng = engine.Engine(tgt, drf, 1, 160, K, T, 128)
+    eng.fused_draft = name.endswith("natural_init") or name == "llama_bf16"   # both forms of the draft loop are exercised
     res = gu.lockstep(eng, synth, prompt[0], ref["iterations"], K, 23, ref["trace"],
                       peaky=bool(arch.dtype) and scale > 1.0)
     assert eng.tkv.status() == 0 and eng.dkv.status() == 0

@@ -235,3 +235,35 @@ def test_bf16_cache_rounding_is_applied_to_k_and_v_only():
     kv = c.kv[:, :, :, :5]
     rounded = torch.from_numpy(kv).bfloat16().float().numpy()
     assert np.array_equal(kv, rounded) and np.abs(kv).max() > 0
+
+
+@pytest.mark.parametrize("fam", ["gpt2", "llama"])
+def test_bf16_embedding_and_lm_head_reads(fam):
+    """bf16 matrices reach the oracle as uint16 bit patterns.  With every layer matrix and bias zeroed the
+    residual stream is the embedding row (+ learned position row), so the logits are
+    norm(E[tok] (+ P[pos])) . W_lm^T: written out here in float64 from the widened bit patterns, which pins the
+    bf16 branch of the embedding read, of the position table and of the LM head (tied and untied)."""
+    arch = synth.gpt2_like(2, 64, 4, 128, 97, 16, dtype=synth.DT_BF16) if fam == "gpt2" else synth.llama_like(2, 64, 2, 96, 97)
+    ws = synth.gen_weights(arch, 5)
+    for i, n in enumerate(synth.tensor_names(arch)):
+        base = n.split(".")[-1]
+        if "." in n and ws[i] is not None and not base.endswith("_g"):
+            ws[i] = np.zeros_like(ws[i])          # all layer matrices and biases (bf16 zero is the zero pattern)
+    toks = np.array([3, 96, 0, 41, 3], np.int32)
+    got = od.Model(arch, ws).forward_full(toks)
+    names = synth.tensor_names(arch)
+    f = lambda n: None if ws[names.index(n)] is None else (
+        synth.bf16_bits_to_f32(ws[names.index(n)]).astype(np.float64) if ws[names.index(n)].dtype == np.uint16
+        else ws[names.index(n)].astype(np.float64))
+    E, P, g, b = f("tok_emb"), f("pos_emb"), f("lnf_g"), f("lnf_b")
+    W = E if arch.tie_lm_head else f("w_lm")
+    for i, t in enumerate(toks):
+        x = E[t] + (P[i] if P is not None else 0.0)
+        x = x.astype(np.float32).astype(np.float64)            # the residual stream is stored in fp32
+        if arch.norm == synth.NORM_LAYERNORM:
+            y = (x - x.mean()) / np.sqrt(x.var() + arch.norm_eps) * g + b
+        else:
+            y = x / np.sqrt((x * x).mean() + arch.norm_eps) * g
+        ref = W @ y.astype(np.float32).astype(np.float64)
+        assert np.abs(got[i] - ref).max() <= 1e-5 * max(1.0, np.abs(ref).max()), (fam, i)
+    assert np.abs(got).max() > 1e-3
