@@ -133,6 +133,8 @@ void kv_destroy(ssd_kv *kv);
 /*
  * Functional (not tuned) prompt pass: feeds dev_tokens[b, 0 .. n_tokens[b]) of every sequence
  * (row stride max_tokens) in chunks and commits them, so the cache holds n_tokens[b] more rows.
+ * A chunk is as many rows per sequence as SSD_MAX_ROWS / batch, SSD_MAX_ROWS_PER_SEQ and the workspace
+ * allow (size the workspace with ssd_workspace_bytes for that many rows to get the fewest passes).
  * No logits are produced.  dev_n_tokens: int32 [batch] on the device, values <= max_tokens.
  * (Section "KV Caching", Figure 1: the pass that fills the cache before sampling starts.)
  */

@@ -938,11 +938,17 @@ int kv_prefill(ssd_model *m, ssd_kv *kv, const int32_t *dev_tokens, const int32_
     if (!same_cache_shape(m, kv)) return SSD_E_ARG;
     if (kv_bound(kv) + max_tokens > kv->S) return SSD_E_CAPACITY;
     cudaStream_t st = (cudaStream_t)stream;
+    // rows per sequence and pass: as many as the row limits and the caller's workspace allow (every pass streams
+    // all weights once, whatever its rows)
     int C = kMaxRows / kv->B;
-    if (C > 8) C = 8;
+    if (C > kMaxRowsPerSeq) C = kMaxRowsPerSeq;
     if (C < 1) return SSD_E_CAPACITY;
     Workspace w;
     int rc = check_ws(m, kv->B, C, dev_ws, ws_bytes, &w);
+    while (rc == SSD_E_CAPACITY && C > 1) {
+        C = C > 8 ? C / 2 : C - 1;
+        rc = check_ws(m, kv->B, C, dev_ws, ws_bytes, &w);
+    }
     if (rc) return rc;
     const int chunks = ceil_div(max_tokens, C);
     for (int c = 0; c < chunks; ++c) {

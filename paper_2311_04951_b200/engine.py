@@ -78,7 +78,7 @@ class Engine:
         self.out_cap = out_cap
         self.out_tokens = torch.zeros(batch, out_cap, dtype=torch.int32, device=dev)
         self.out_count = torch.zeros(batch, dtype=torch.int32, device=dev)
-        self.chunk = min(8, B.MAX_ROWS // batch)
+        self.chunk = min(B.MAX_ROWS_PER_SEQ, B.MAX_ROWS // batch)   # rows per sequence of a prompt-pass forward
         self.ws_pre_t = target.new_workspace(batch, self.chunk, max_len)
         if draft is not None and K > 0:
             self.dkv = B.KV(draft, batch, max_len)

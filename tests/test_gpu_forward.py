@@ -184,3 +184,39 @@ def test_row_counts_of_the_single_kernel_gemms(Bn, M):
         oc = omodel.new_cache(S)
         oc.feed(prompts[b], want_logits=False)
         gu.assert_logits_close(got[b], oc.feed(rows[b], advance=False))
+
+
+@pytest.mark.parametrize("name,Bn", [("llama_bf16", 2), ("neox_bf16", 1), ("gpt2_f32", 3)])
+def test_prompt_pass_in_large_chunks_matches_oracle(name, Bn):
+    """kv_prefill with a workspace for 32 (or 64 / batch) rows per sequence: chunks of up to 32 rows, two 16-row
+    attention tiles, ragged prompt lengths that end inside a chunk; cache rows and a following verification pass
+    against the oracle."""
+    arch = ARCHS[name]
+    ws_np = gu.scaled_weights(synth, arch, 3, 6.0)
+    omodel = od.Model(arch, ws_np)
+    model = B.Model(arch, B.upload_weights(arch, ws_np))
+    S, P = 96, 70
+    if arch.pos == 0:
+        S = P = min(S, arch.max_pos) - 8
+        S += 8
+    lens = np.array([P, P - 33, 5][:Bn], np.int32)
+    prompts = synth.gen_prompt(14, Bn, P, arch.vocab)
+    C = min(B.MAX_ROWS_PER_SEQ, B.MAX_ROWS // Bn)
+    kv = B.KV(model, Bn, S)
+    dev = "cuda"
+    B.kv_prefill(model, kv, torch.from_numpy(prompts).to(dev), torch.from_numpy(lens).to(dev), model.new_workspace(Bn, C, S))
+    assert kv.status() == 0 and kv.lengths().tolist() == lens.tolist()
+    rows = synth.gen_prompt(15, Bn, 3, arch.vocab)
+    got = gpu_logits(model, kv, model.new_workspace(Bn, 3, S), rows, 2)
+    cache = kv.cache_view().float().cpu().numpy()
+    for b in range(Bn):
+        oc = omodel.new_cache(S)
+        oc.feed(prompts[b, :lens[b]], want_logits=False)
+        gu.assert_logits_close(got[b], oc.feed(rows[b], advance=False))
+        n = int(lens[b])
+        g, r = cache[:, b, :, :, :n], oc.kv[:, :, :, :n]
+        # (layer-2 rows of these scaled-up models carry the bf16 roundings of two layers of cached keys / values, which
+        #  differ between 32-row and 1-row passes: the relative term is taken against the row's largest entry)
+        tol = gu.LOGIT_RTOL * np.abs(r).max(axis=-1, keepdims=True) + gu.LOGIT_ATOL if arch.dtype else 1e-4
+        bad = np.argwhere(np.abs(g - r) > tol)
+        assert bad.shape[0] == 0, (b, bad[:8].tolist(), [(float(g[tuple(i)]), float(r[tuple(i)])) for i in bad[:8]])
