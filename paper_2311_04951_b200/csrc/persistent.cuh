@@ -1170,7 +1170,8 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
 constexpr int kTcChunk = 128;
 constexpr int kTcStages = 4;  // K / V ring stages of 32 KB: the bytes in flight set the chunk rate (3 stages: 2.7 us per chunk)
 constexpr int kTcKvStage = kTcChunk * 128 * 2;  // one K or V chunk: two 64-column panels of 128 rows x 128 B
-constexpr int kTcQOff = kTcStages * kTcKvStage, kTcPOff = kTcQOff + 8192, kTcMiscOff = kTcPOff + 8192;
+constexpr int kTcPBytes = 8192;  // one P tile (16 hi + 16 lo rows x 128 positions, bf16); two of them, used in turn
+constexpr int kTcQOff = kTcStages * kTcKvStage, kTcPOff = kTcQOff + 8192, kTcMiscOff = kTcPOff + 2 * kTcPBytes;
 constexpr int kTcScratchBytes = kTcMiscOff + 1536 + kAttnRows * 128 * 4;  // + per-thread running sums [16][128]
 // Its mbarriers live outside the scratch (which the weight ring reuses), are initialised once per kernel
 // and keep running: cnt[i] = phases barrier i has completed before the current item.  A parity wait is
@@ -1178,7 +1179,12 @@ constexpr int kTcScratchBytes = kTcMiscOff + 1536 + kAttnRows * 128 * 4;  // + p
 // cannot pass by two phases; the threads that patch this pass's rows into a chunk skip most chunks, so
 // they do not wait on the ring's barriers: the MMA issuer, which follows every stage, tells them through
 // `landed` when such a chunk has arrived, and hears back through `fixed`.
-enum { AB_KV_FULL = 0, AB_KV_FREE = kTcStages, AB_S_FULL = 2 * kTcStages, AB_P_READY = AB_S_FULL + 2, AB_O_DONE, AB_FIXED, AB_LANDED, AB_COUNT };
+enum { AB_KV_FULL = 0, AB_KV_FREE = kTcStages, AB_S_FULL = 2 * kTcStages, AB_P_READY = AB_S_FULL + 2, AB_O_DONE /* two: chunk parity */,
+       AB_FIXED = AB_O_DONE + 2, AB_LANDED, AB_COUNT };
+// The running maximum of a row is only raised when a chunk's maximum exceeds it by more than this (log2 units):
+// P then stays below 2^8, the sums and O^T absorb it, and the dependent rescale of O^T - which has to wait for the
+// previous chunk's P V - becomes rare instead of happening in every other chunk.
+constexpr float kTcMaxSlack = 8.f;
 
 __device__ __forceinline__ void tc_ld_32(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
@@ -1295,7 +1301,9 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
 #pragma unroll
     for (int i = 0; i < kTcStages; ++i) { c_full[i] = acnt[AB_KV_FULL + i]; c_free[i] = acnt[AB_KV_FREE + i]; }
     const uint32_t c_s0 = acnt[AB_S_FULL], c_s1 = acnt[AB_S_FULL + 1];
-    const uint32_t c_p = acnt[AB_P_READY], c_o = acnt[AB_O_DONE], c_fix = acnt[AB_FIXED], c_land = acnt[AB_LANDED];
+    const uint32_t c_p = acnt[AB_P_READY], c_o0 = acnt[AB_O_DONE], c_o1 = acnt[AB_O_DONE + 1], c_fix = acnt[AB_FIXED], c_land = acnt[AB_LANDED];
+    // P V of chunk c completes phase c >> 1 of o_done[c & 1]
+    auto o_par = [&](int c) { return ((c & 1 ? c_o1 : c_o0) + (uint32_t)(c >> 1)) & 1u; };
     auto full_par = [&](int j) { return (c_full[j % kTcStages] + (uint32_t)(j / kTcStages)) & 1u; };          // stage j has landed
     auto free_par = [&](int j) { return ((c_free[j % kTcStages] + (uint32_t)(j / kTcStages)) & 1u) ^ 1u; };   // its slot was released
     int n_fix_total = 0;
@@ -1331,8 +1339,8 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
         uint8_t *panel = qt + (v8 >> 3) * 4096;
         *reinterpret_cast<uint4 *>(panel + sw128(ml, v8 & 7)) = *reinterpret_cast<uint4 *>(hq);
         *reinterpret_cast<uint4 *>(panel + sw128(16 + ml, v8 & 7)) = *reinterpret_cast<uint4 *>(lq);
-        reinterpret_cast<uint4 *>(pt)[2 * tid] = make_uint4(0, 0, 0, 0);
-        reinterpret_cast<uint4 *>(pt)[2 * tid + 1] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) reinterpret_cast<uint4 *>(pt)[4 * tid + i] = make_uint4(0, 0, 0, 0);  // both P tiles
     }
     fence_async_proxy();
     named_bar(3, kAttnThreadsP);
@@ -1391,8 +1399,8 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks)  // k = 16 positions per step: two 8-row groups of the V tile
                     tc_mma_bf16(tO, umma_desc(va + ks * 2048, kTcKvStage / 2, 1024),
-                                umma_desc(pa + (ks >> 2) * 4096 + (ks & 3) * 32, 16, 1024), idO, (c | ks) ? 1u : 0u);
-                tc_commit(o_done);
+                                umma_desc(pa + (c & 1) * kTcPBytes + (ks >> 2) * 4096 + (ks & 3) * 32, 16, 1024), idO, (c | ks) ? 1u : 0u);
+                tc_commit(&o_done[c & 1]);
                 tc_commit(&kv_free[jv % kTcStages]);
             }
         }
@@ -1491,12 +1499,9 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
                 }
             }
             named_bar(6, 128);
-            if (c > 0) {  // P V of the previous chunk has read the P tile and written O^T
-                wait(o_done, (c_o + c - 1) & 1u);
-                tc_fence_after();
-            }
+            if (c > 1) wait(&o_done[c & 1], o_par(c - 2));  // this chunk's P tile was last read by P V of chunk c - 2
             bool moved = false;
-            uint8_t *panel = pt + (tid >> 6) * 4096;
+            uint8_t *panel = pt + (c & 1) * kTcPBytes + (tid >> 6) * 4096;
             const int cc = (tid & 63) >> 3, e = (tid & 7) * 2;
 #pragma unroll 1
             for (int blk = 0; blk < nblk; ++blk) {
@@ -1512,7 +1517,8 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
                         const bool vis = pos < p_end && pos <= len + m_base + r;
                         const float v = vis ? (a[i] + b2[i]) * sc : -INFINITY;
                         const float mc = fmaxf(fmaxf(wmax[r], wmax[16 + r]), fmaxf(wmax[32 + r], wmax[48 + r]));
-                        const float m_old = wmrun[warp * 16 + r], m_new = fmaxf(m_old, mc);
+                        const float m_old = wmrun[warp * 16 + r];
+                        const float m_new = (mc > m_old + kTcMaxSlack || m_old == -INFINITY) ? fmaxf(m_old, mc) : m_old;
                         float pv = 0.f;
                         if (m_new > -INFINITY) {
                             fl[i] = exp2f(m_old - m_new);  // 0 on the first non-empty chunk
@@ -1541,7 +1547,9 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
                 }
             }
             __syncwarp();
-            if (c > 0 && moved) {  // thread = head dim tid: scale the accumulated O^T
+            if (c > 0 && moved) {  // thread = head dim tid: scale the accumulated O^T, once P V of the previous chunk has written it
+                wait(&o_done[(c - 1) & 1], o_par(c - 1));
+                tc_fence_after();
                 float o[32];
                 tc_ld_32(tO + lane_sel, o);
 #pragma unroll
@@ -1564,8 +1572,9 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
             for (int o = 16; o; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
             if (lane == 0) wsum[warp * 16 + r] = t;
         }
+        if (n_chunks > 1) wait(&o_done[(n_chunks - 2) & 1], o_par(n_chunks - 2));
         if (n_chunks > 0) {
-            wait(o_done, (c_o + n_chunks - 1) & 1u);
+            wait(&o_done[(n_chunks - 1) & 1], o_par(n_chunks - 1));
             tc_fence_after();
         }
         named_bar(6, 128);
@@ -1612,7 +1621,8 @@ __device__ __noinline__ void attention_item_tc(const FwdParams &p, int layer, in
         acnt[AB_S_FULL] = c_s0 + (uint32_t)((n_chunks + 1) / 2);
         acnt[AB_S_FULL + 1] = c_s1 + (uint32_t)(n_chunks / 2);
         acnt[AB_P_READY] = c_p + n_chunks;
-        acnt[AB_O_DONE] = c_o + n_chunks;
+        acnt[AB_O_DONE] = c_o0 + (uint32_t)((n_chunks + 1) / 2);
+        acnt[AB_O_DONE + 1] = c_o1 + (uint32_t)(n_chunks / 2);
         acnt[AB_FIXED] = c_fix + n_fix_total;
         acnt[AB_LANDED] = c_land + n_fix_total;
     }
