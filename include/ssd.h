@@ -92,6 +92,15 @@ int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n
  * fills it once with a synchronous copy; it must outlive the model and its layer-skip drafts. */
 size_t ssd_model_desc_bytes(const ssd_arch *arch);
 
+/* Workspace bytes of the many-row prompt pass for `batch` sequences x rows_per_seq rows per pass
+ * (rows_per_seq is cut to 8192 / batch); 0 when the model has no such pass (fp32 weights, a head
+ * dimension that is not a multiple of 16, widths that are not multiples of 8). */
+size_t ssd_prefill_workspace_bytes(const ssd_model *m, int batch, int rows_per_seq);
+
+/* Which form kv_prefill takes: 0 (default) the many-row form from 256 rows per pass, 1 never,
+ * 2 wherever the model and the workspace allow it (for tests on small shapes).  SSD_E_ARG otherwise. */
+int ssd_set_prefill_mode(int mode);
+
 /* bf16 models run the whole forward as one cooperative kernel by default; 0 selects one launch per
  * step instead (same results up to fp32 summation order; kept for comparison). */
 int ssd_set_persistent(int enable);
@@ -131,11 +140,22 @@ int kv_init(const ssd_model *m, int batch, int max_len, void *dev_buf, size_t by
 void kv_destroy(ssd_kv *kv);
 
 /*
- * Functional (not tuned) prompt pass: feeds dev_tokens[b, 0 .. n_tokens[b]) of every sequence
- * (row stride max_tokens) in chunks and commits them, so the cache holds n_tokens[b] more rows.
- * A chunk is as many rows per sequence as SSD_MAX_ROWS / batch, SSD_MAX_ROWS_PER_SEQ and the workspace
- * allow (size the workspace with ssd_workspace_bytes for that many rows to get the fewest passes).
- * No logits are produced.  dev_n_tokens: int32 [batch] on the device, values <= max_tokens.
+ * Prompt pass: feeds dev_tokens[b, 0 .. n_tokens[b]) of every sequence (row stride max_tokens) and
+ * commits them, so the cache holds n_tokens[b] more rows.  No logits are produced.
+ * dev_n_tokens: int32 [batch] on the device, values <= max_tokens.
+ * Two forms, chosen by the workspace the caller passes:
+ *  - bf16 models whose workspace holds ssd_prefill_workspace_bytes(m, batch, c) for some c with
+ *    batch * c >= 256 rows take the many-row form: equal passes of up to 8192 / batch rows per sequence
+ *    (the largest the workspace fits), every linear layer as a tiled tcgen05 GEMM over 128 rows x 256
+ *    weight rows per CTA with the activations as bf16 hi + lo, causal attention over 64-row tiles
+ *    against the cache.  Compute-bound; the arithmetic is that of the few-row passes up to fp32
+ *    summation order.
+ *  - otherwise chunks through the few-row forward: as many rows per sequence as SSD_MAX_ROWS / batch,
+ *    SSD_MAX_ROWS_PER_SEQ and the workspace allow (size it with ssd_workspace_bytes for that many rows
+ *    to get the fewest passes); every pass streams all weights once.
+ * Errors as the forward passes: SSD_E_CAPACITY when the prompt does not fit the cache or the workspace
+ * holds not even a one-row pass; device-side conditions (a sequence that does not fit, a wait that ran
+ * out) through the cache's status word.
  * (Section "KV Caching", Figure 1: the pass that fills the cache before sampling starts.)
  */
 int kv_prefill(ssd_model *m, ssd_kv *kv, const int32_t *dev_tokens, const int32_t *dev_n_tokens, int max_tokens,

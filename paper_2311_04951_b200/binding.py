@@ -38,7 +38,8 @@ EXPORTS = ["ssd_model_create", "ssd_model_desc_bytes", "ssd_set_persistent", "ss
            "ssd_workspace_bytes", "kv_init", "kv_destroy", "kv_prefill", "draft_step", "target_verify",
            "kv_commit", "kv_rollback", "spec_advance", "kv_lengths", "ssd_device_status",
            "verify_from_logits", "verify_from_logits_noalloc", "verify_scratch_bytes", "attention_rows", "ssd_last_logits", "ssd_set_trace", "ssd_read_trace", "ssd_launch_count",
-           "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror", "ssd_set_wait_limit", "ssd_wait_probe", "ssd_set_sampling", "draft_steps"]
+           "ssd_gemm_profile", "ssd_gemm_profile_read", "ssd_strerror", "ssd_set_wait_limit", "ssd_wait_probe", "ssd_set_sampling", "draft_steps",
+           "ssd_prefill_workspace_bytes", "ssd_set_prefill_mode"]
 
 
 def lib_path() -> str:
@@ -62,6 +63,9 @@ def load():
     L.ssd_model_desc_bytes.restype = sz
     L.ssd_set_persistent.argtypes = [i32]
     L.ssd_set_attention_mode.argtypes = [i32]
+    L.ssd_set_prefill_mode.argtypes = [i32]
+    L.ssd_prefill_workspace_bytes.argtypes = [vp, i32, i32]
+    L.ssd_prefill_workspace_bytes.restype = sz
     L.ssd_model_share_prefix.argtypes = [vp, i32, pp]
     L.ssd_model_destroy.argtypes = [vp]
     L.ssd_model_destroy.restype = None
@@ -173,6 +177,10 @@ class Model:
 
     def workspace_bytes(self, batch: int, rows_per_seq: int, max_len: int) -> int:
         return int(load().ssd_workspace_bytes(self.h, batch, rows_per_seq, max_len))
+
+    def prefill_workspace_bytes(self, batch: int, rows_per_seq: int) -> int:
+        """Workspace of the many-row prompt pass (0: this model has none)."""
+        return int(load().ssd_prefill_workspace_bytes(self.h, batch, rows_per_seq))
 
     def new_workspace(self, batch: int, rows_per_seq: int, max_len: int) -> torch.Tensor:
         n = self.workspace_bytes(batch, rows_per_seq, max_len)
@@ -329,6 +337,11 @@ def set_persistent(enable: bool) -> None:
 def set_attention_mode(mode: int) -> None:
     """0: per pass (default); 1: warp-MMA attention items; 2: tensor-core items wherever they apply."""
     _check(load().ssd_set_attention_mode(int(mode)), "ssd_set_attention_mode")
+
+
+def set_prefill_mode(mode: int) -> None:
+    """0: many-row prompt pass from 256 rows per pass (default); 1: never; 2: wherever it applies."""
+    _check(load().ssd_set_prefill_mode(int(mode)), "ssd_set_prefill_mode")
 
 
 def set_trace(enable: bool) -> None:

@@ -1,0 +1,373 @@
+// Prompt pass over many rows at once (Section "KV Caching", Figure 1: the pass that fills the cache before
+// sampling starts).  With hundreds or thousands of rows per forward the linear layers are compute-bound: this
+// file holds the two kernels that differ from the few-row path - a tiled tcgen05 GEMM over 128 activation rows
+// x 256 weight rows per CTA, and a causal attention over row tiles whose keys / values all sit in the cache -
+// the row-wise steps (set-up, embedding, norms, activation, rotary + append) are the stepwise path's kernels,
+// which take any number of rows.
+//
+// prefill_gemm_kernel:  out[r, n] += sum_k (Xhi[r, k] + Xlo[r, k]) * W[n, k]
+//   * one CTA per (128-row, 256-column) output tile, 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer,
+//     warps 2-5 = epilogue (one tensor-memory lane quadrant each);
+//   * a stage of the shared-memory ring = the activation rows' hi tile and lo tile (128 rows x 64 k, bf16) and
+//     the weight tile (256 rows x 64 k), all by 2-D tensor-map copies with the 128-byte swizzle, 64 KB;
+//   * per stage eight tcgen05.mma (M = 128, N = 256, K = 16): four k-steps with the hi tile, four with the lo
+//     tile, into ONE fp32 accumulator in tensor memory: W hi + W lo is the fp32-activation product to ~2^-17,
+//     the same arithmetic as the few-row path (the price is half the tensor throughput);
+//   * the tile is owned by this CTA alone (no split over k), so the epilogue adds the accumulator to the
+//     output with plain loads and stores.
+// Every wait is bounded; on time-out the kernel records SSD_E_TIMEOUT, drains its copies and returns.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+#include "gemm.cuh"
+#include "persistent.cuh"
+
+namespace ssd {
+
+constexpr int kPfTileM = 128, kPfTileN = 256, kPfStages = 3;
+constexpr int kPfABytes = kPfTileM * kTileK * 2;            // 16 KB: one of hi / lo
+constexpr int kPfWBytes = kPfTileN * kTileK * 2;            // 32 KB
+constexpr int kPfStageBytes = 2 * kPfABytes + kPfWBytes;    // 64 KB
+constexpr int kPfThreads = 192;
+constexpr size_t kPfSmem = 1024 + (size_t)kPfStages * kPfStageBytes + 256;
+
+struct PfGemmArgs {
+    float *out;  // [R, ldo] fp32, accumulated into
+    int ldo, N, Kd, R;
+    long long wait_cycles;  // bound of every wait that takes work
+    int32_t *status;
+};
+
+__global__ void __launch_bounds__(kPfThreads, 1)
+prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmXhi,
+                    const __grid_constant__ CUtensorMap tmXlo, const PfGemmArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t *full = (uint64_t *)(smem + (size_t)kPfStages * kPfStageBytes);
+    uint64_t *empty = full + kPfStages;
+    uint64_t *acc_full = empty + kPfStages;
+    uint32_t *tmem_slot = (uint32_t *)(acc_full + 1);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.y * kPfTileM, n0 = blockIdx.x * kPfTileN;
+    const int kchunks = (a.Kd + kTileK - 1) / kTileK;
+
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(256)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPfStages; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(acc_full, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    int issued = 0;
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kc = 0; kc < kchunks; ++kc, ++issued) {
+                const int s = kc % kPfStages;
+                if (kc >= kPfStages && !mbar_wait_limit(&empty[s], ((kc / kPfStages) - 1) & 1, a.wait_cycles)) {
+                    set_status(a.status, kTimeoutCode);
+                    *abort_flag = 1;
+                    break;
+                }
+                if (*abort_flag) break;
+                uint8_t *st = smem + (size_t)s * kPfStageBytes;
+                mbar_expect_tx(&full[s], kPfStageBytes);
+                tma_load_2d(st, &tmXhi, kc * kTileK, m0, &full[s]);
+                tma_load_2d(st + kPfABytes, &tmXlo, kc * kTileK, m0, &full[s]);
+                tma_load_2d(st + 2 * kPfABytes, &tmW, kc * kTileK, n0, &full[s]);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16(kPfTileM, kPfTileN);
+            bool ok = true;
+            for (int kc = 0; kc < kchunks; ++kc) {
+                const int s = kc % kPfStages;
+                if (*abort_flag || !mbar_wait_limit(&full[s], (kc / kPfStages) & 1, a.wait_cycles)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t st = smem_u32(smem + (size_t)s * kPfStageBytes);
+                const uint64_t hi = umma_desc_sw128(st), lo = umma_desc_sw128(st + kPfABytes), w = umma_desc_sw128(st + 2 * kPfABytes);
+#pragma unroll
+                for (int ks = 0; ks < kTileK / 16; ++ks) tc_mma_bf16(tmem, hi + 2 * ks, w + 2 * ks, idesc, (kc | ks) ? 1u : 0u);
+#pragma unroll
+                for (int ks = 0; ks < kTileK / 16; ++ks) tc_mma_bf16(tmem, lo + 2 * ks, w + 2 * ks, idesc, 1u);
+                tc_commit(&empty[s]);
+            }
+            if (!ok) {
+                set_status(a.status, kTimeoutCode);
+                *abort_flag = 1;
+            }
+            tc_commit(acc_full);  // (arrives once everything issued so far has completed: also on the error path)
+        }
+        __syncwarp();
+    } else {
+        // epilogue: accumulator row r sits in tensor-memory lane r; warp w reaches lanes 32 (w % 4) ..
+        const int quad = warp & 3, row = m0 + quad * 32 + lane;
+        const bool landed = mbar_wait_limit(acc_full, 0, 4 * a.wait_cycles);
+        if (!landed) set_status(a.status, kTimeoutCode);
+        tc_fence_after();
+        if (__all_sync(0xffffffffu, landed && !*abort_flag)) {  // (the tensor-memory loads are warp-wide)
+            float *orow = a.out + (size_t)row * a.ldo + n0;
+            const bool vec = ((uintptr_t)a.out & 15) == 0 && (a.ldo & 3) == 0;
+#pragma unroll 1
+            for (int cb = 0; cb < kPfTileN / 32; ++cb) {
+                if (n0 + cb * 32 >= a.N) break;
+                float v[32];
+                tc_ld_32(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cb * 32), v);
+                if (row < a.R) {
+                    if (vec && n0 + cb * 32 + 31 < a.N) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            float4 o = *reinterpret_cast<float4 *>(orow + cb * 32 + 4 * i);
+                            o.x += v[4 * i]; o.y += v[4 * i + 1]; o.z += v[4 * i + 2]; o.w += v[4 * i + 3];
+                            *reinterpret_cast<float4 *>(orow + cb * 32 + 4 * i) = o;
+                        }
+                    } else {
+                        for (int i = 0; i < 32; ++i)
+                            if (n0 + cb * 32 + i < a.N) orow[cb * 32 + i] += v[i];
+                    }
+                }
+            }
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 0) {
+        if (lane == 0 && *abort_flag)  // error path only: copies that may still land in this CTA's shared memory
+            for (int i = (issued > kPfStages ? issued - kPfStages : 0); i < issued; ++i) mbar_wait(&full[i % kPfStages], (i / kPfStages) & 1);
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(256) : "memory");
+    }
+}
+
+// x[r, :] += bias  (the out-projection's bias, before that projection accumulates into the residual stream)
+__global__ void add_bias_kernel(float *x, const float *bias, int d) {
+    if (!bias) return;
+    float *row = x + (size_t)blockIdx.x * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) row[i] += bias[i];
+}
+
+// prefill_attn_kernel: causal attention of 64 query rows of one (sequence, head) over the cache, which already
+// holds this pass's keys / values (the append kernel has run).  Four warps of 16 rows each; K / V chunks of 64
+// positions go through two cp.async buffers shared by the four warps; per warp and chunk
+//   S [16 x 64] = Q (bf16 hi + lo) K^T,   running max / sum in registers (base-2 exponentials),
+//   O [16 x Dh] += P (bf16 hi + lo) V,
+// on mma.sync tiles (m16n8k16): the projections carry ~95 % of a prompt pass's arithmetic, so this step stays on
+// the warp-level path.  Row m of the sequence sees positions <= len + m.  The result goes to the out-projection
+// operand as bf16 hi + lo, row-major; rows that are not fed get zeros.
+constexpr int kPaRows = 64, kPaThreads = 128, kPaChunk = 64;
+inline size_t prefill_attn_smem(int Dh) {
+    return (size_t)2 * kPaRows * (Dh + 8) * 2 + (size_t)2 * 2 * kPaChunk * (Dh + 8) * 2;
+}
+
+struct PfAttnArgs {
+    const float *q;              // [B * M, d] position-encoded queries
+    const __nv_bfloat16 *cache;  // this layer's slab [B][2][H][S][Dh]
+    const int32_t *len;          // [B] committed lengths
+    const int32_t *n_eff;        // [B] rows fed per sequence
+    __nv_bfloat16 *out_hi, *out_lo;  // [B * M, d]
+    int M, H, Dh, S, d;
+    float scale;
+};
+
+__global__ void __launch_bounds__(kPaThreads) prefill_attn_kernel(const PfAttnArgs a) {
+    extern __shared__ __align__(16) uint8_t pa_smem[];
+    const int mt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int Dh = a.Dh, pitch = Dh + 8;
+    const uint32_t pitchB = (uint32_t)pitch * 2u;
+    __nv_bfloat16 *Qhi = reinterpret_cast<__nv_bfloat16 *>(pa_smem);
+    __nv_bfloat16 *Qlo = Qhi + kPaRows * pitch;
+    __nv_bfloat16 *KV = Qlo + kPaRows * pitch;  // buffer i: K at KV + i * 2 * 64 * pitch, V 64 * pitch later
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
+    const int nk = Dh >> 4, vpr = Dh >> 3;
+    const int len = a.len[b], n = a.n_eff[b];
+    const int m_base = mt * kPaRows, r0 = b * a.M;
+    const int rows_fed = max(0, min(kPaRows, n - m_base));
+    const int p_end = rows_fed > 0 ? min(len + m_base + rows_fed, a.S) : 0;  // positions any row of this tile sees
+    const int n_chunks = (p_end + kPaChunk - 1) / kPaChunk;
+    const float sc = a.scale * 1.4426950408889634f;
+    const __nv_bfloat16 *kc = a.cache + ((size_t)(b * 2) * a.H + h) * a.S * Dh;
+    const __nv_bfloat16 *vc = kc + (size_t)a.H * a.S * Dh;
+
+    auto load_chunk = [&](int c) {
+        __nv_bfloat16 *Kb = KV + (size_t)(c & 1) * 2 * kPaChunk * pitch, *Vb = Kb + kPaChunk * pitch;
+        const int t0 = c * kPaChunk;
+        for (int i = tid; i < kPaChunk * vpr; i += kPaThreads) {
+            const int pp = i / vpr, v8 = i % vpr, pos = t0 + pp;
+            __nv_bfloat16 *dk = Kb + pp * pitch + v8 * 8, *dv = Vb + pp * pitch + v8 * 8;
+            if (pos < p_end) {
+                cp_async16(dk, kc + (size_t)pos * Dh + v8 * 8);
+                cp_async16(dv, vc + (size_t)pos * Dh + v8 * 8);
+            } else {  // masked positions: P is 0 there, and 0 x these zeros stays 0
+                *reinterpret_cast<uint4 *>(dk) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4 *>(dv) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        cp_async_commit();
+    };
+    if (n_chunks > 0) load_chunk(0);
+    // Q rows of this tile as bf16 hi / lo
+    for (int i = tid; i < kPaRows * vpr; i += kPaThreads) {
+        const int ml = i / vpr, v8 = i % vpr, m = m_base + ml;
+        float qv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) qv[u] = 0.f;
+        if (m < n) {
+            const float *src = a.q + (size_t)(r0 + m) * a.d + h * Dh + v8 * 8;
+            const float4 x0 = *reinterpret_cast<const float4 *>(src), x1 = *reinterpret_cast<const float4 *>(src + 4);
+            qv[0] = x0.x; qv[1] = x0.y; qv[2] = x0.z; qv[3] = x0.w; qv[4] = x1.x; qv[5] = x1.y; qv[6] = x1.z; qv[7] = x1.w;
+        }
+        __nv_bfloat16 hq[8], lq[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            hq[u] = __float2bfloat16_rn(qv[u]);
+            lq[u] = __float2bfloat16_rn(qv[u] - __bfloat162float(hq[u]));
+        }
+        *reinterpret_cast<uint4 *>(Qhi + ml * pitch + v8 * 8) = *reinterpret_cast<uint4 *>(hq);
+        *reinterpret_cast<uint4 *>(Qlo + ml * pitch + v8 * 8) = *reinterpret_cast<uint4 *>(lq);
+    }
+
+    float o[16][4];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    const int row_lo = m_base + 16 * warp;           // this warp's rows: row_lo + g, row_lo + g + 8
+    const int warp_end = len + row_lo + 15;           // last position any of them sees
+
+    for (int c = 0; c < n_chunks; ++c) {
+        if (c + 1 < n_chunks) load_chunk(c + 1); else cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();  // chunk c (and, first time, Q) is in shared memory
+        const int t0 = c * kPaChunk;
+        if (t0 <= warp_end && row_lo < n) {
+            const __nv_bfloat16 *Kb = KV + (size_t)(c & 1) * 2 * kPaChunk * pitch, *Vb = Kb + kPaChunk * pitch;
+            float s[8][4];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+            const uint32_t qa = smem_u32(Qhi) + (uint32_t)(16 * warp + (lane & 15)) * pitchB + (uint32_t)(lane >> 4) * 16u;
+            const uint32_t ql = qa + (uint32_t)kPaRows * pitchB;
+            const uint32_t ka = smem_u32(Kb) + (uint32_t)((lane & 7) + 8 * (lane >> 4)) * pitchB + (uint32_t)((lane >> 3) & 1) * 16u;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                if (ks < nk) {
+                    uint32_t a0, a1, a2, a3, c0, c1, c2, c3;
+                    ldmatrix_x4(qa + ks * 32, a0, a1, a2, a3);
+                    ldmatrix_x4(ql + ks * 32, c0, c1, c2, c3);
+#pragma unroll
+                    for (int j2 = 0; j2 < 4; ++j2) {  // 16 positions: (0-7: k lo, k hi), (8-15: k lo, k hi)
+                        uint32_t k0, k1, k2, k3;
+                        ldmatrix_x4(ka + (uint32_t)(16 * j2) * pitchB + ks * 32, k0, k1, k2, k3);
+                        mma_bf16(s[2 * j2], a0, a1, a2, a3, k0, k1);
+                        mma_bf16(s[2 * j2], c0, c1, c2, c3, k0, k1);
+                        mma_bf16(s[2 * j2 + 1], a0, a1, a2, a3, k2, k3);
+                        mma_bf16(s[2 * j2 + 1], c0, c1, c2, c3, k2, k3);
+                    }
+                }
+            }
+            // mask, running max / sum (rows g and g + 8)
+#pragma unroll
+            for (int hrow = 0; hrow < 2; ++hrow) {
+                const int m = row_lo + g + 8 * hrow;
+                const int last = m < n ? len + m : -1;  // last visible position
+                float mx = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int pos = t0 + 8 * j + 2 * t + e;
+                        const float v = pos <= last ? s[j][2 * hrow + e] * sc : -INFINITY;
+                        s[j][2 * hrow + e] = v;
+                        mx = fmaxf(mx, v);
+                    }
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float m_new = fmaxf(m_run[hrow], mx);
+                float f = 1.f, sum = 0.f;
+                if (m_new > -INFINITY) {
+                    f = exp2f(m_run[hrow] - m_new);  // 0 on the first non-empty block
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const float pv = exp2f(s[j][2 * hrow + e] - m_new);
+                            s[j][2 * hrow + e] = pv;
+                            sum += pv;
+                        }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) s[j][2 * hrow] = s[j][2 * hrow + 1] = 0.f;
+                }
+                m_run[hrow] = m_new;
+                l_run[hrow] = l_run[hrow] * f + sum;  // this thread's share; lanes are summed at the end
+#pragma unroll
+                for (int j = 0; j < 16; ++j) { o[j][2 * hrow] *= f; o[j][2 * hrow + 1] *= f; }
+            }
+            // O += P V: k = 16 positions per step, n = the head's columns
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                uint32_t ph[4], pl[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {  // a0: (row g, k 2t..) a1: (row g+8, ..) a2: (row g, k 8+2t..) a3: (row g+8, ..)
+                    const int j = 2 * kk + (q >> 1), hrow = q & 1;
+                    const float x0 = s[j][2 * hrow], x1 = s[j][2 * hrow + 1];
+                    const __nv_bfloat162 hv = __floats2bfloat162_rn(x0, x1);
+                    ph[q] = *reinterpret_cast<const uint32_t *>(&hv);
+                    pl[q] = pack_bf16x2(x0 - __low2float(hv), x1 - __high2float(hv));
+                }
+                const uint32_t va = smem_u32(Vb) + (uint32_t)(16 * kk + (lane & 15)) * pitchB;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    if (j < 2 * nk) {
+                        uint32_t b0, b1;
+                        ldmatrix_x2_trans(va + j * 16, b0, b1);
+                        mma_bf16(o[j], ph[0], ph[1], ph[2], ph[3], b0, b1);
+                        mma_bf16(o[j], pl[0], pl[1], pl[2], pl[3], b0, b1);
+                    }
+                }
+            }
+        }
+        __syncthreads();  // everyone is done with this buffer before it is refilled
+    }
+    cp_async_wait<0>();
+    // output: rows g, g + 8 of this warp; columns 8 j + 2 t, + 1
+#pragma unroll
+    for (int hrow = 0; hrow < 2; ++hrow) {
+        float L = l_run[hrow];
+        L += __shfl_xor_sync(0xffffffffu, L, 1);
+        L += __shfl_xor_sync(0xffffffffu, L, 2);
+        const int m = row_lo + g + 8 * hrow;
+        if (m >= a.M) continue;
+        const float inv = (m < n && L > 0.f) ? 1.f / L : 0.f;
+        const size_t base = (size_t)(r0 + m) * a.d + h * Dh + 2 * t;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            if (j < 2 * nk) {
+                const float y0 = o[j][2 * hrow] * inv, y1 = o[j][2 * hrow + 1] * inv;
+                const __nv_bfloat162 hv = __floats2bfloat162_rn(y0, y1);
+                const __nv_bfloat162 lv = __floats2bfloat162_rn(y0 - __low2float(hv), y1 - __high2float(hv));
+                *reinterpret_cast<__nv_bfloat162 *>(a.out_hi + base + 8 * j) = hv;
+                *reinterpret_cast<__nv_bfloat162 *>(a.out_lo + base + 8 * j) = lv;
+            }
+        }
+    }
+}
+
+}  // namespace ssd

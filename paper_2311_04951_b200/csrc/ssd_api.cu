@@ -18,6 +18,7 @@
 #include "persistent.cuh"
 #include "rowops.cuh"
 #include "tail.cuh"
+#include "prefill.cuh"
 
 using namespace ssd;
 
@@ -36,6 +37,7 @@ int g_attn_mode = 0;       // 0: choose per pass; 1: warp-MMA attention items; 2
 bool g_trace = false;       // stamp the global timer after every grid barrier of the forward kernel
 int g_top_k = 0;           // restriction of both models' distributions before sampling / verification (0: none)
 float g_top_p = 1.0f;      // (1: none)
+int g_prefill_mode = 0;    // 0: many-row prompt pass where it pays; 1: never; 2: wherever the model allows it
 long long g_wait_cycles = 0;  // 0: the kernels' default bound (about two seconds) on every wait that takes work
 bool g_prof = false;
 std::vector<cudaEvent_t> g_prof_events;  // pairs
@@ -161,6 +163,8 @@ int init_device_once() {
     rc |= set_smem(attn_partial_kernel<__nv_bfloat16, 8>, attn_smem<__nv_bfloat16, 8>(128));
     rc |= set_smem(attn_partial_kernel<__nv_bfloat16, 16>, attn_smem<__nv_bfloat16, 16>(128));
     rc |= set_smem(attn_partial_kernel<__nv_bfloat16, 32>, attn_smem<__nv_bfloat16, 32>(128));
+    rc |= set_smem(prefill_gemm_kernel, kPfSmem);
+    rc |= set_smem(prefill_attn_kernel, prefill_attn_smem(128));
     if (rc) return SSD_E_CUDA;
     g_attr_done = true;
     return SSD_OK;
@@ -173,6 +177,7 @@ struct ssd_model {
     ssd_arch a;
     std::vector<const void *> w;  // 2 + 12 L + 3 tensors
     std::vector<CUtensorMap> tm;  // bf16 models: per layer {qkv, o, in, out}, then lm head
+    std::vector<CUtensorMap> tm256;  // the same four per layer with 256-row boxes (many-row prompt pass)
     int d_in;
     const ModelDesc *dev_desc;    // bf16 models: the same maps + vector pointers in device memory (caller-owned)
 };
@@ -232,8 +237,13 @@ int build_maps(ssd_model *m) {
     if (m->a.dtype != 1) return SSD_OK;
     const ssd_arch &a = m->a;
     m->tm.resize((size_t)4 * a.n_layers + 1);
+    m->tm256.resize((size_t)4 * a.n_layers);
     for (int l = 0; l < a.n_layers; ++l) {
         int rc = 0;
+        rc |= make_map(&m->tm256[4 * l + 0], lw(m, l, L_WQKV), 3 * a.d_model, a.d_model, kPfTileN);
+        rc |= make_map(&m->tm256[4 * l + 1], lw(m, l, L_WO), a.d_model, a.d_model, kPfTileN);
+        rc |= make_map(&m->tm256[4 * l + 2], lw(m, l, L_WIN), m->d_in, a.d_model, kPfTileN);
+        rc |= make_map(&m->tm256[4 * l + 3], lw(m, l, L_WOUT), a.d_model, a.d_ff, kPfTileN);
         rc |= make_map(&m->tm[4 * l + 0], lw(m, l, L_WQKV), 3 * a.d_model, a.d_model, kTileN);
         rc |= make_map(&m->tm[4 * l + 1], lw(m, l, L_WO), a.d_model, a.d_model, kTileN);
         rc |= make_map(&m->tm[4 * l + 2], lw(m, l, L_WIN), m->d_in, a.d_model, kTileN);
@@ -740,6 +750,157 @@ int forward(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int
     return SSD_OK;
 }
 
+
+// ---- prompt pass over many rows (bf16 models) --------------------------------------------------
+constexpr int kWideMaxRows = 8192;  // rows of one many-row pass (sequences x rows per sequence)
+constexpr int kWideMinRows = 256;   // below this the few-row kernel's passes are as fast
+
+struct WideWs {
+    RowInfo ri;
+    int32_t *n_rows_tmp;
+    float *x, *qkv, *qrot, *t_in;
+    Operand xn1, xn2, ao, act;
+    int rows_pad;
+    size_t bytes;
+};
+
+WideWs carve_wide(const ssd_model *m, int B, int C, uint8_t *base) {
+    const ssd_arch &a = m->a;
+    const size_t R = (size_t)B * C, Rp = align_up(R, kPfTileM), d = a.d_model, F = a.d_ff;
+    size_t off = 0;
+    auto take = [&](size_t bytes) -> uint8_t * {
+        uint8_t *p = base ? base + off : nullptr;
+        off += align_up(bytes, 1024);
+        return p;
+    };
+    WideWs w;
+    memset(&w, 0, sizeof(w));
+    const size_t half = a.pos == 1 ? a.rotary_dim / 2 : 0;
+    w.ri.seq = (int32_t *)take(sizeof(int32_t) * R);
+    w.ri.pos = (int32_t *)take(sizeof(int32_t) * R);
+    w.ri.valid = (int32_t *)take(sizeof(int32_t) * R);
+    w.ri.n_eff = (int32_t *)take(sizeof(int32_t) * B);
+    w.ri.rope_cos = (float *)take(sizeof(float) * R * (half ? half : 1));
+    w.ri.rope_sin = (float *)take(sizeof(float) * R * (half ? half : 1));
+    w.n_rows_tmp = (int32_t *)take(sizeof(int32_t) * B);
+    w.x = (float *)take(sizeof(float) * R * d);
+    w.qkv = (float *)take(sizeof(float) * R * 3 * d);
+    w.qrot = (float *)take(sizeof(float) * R * d);
+    w.t_in = (float *)take(sizeof(float) * R * m->d_in);
+    auto operand = [&](size_t ld, bool needed) {  // rows padded to whole 128-row tiles; hi and lo apart
+        Operand o;
+        o.f32 = nullptr; o.hi = nullptr; o.lo = nullptr; o.ld = (int)ld;
+        if (!needed) return o;
+        o.hi = (__nv_bfloat16 *)take(2 * Rp * ld);
+        o.lo = (__nv_bfloat16 *)take(2 * Rp * ld);
+        return o;
+    };
+    w.xn1 = operand(d, true);
+    w.xn2 = operand(d, a.parallel_residual != 0);
+    w.ao = operand(d, true);
+    w.act = operand(F, true);
+    w.rows_pad = (int)Rp;
+    w.bytes = off;
+    return w;
+}
+
+bool wide_path_ok(const ssd_model *m) {
+    const ssd_arch &a = m->a;
+    return a.dtype == 1 && g_prefill_mode != 1 && a.head_dim % 16 == 0 && a.d_model % 8 == 0 && a.d_ff % 8 == 0 &&
+           !m->tm256.empty();
+}
+
+// out[R, ldo] += X[R, Kd] W[N, Kd]^T over 128 x 256 output tiles
+int gemm_wide(cudaStream_t st, const CUtensorMap *tw, const Operand &X, int rows_pad, int R, int Kd, int N, float *out,
+              int ldo, int32_t *status) {
+    CUtensorMap th, tl;
+    if (make_map(&th, X.hi, rows_pad, Kd, kPfTileM) || make_map(&tl, X.lo, rows_pad, Kd, kPfTileM)) return SSD_E_CUDA;
+    PfGemmArgs g;
+    g.out = out; g.ldo = ldo; g.N = N; g.Kd = Kd; g.R = R; g.status = status;
+    g.wait_cycles = g_wait_cycles > 0 ? g_wait_cycles : kWaitCycles;
+    LAUNCH(prefill_gemm_kernel, dim3(ceil_div(N, kPfTileN), rows_pad / kPfTileM), kPfThreads, kPfSmem, st, *tw, th, tl, g);
+    return SSD_OK;
+}
+
+// One decoder forward over B x C prompt rows: fills the cache (no logits).  The structure of the stepwise
+// forward with the two many-row kernels in place of the few-row GEMM and attention.
+int forward_wide(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int C, const int32_t *n_rows,
+                 const WideWs &w, cudaStream_t st) {
+    const ssd_arch &a = m->a;
+    const int B = kv->B, R = B * C, d = a.d_model, F = a.d_ff, Rp = w.rows_pad;
+    SetupArgs s;
+    s.B = B; s.M = C; s.n_rows = n_rows; s.len = kv->len; s.s_max = kv->S;
+    s.pos_limit = a.pos == 0 ? a.max_pos : 0;
+    s.rotary_dim = a.pos == 1 ? a.rotary_dim : 0;
+    s.rotary_base = a.rotary_base;
+    s.ri = w.ri;
+    s.status = kv->status;
+    LAUNCH(setup_rows_kernel, R, 64, 0, st, s);
+    LAUNCH(embed_kernel<__nv_bfloat16>, R, 256, 0, st, (const __nv_bfloat16 *)m->w[T_TOK],
+           (const __nv_bfloat16 *)m->w[T_POS], tokens, tok_stride, C, a.vocab, d, w.ri, w.x);
+    auto norm_args = [&](const float *g1, const float *b1, Operand o1) {
+        NormArgs n;
+        memset(&n, 0, sizeof(n));
+        n.x = w.x; n.d = d; n.kind = a.norm; n.eps = a.norm_eps;
+        n.n_norms = 1; n.g[0] = g1; n.b[0] = b1; n.out[0] = o1;
+        return n;
+    };
+    int rc;
+    for (int l = 0; l < a.n_layers; ++l) {
+        const CUtensorMap *tm = &m->tm256[4 * l];
+        const float *b_qkv = (const float *)lw(m, l, L_BQKV), *b_o = (const float *)lw(m, l, L_BO);
+        const float *b_in = (const float *)lw(m, l, L_BIN), *b_out = (const float *)lw(m, l, L_BOUT);
+        NormArgs n1 = norm_args((const float *)lw(m, l, L_LN1G), (const float *)lw(m, l, L_LN1B), w.xn1);
+        n1.init[n1.n_init++] = InitJob{w.qkv, b_qkv, 3 * d, 3 * d};
+        if (a.parallel_residual) {
+            n1.n_norms = 2;
+            n1.g[1] = (const float *)lw(m, l, L_LN2G);
+            n1.b[1] = (const float *)lw(m, l, L_LN2B);
+            n1.out[1] = w.xn2;
+            n1.init[n1.n_init++] = InitJob{w.t_in, b_in, m->d_in, m->d_in};
+        }
+        LAUNCH(norm_kernel, R, 256, 0, st, n1);
+        if ((rc = gemm_wide(st, tm + 0, w.xn1, Rp, R, d, 3 * d, w.qkv, 3 * d, kv->status))) return rc;
+        if (a.parallel_residual)
+            if ((rc = gemm_wide(st, tm + 2, w.xn2, Rp, R, d, m->d_in, w.t_in, m->d_in, kv->status))) return rc;
+        RopeArgs ra;
+        ra.qkv = w.qkv; ra.q_out = w.qrot;
+        ra.cache = kv->cache + (size_t)l * kv->layer_bytes;
+        ra.d = d; ra.H = a.n_heads; ra.Dh = a.head_dim; ra.S = kv->S;
+        ra.rotary_dim = a.pos == 1 ? a.rotary_dim : 0;
+        ra.ri = w.ri;
+        LAUNCH(rope_append_kernel<__nv_bfloat16>, R, 256, 0, st, ra);
+        PfAttnArgs at;
+        at.q = w.qrot;
+        at.cache = (const __nv_bfloat16 *)(kv->cache + (size_t)l * kv->layer_bytes);
+        at.len = kv->len; at.n_eff = w.ri.n_eff;
+        at.out_hi = w.ao.hi; at.out_lo = w.ao.lo;
+        at.M = C; at.H = a.n_heads; at.Dh = a.head_dim; at.S = kv->S; at.d = d;
+        at.scale = 1.0f / sqrtf((float)a.head_dim);
+        LAUNCH(prefill_attn_kernel, dim3(ceil_div(C, kPaRows), a.n_heads, B), kPaThreads, prefill_attn_smem(a.head_dim), st,
+               at);
+        // the residual-stream biases of the projections that accumulate into x
+        if (a.parallel_residual) {
+            BiasJob bj{b_o, b_out};
+            LAUNCH(act_kernel, dim3(ceil_div(F, 256), R), 256, 0, st, w.t_in, m->d_in, F, a.act == 1, w.act, w.x, d, bj);
+            if ((rc = gemm_wide(st, tm + 1, w.ao, Rp, R, d, d, w.x, d, kv->status))) return rc;
+            if ((rc = gemm_wide(st, tm + 3, w.act, Rp, R, F, d, w.x, d, kv->status))) return rc;
+        } else {
+            LAUNCH(add_bias_kernel, R, 256, 0, st, w.x, b_o, d);
+            if ((rc = gemm_wide(st, tm + 1, w.ao, Rp, R, d, d, w.x, d, kv->status))) return rc;
+            NormArgs n2 = norm_args((const float *)lw(m, l, L_LN2G), (const float *)lw(m, l, L_LN2B), w.xn1);
+            n2.init[n2.n_init++] = InitJob{w.t_in, b_in, m->d_in, m->d_in};
+            LAUNCH(norm_kernel, R, 256, 0, st, n2);
+            if ((rc = gemm_wide(st, tm + 2, w.xn1, Rp, R, d, m->d_in, w.t_in, m->d_in, kv->status))) return rc;
+            BiasJob bj{b_out, nullptr};
+            LAUNCH(act_kernel, dim3(ceil_div(F, 256), R), 256, 0, st, w.t_in, m->d_in, F, a.act == 1, w.act, w.x, d, bj);
+            if ((rc = gemm_wide(st, tm + 3, w.act, Rp, R, F, d, w.x, d, kv->status))) return rc;
+        }
+    }
+    kv->last_rows = C;
+    return SSD_OK;
+}
+
 int check_ws(const ssd_model *m, int B, int M, void *ws, size_t ws_bytes, Workspace *out) {
     if (!ws) return SSD_E_ARG;
     if (B * M > kMaxRows || M > kMaxRowsPerSeq || M < 1) return SSD_E_CAPACITY;
@@ -822,6 +983,19 @@ int ssd_set_attention_mode(int mode) {
     if (mode < 0 || mode > 2) return SSD_E_ARG;
     g_attn_mode = mode;
     return SSD_OK;
+}
+
+int ssd_set_prefill_mode(int mode) {
+    if (mode < 0 || mode > 2) return SSD_E_ARG;
+    g_prefill_mode = mode;
+    return SSD_OK;
+}
+
+size_t ssd_prefill_workspace_bytes(const ssd_model *m, int batch, int rows_per_seq) {
+    if (!m || batch < 1 || rows_per_seq < 1 || !wide_path_ok(m)) return 0;
+    if ((long long)batch * rows_per_seq > kWideMaxRows) rows_per_seq = kWideMaxRows / batch;
+    if (rows_per_seq < 1) return 0;
+    return carve_wide(m, batch, rows_per_seq, nullptr).bytes;
 }
 
 int ssd_set_persistent(int enable) {
@@ -938,6 +1112,30 @@ int kv_prefill(ssd_model *m, ssd_kv *kv, const int32_t *dev_tokens, const int32_
     if (!same_cache_shape(m, kv)) return SSD_E_ARG;
     if (kv_bound(kv) + max_tokens > kv->S) return SSD_E_CAPACITY;
     cudaStream_t st = (cudaStream_t)stream;
+    if (max_tokens == 0) return SSD_OK;
+    if (wide_path_ok(m) && dev_ws && ((uintptr_t)dev_ws & 255) == 0) {
+        // many rows per pass: the largest share of the prompt (in equal passes) whose buffers fit the workspace
+        int cap = kWideMaxRows / kv->B;
+        while (cap >= 1 && carve_wide(m, kv->B, cap < max_tokens ? cap : max_tokens, nullptr).bytes > ws_bytes) cap /= 2;
+        if (cap >= 1) {
+            const int passes = ceil_div(max_tokens, cap);
+            int Cw = ceil_div(ceil_div(max_tokens, passes), 16) * 16;
+            if (Cw > max_tokens) Cw = max_tokens;
+            if (Cw > cap) Cw = cap;
+            if (g_prefill_mode == 2 || kv->B * Cw >= kWideMinRows) {
+                const WideWs ww = carve_wide(m, kv->B, Cw, (uint8_t *)dev_ws);
+                const int chunks = ceil_div(max_tokens, Cw);
+                for (int c = 0; c < chunks; ++c) {
+                    LAUNCH(prefill_rows_kernel, ceil_div(kv->B, 64), 64, 0, st, dev_n_tokens, c, Cw, ww.n_rows_tmp, kv->B);
+                    int rcw = forward_wide(m, kv, dev_tokens + (size_t)c * Cw, max_tokens, Cw, ww.n_rows_tmp, ww, st);
+                    if (rcw) return rcw;
+                    const unsigned seq = kv_note_op(kv, Cw);
+                    LAUNCH(kv_commit_rows_kernel, 1, 64, 0, st, kv->len, ww.ri.n_eff, kv->B, kv->mailbox_dev, seq);
+                }
+                return SSD_OK;
+            }
+        }
+    }
     // rows per sequence and pass: as many as the row limits and the caller's workspace allow (every pass streams
     // all weights once, whatever its rows)
     int C = kMaxRows / kv->B;

@@ -63,6 +63,7 @@ class Engine:
         # in-kernel tail costs grid barriers where the other path costs two small launches); the per-token form
         # is the default because it is the faster one at batch 1.
         self.fused_draft = False
+        self.prompt_ws_cap = 4 << 30      # bytes of temporary workspace the prompt pass may take
         V = target.arch.vocab
         dev = "cuda"
         self.tkv = B.KV(target, batch, max_len)
@@ -118,14 +119,27 @@ class Engine:
         if P > 1:
             body = prompts[:, :P - 1].contiguous()
             n = torch.full((self.batch,), P - 1, dtype=torch.int32, device=prompts.device)
-            B.kv_prefill(self.target, self.tkv, body, n, self.ws_pre_t)
+            B.kv_prefill(self.target, self.tkv, body, n, self._prompt_workspace(self.target, P - 1, self.ws_pre_t))
             if self.dkv is not None:
-                B.kv_prefill(self.draft, self.dkv, body, n, self.ws_pre_d)
+                B.kv_prefill(self.draft, self.dkv, body, n, self._prompt_workspace(self.draft, P - 1, self.ws_pre_d))
         self.rows[:, 0] = prompts[:, P - 1]
         if self.dkv is not None:
             self.draft_in[:, 0] = prompts[:, P - 1]
             self.draft_n_in.fill_(1)
         self.out_count.zero_()
+
+    def _prompt_workspace(self, model: "B.Model", n_tokens: int, small: torch.Tensor) -> torch.Tensor:
+        """Workspace for the prompt pass: from 256 rows per pass a temporary block for the many-row form (up to
+        `prompt_ws_cap` bytes, released after the pass), else the few-row workspace."""
+        rows = min(n_tokens, 8192 // self.batch)
+        while rows * self.batch >= 256:
+            nbytes = model.prefill_workspace_bytes(self.batch, rows)
+            if nbytes == 0:
+                break
+            if nbytes <= self.prompt_ws_cap:
+                return B.device_buffer(nbytes)
+            rows //= 2
+        return small
 
     def set_k(self, k: int) -> None:
         """Draft k <= K tokens in the following iterations: the row block and the q block become [batch, k + 1]
