@@ -13,8 +13,8 @@
 //   * per stage eight tcgen05.mma (M = 128, N = 256, K = 16): four k-steps with the hi tile, four with the lo
 //     tile, into ONE fp32 accumulator in tensor memory: W hi + W lo is the fp32-activation product to ~2^-17,
 //     the same arithmetic as the few-row path (the price is half the tensor throughput);
-//   * the tile is owned by this CTA alone (no split over k), so the epilogue adds the accumulator to the
-//     output with plain loads and stores.
+//   * the tile is owned by this CTA alone (no split over k), so the epilogue writes accumulator + bias over the
+//     output, or adds them to it (the residual stream), with plain loads and stores.
 // Every wait is bounded; on time-out the kernel records SSD_E_TIMEOUT, drains its copies and returns.
 #pragma once
 #include <cuda.h>
@@ -22,6 +22,7 @@
 #include "common.cuh"
 #include "gemm.cuh"
 #include "persistent.cuh"
+#include "rowops.cuh"
 
 namespace ssd {
 
@@ -33,7 +34,9 @@ constexpr int kPfThreads = 192;
 constexpr size_t kPfSmem = 1024 + (size_t)kPfStages * kPfStageBytes + 256;
 
 struct PfGemmArgs {
-    float *out;  // [R, ldo] fp32, accumulated into
+    float *out;         // [R, ldo] fp32
+    const float *bias;  // [N] or null
+    int accumulate;     // 1: out += X W^T + bias (the residual stream); 0: out = X W^T + bias
     int ldo, N, Kd, R;
     long long wait_cycles;  // bound of every wait that takes work
     int32_t *status;
@@ -125,7 +128,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
         tc_fence_after();
         if (__all_sync(0xffffffffu, landed && !*abort_flag)) {  // (the tensor-memory loads are warp-wide)
             float *orow = a.out + (size_t)row * a.ldo + n0;
-            const bool vec = ((uintptr_t)a.out & 15) == 0 && (a.ldo & 3) == 0;
+            const bool vec = ((uintptr_t)a.out & 15) == 0 && (a.ldo & 3) == 0 && (!a.bias || ((uintptr_t)a.bias & 15) == 0);
 #pragma unroll 1
             for (int cb = 0; cb < kPfTileN / 32; ++cb) {
                 if (n0 + cb * 32 >= a.N) break;
@@ -133,15 +136,34 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                 tc_ld_32(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cb * 32), v);
                 if (row < a.R) {
                     if (vec && n0 + cb * 32 + 31 < a.N) {
+                        if (a.bias) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            float4 o = *reinterpret_cast<float4 *>(orow + cb * 32 + 4 * i);
-                            o.x += v[4 * i]; o.y += v[4 * i + 1]; o.z += v[4 * i + 2]; o.w += v[4 * i + 3];
-                            *reinterpret_cast<float4 *>(orow + cb * 32 + 4 * i) = o;
+                            for (int i = 0; i < 8; ++i) {
+                                const float4 bv = __ldg(reinterpret_cast<const float4 *>(a.bias + n0 + cb * 32 + 4 * i));
+                                v[4 * i] += bv.x; v[4 * i + 1] += bv.y; v[4 * i + 2] += bv.z; v[4 * i + 3] += bv.w;
+                            }
                         }
+                        if (a.accumulate) {
+                            float4 o[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) o[i] = *reinterpret_cast<const float4 *>(orow + cb * 32 + 4 * i);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                v[4 * i] += o[i].x; v[4 * i + 1] += o[i].y; v[4 * i + 2] += o[i].z; v[4 * i + 3] += o[i].w;
+                            }
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            *reinterpret_cast<float4 *>(orow + cb * 32 + 4 * i) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
                     } else {
-                        for (int i = 0; i < 32; ++i)
-                            if (n0 + cb * 32 + i < a.N) orow[cb * 32 + i] += v[i];
+                        for (int i = 0; i < 32; ++i) {
+                            const int col = n0 + cb * 32 + i;
+                            if (col < a.N) {
+                                float y = v[i] + (a.bias ? a.bias[col] : 0.f);
+                                if (a.accumulate) y += orow[cb * 32 + i];
+                                orow[cb * 32 + i] = y;
+                            }
+                        }
                     }
                 }
             }
@@ -158,11 +180,91 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     }
 }
 
-// x[r, :] += bias  (the out-projection's bias, before that projection accumulates into the residual stream)
-__global__ void add_bias_kernel(float *x, const float *bias, int d) {
-    if (!bias) return;
-    float *row = x + (size_t)blockIdx.x * d;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) row[i] += bias[i];
+// Row norm for the many-row pass: one CTA of 256 threads per row, the row held in registers (float4 per thread,
+// up to 8192 columns; wider rows are re-read), statistics in fp64, one or two outputs (bf16 hi + lo, row-major)
+// from the same statistics.
+struct PfNormArgs {
+    const float *x;
+    int d, kind;  // 0 LayerNorm, 1 RMSNorm
+    float eps;
+    int n_norms;
+    const float *g[2], *b[2];
+    __nv_bfloat16 *hi[2], *lo[2];
+};
+__device__ __forceinline__ void store_hilo4(__nv_bfloat16 *hi, __nv_bfloat16 *lo, size_t idx, float4 y) {
+    const __nv_bfloat162 h01 = __floats2bfloat162_rn(y.x, y.y), h23 = __floats2bfloat162_rn(y.z, y.w);
+    const __nv_bfloat162 l01 = __floats2bfloat162_rn(y.x - __low2float(h01), y.y - __high2float(h01));
+    const __nv_bfloat162 l23 = __floats2bfloat162_rn(y.z - __low2float(h23), y.w - __high2float(h23));
+    uint2 hv, lv;
+    hv.x = *reinterpret_cast<const uint32_t *>(&h01); hv.y = *reinterpret_cast<const uint32_t *>(&h23);
+    lv.x = *reinterpret_cast<const uint32_t *>(&l01); lv.y = *reinterpret_cast<const uint32_t *>(&l23);
+    *reinterpret_cast<uint2 *>(hi + idx) = hv;
+    *reinterpret_cast<uint2 *>(lo + idx) = lv;
+}
+__global__ void __launch_bounds__(256) prefill_norm_kernel(const PfNormArgs a) {  // d % 4 == 0
+    __shared__ double red[32];
+    const int r = blockIdx.x, q4 = a.d >> 2;
+    const float4 *x4 = reinterpret_cast<const float4 *>(a.x + (size_t)r * a.d);
+    float4 v[8];
+    double s = 0.0, ss = 0.0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int i = threadIdx.x + 256 * k;
+        v[k] = i < q4 ? x4[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        s += ((double)v[k].x + (double)v[k].y) + ((double)v[k].z + (double)v[k].w);
+    }
+    for (int i = threadIdx.x + 2048; i < q4; i += 256) {
+        const float4 w = x4[i];
+        s += ((double)w.x + (double)w.y) + ((double)w.z + (double)w.w);
+    }
+    double mean = 0.0;
+    if (a.kind == 0) mean = block_sum(s, red) / a.d;
+    auto sq = [&](const float4 &w) {
+        const double c0 = w.x - mean, c1 = w.y - mean, c2 = w.z - mean, c3 = w.w - mean;
+        return (c0 * c0 + c1 * c1) + (c2 * c2 + c3 * c3);
+    };
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+        if (threadIdx.x + 256 * k < q4) ss += sq(v[k]);
+    for (int i = threadIdx.x + 2048; i < q4; i += 256) ss += sq(x4[i]);
+    const double rstd = rsqrt(block_sum(ss, red) / a.d + (double)a.eps);
+#pragma unroll
+    for (int n = 0; n < 2; ++n) {
+        if (n >= a.n_norms) break;
+        const float4 *g4 = reinterpret_cast<const float4 *>(a.g[n]);
+        const float4 *b4 = reinterpret_cast<const float4 *>(a.b[n]);
+        auto emit = [&](int i, const float4 &w) {
+            const float4 g = __ldg(g4 + i);
+            const float4 bb = b4 ? __ldg(b4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float4 y;
+            y.x = (float)(((double)w.x - mean) * rstd * (double)g.x + (double)bb.x);
+            y.y = (float)(((double)w.y - mean) * rstd * (double)g.y + (double)bb.y);
+            y.z = (float)(((double)w.z - mean) * rstd * (double)g.z + (double)bb.z);
+            y.w = (float)(((double)w.w - mean) * rstd * (double)g.w + (double)bb.w);
+            store_hilo4(a.hi[n], a.lo[n], (size_t)r * a.d + 4 * (size_t)i, y);
+        };
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+            if (threadIdx.x + 256 * k < q4) emit(threadIdx.x + 256 * k, v[k]);
+        for (int i = threadIdx.x + 2048; i < q4; i += 256) emit(i, x4[i]);
+    }
+}
+
+// act[r, i] = GELU(t[r, i])  or  SiLU(t[r, i]) * t[r, F + i], four columns per thread; grid (ceil(F / 1024), R); F % 4 == 0
+__global__ void __launch_bounds__(256) prefill_act_kernel(const float *__restrict__ t, int ld_t, int F, int swiglu,
+                                                          __nv_bfloat16 *hi, __nv_bfloat16 *lo) {
+    const int r = blockIdx.y, i = 4 * (blockIdx.x * 256 + threadIdx.x);
+    if (i >= F) return;
+    const float *tr = t + (size_t)r * ld_t;
+    const float4 u = *reinterpret_cast<const float4 *>(tr + i);
+    float4 y;
+    if (swiglu) {
+        const float4 w = *reinterpret_cast<const float4 *>(tr + F + i);
+        y = make_float4(silu(u.x) * w.x, silu(u.y) * w.y, silu(u.z) * w.z, silu(u.w) * w.w);
+    } else {
+        y = make_float4(gelu_erf(u.x), gelu_erf(u.y), gelu_erf(u.z), gelu_erf(u.w));
+    }
+    store_hilo4(hi, lo, (size_t)r * F + i, y);
 }
 
 // prefill_attn_kernel: causal attention of 64 query rows of one (sequence, head) over the cache, which already

@@ -806,24 +806,26 @@ WideWs carve_wide(const ssd_model *m, int B, int C, uint8_t *base) {
 
 bool wide_path_ok(const ssd_model *m) {
     const ssd_arch &a = m->a;
-    return a.dtype == 1 && g_prefill_mode != 1 && a.head_dim % 16 == 0 && a.d_model % 8 == 0 && a.d_ff % 8 == 0 &&
+    return a.dtype == 1 && g_prefill_mode != 1 && a.head_dim % 16 == 0 && a.d_model % 8 == 0 && a.d_ff % 8 == 0 && m->d_in % 4 == 0 &&
            !m->tm256.empty();
 }
 
-// out[R, ldo] += X[R, Kd] W[N, Kd]^T over 128 x 256 output tiles
+// out[R, ldo] (+)= X[R, Kd] W[N, Kd]^T + bias over 128 x 256 output tiles
 int gemm_wide(cudaStream_t st, const CUtensorMap *tw, const Operand &X, int rows_pad, int R, int Kd, int N, float *out,
-              int ldo, int32_t *status) {
+              int ldo, const float *bias, bool accumulate, int32_t *status) {
     CUtensorMap th, tl;
     if (make_map(&th, X.hi, rows_pad, Kd, kPfTileM) || make_map(&tl, X.lo, rows_pad, Kd, kPfTileM)) return SSD_E_CUDA;
     PfGemmArgs g;
-    g.out = out; g.ldo = ldo; g.N = N; g.Kd = Kd; g.R = R; g.status = status;
+    g.out = out; g.bias = bias; g.accumulate = accumulate ? 1 : 0;
+    g.ldo = ldo; g.N = N; g.Kd = Kd; g.R = R; g.status = status;
     g.wait_cycles = g_wait_cycles > 0 ? g_wait_cycles : kWaitCycles;
     LAUNCH(prefill_gemm_kernel, dim3(ceil_div(N, kPfTileN), rows_pad / kPfTileM), kPfThreads, kPfSmem, st, *tw, th, tl, g);
     return SSD_OK;
 }
 
-// One decoder forward over B x C prompt rows: fills the cache (no logits).  The structure of the stepwise
-// forward with the two many-row kernels in place of the few-row GEMM and attention.
+// One decoder forward over B x C prompt rows: fills the cache (no logits).  The steps of the stepwise forward with
+// many-row kernels: the projections write (q, k, v and the MLP input) or add to (the residual stream) their output
+// together with the bias, so nothing is pre-loaded.
 int forward_wide(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride, int C, const int32_t *n_rows,
                  const WideWs &w, cudaStream_t st) {
     const ssd_arch &a = m->a;
@@ -838,11 +840,11 @@ int forward_wide(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride
     LAUNCH(setup_rows_kernel, R, 64, 0, st, s);
     LAUNCH(embed_kernel<__nv_bfloat16>, R, 256, 0, st, (const __nv_bfloat16 *)m->w[T_TOK],
            (const __nv_bfloat16 *)m->w[T_POS], tokens, tok_stride, C, a.vocab, d, w.ri, w.x);
-    auto norm_args = [&](const float *g1, const float *b1, Operand o1) {
-        NormArgs n;
+    auto norm_args = [&](const float *g1, const float *b1, const Operand &o1) {
+        PfNormArgs n;
         memset(&n, 0, sizeof(n));
         n.x = w.x; n.d = d; n.kind = a.norm; n.eps = a.norm_eps;
-        n.n_norms = 1; n.g[0] = g1; n.b[0] = b1; n.out[0] = o1;
+        n.n_norms = 1; n.g[0] = g1; n.b[0] = b1; n.hi[0] = o1.hi; n.lo[0] = o1.lo;
         return n;
     };
     int rc;
@@ -850,19 +852,17 @@ int forward_wide(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride
         const CUtensorMap *tm = &m->tm256[4 * l];
         const float *b_qkv = (const float *)lw(m, l, L_BQKV), *b_o = (const float *)lw(m, l, L_BO);
         const float *b_in = (const float *)lw(m, l, L_BIN), *b_out = (const float *)lw(m, l, L_BOUT);
-        NormArgs n1 = norm_args((const float *)lw(m, l, L_LN1G), (const float *)lw(m, l, L_LN1B), w.xn1);
-        n1.init[n1.n_init++] = InitJob{w.qkv, b_qkv, 3 * d, 3 * d};
+        PfNormArgs n1 = norm_args((const float *)lw(m, l, L_LN1G), (const float *)lw(m, l, L_LN1B), w.xn1);
         if (a.parallel_residual) {
             n1.n_norms = 2;
             n1.g[1] = (const float *)lw(m, l, L_LN2G);
             n1.b[1] = (const float *)lw(m, l, L_LN2B);
-            n1.out[1] = w.xn2;
-            n1.init[n1.n_init++] = InitJob{w.t_in, b_in, m->d_in, m->d_in};
+            n1.hi[1] = w.xn2.hi; n1.lo[1] = w.xn2.lo;
         }
-        LAUNCH(norm_kernel, R, 256, 0, st, n1);
-        if ((rc = gemm_wide(st, tm + 0, w.xn1, Rp, R, d, 3 * d, w.qkv, 3 * d, kv->status))) return rc;
+        LAUNCH(prefill_norm_kernel, R, 256, 0, st, n1);
+        if ((rc = gemm_wide(st, tm + 0, w.xn1, Rp, R, d, 3 * d, w.qkv, 3 * d, b_qkv, false, kv->status))) return rc;
         if (a.parallel_residual)
-            if ((rc = gemm_wide(st, tm + 2, w.xn2, Rp, R, d, m->d_in, w.t_in, m->d_in, kv->status))) return rc;
+            if ((rc = gemm_wide(st, tm + 2, w.xn2, Rp, R, d, m->d_in, w.t_in, m->d_in, b_in, false, kv->status))) return rc;
         RopeArgs ra;
         ra.qkv = w.qkv; ra.q_out = w.qrot;
         ra.cache = kv->cache + (size_t)l * kv->layer_bytes;
@@ -879,23 +879,14 @@ int forward_wide(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride
         at.scale = 1.0f / sqrtf((float)a.head_dim);
         LAUNCH(prefill_attn_kernel, dim3(ceil_div(C, kPaRows), a.n_heads, B), kPaThreads, prefill_attn_smem(a.head_dim), st,
                at);
-        // the residual-stream biases of the projections that accumulate into x
-        if (a.parallel_residual) {
-            BiasJob bj{b_o, b_out};
-            LAUNCH(act_kernel, dim3(ceil_div(F, 256), R), 256, 0, st, w.t_in, m->d_in, F, a.act == 1, w.act, w.x, d, bj);
-            if ((rc = gemm_wide(st, tm + 1, w.ao, Rp, R, d, d, w.x, d, kv->status))) return rc;
-            if ((rc = gemm_wide(st, tm + 3, w.act, Rp, R, F, d, w.x, d, kv->status))) return rc;
-        } else {
-            LAUNCH(add_bias_kernel, R, 256, 0, st, w.x, b_o, d);
-            if ((rc = gemm_wide(st, tm + 1, w.ao, Rp, R, d, d, w.x, d, kv->status))) return rc;
-            NormArgs n2 = norm_args((const float *)lw(m, l, L_LN2G), (const float *)lw(m, l, L_LN2B), w.xn1);
-            n2.init[n2.n_init++] = InitJob{w.t_in, b_in, m->d_in, m->d_in};
-            LAUNCH(norm_kernel, R, 256, 0, st, n2);
-            if ((rc = gemm_wide(st, tm + 2, w.xn1, Rp, R, d, m->d_in, w.t_in, m->d_in, kv->status))) return rc;
-            BiasJob bj{b_out, nullptr};
-            LAUNCH(act_kernel, dim3(ceil_div(F, 256), R), 256, 0, st, w.t_in, m->d_in, F, a.act == 1, w.act, w.x, d, bj);
-            if ((rc = gemm_wide(st, tm + 3, w.act, Rp, R, F, d, w.x, d, kv->status))) return rc;
+        if ((rc = gemm_wide(st, tm + 1, w.ao, Rp, R, d, d, w.x, d, b_o, true, kv->status))) return rc;
+        if (!a.parallel_residual) {
+            PfNormArgs n2 = norm_args((const float *)lw(m, l, L_LN2G), (const float *)lw(m, l, L_LN2B), w.xn1);
+            LAUNCH(prefill_norm_kernel, R, 256, 0, st, n2);
+            if ((rc = gemm_wide(st, tm + 2, w.xn1, Rp, R, d, m->d_in, w.t_in, m->d_in, b_in, false, kv->status))) return rc;
         }
+        LAUNCH(prefill_act_kernel, dim3(ceil_div(F, 1024), R), 256, 0, st, w.t_in, m->d_in, F, a.act == 1, w.act.hi, w.act.lo);
+        if ((rc = gemm_wide(st, tm + 3, w.act, Rp, R, F, d, w.x, d, b_out, true, kv->status))) return rc;
     }
     kv->last_rows = C;
     return SSD_OK;

@@ -60,8 +60,8 @@ def test_many_row_prompt_pass_matches_oracle(name, many_row_mode):
     kv = B.KV(model, Bn, S)
     n0 = B.launch_count()
     B.kv_prefill(model, kv, torch.from_numpy(prompts).cuda(), torch.from_numpy(lens).cuda(), B.device_buffer(nbytes))
-    # one pass: set-up, embedding, and per layer 4 GEMMs + norm(s) + append + attention + activation (+ bias)
-    per_layer = 8 if arch.parallel_residual else 10
+    # one pass: set-up, embedding, and per layer 4 GEMMs + norm(s) + append + attention + activation
+    per_layer = 8 if arch.parallel_residual else 9
     assert B.launch_count() - n0 == 1 + 2 + per_layer * arch.n_layers + 1
     _check_against_oracle(arch, omodel, model, kv, prompts, lens, S)
 
@@ -115,7 +115,7 @@ def test_many_row_form_is_taken_from_256_rows_and_equals_the_chunked_form():
                 B.set_prefill_mode(0)
     chunks = lambda P: -(-P // C)
     assert caches[(130, 1)][1] == 3 * chunks(130) and caches[(100, 0)][1] == 3 * chunks(100)
-    assert caches[(130, 0)][1] == 1 + 2 + 10 * arch.n_layers + 1
+    assert caches[(130, 0)][1] == 1 + 2 + 9 * arch.n_layers + 1
     _cache_close(arch, caches[(130, 0)][0], caches[(130, 1)][0])
 
 
