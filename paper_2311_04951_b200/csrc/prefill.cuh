@@ -6,8 +6,9 @@
 // which take any number of rows.
 //
 // prefill_gemm_kernel:  out[r, n] += sum_k (Xhi[r, k] + Xlo[r, k]) * W[n, k]
-//   * one CTA per (128-row, 256-column) output tile, 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer,
-//     warps 2-5 = epilogue (one tensor-memory lane quadrant each);
+//   * output tiles of 128 rows x 256 columns, dealt round-robin to one CTA per SM; 192 threads: warp 0 = TMA
+//     producer, warp 1 = MMA issuer, warps 2-5 = epilogue (one tensor-memory lane quadrant each); two accumulators
+//     in tensor memory (2 x 256 columns), so a tile's epilogue runs under the next tile's products;
 //   * a stage of the shared-memory ring = the activation rows' hi tile and lo tile (128 rows x 64 k, bf16) and
 //     the weight tile (256 rows x 64 k), all by 2-D tensor-map copies with the 128-byte swizzle, 64 KB;
 //   * per stage eight tcgen05.mma (M = 128, N = 256, K = 16): four k-steps with the hi tile, four with the lo
@@ -31,7 +32,7 @@ constexpr int kPfABytes = kPfTileM * kTileK * 2;            // 16 KB: one of hi 
 constexpr int kPfWBytes = kPfTileN * kTileK * 2;            // 32 KB
 constexpr int kPfStageBytes = 2 * kPfABytes + kPfWBytes;    // 64 KB
 constexpr int kPfThreads = 192;
-constexpr size_t kPfSmem = 1024 + (size_t)kPfStages * kPfStageBytes + 256;
+constexpr size_t kPfSmem = 1024 + (size_t)kPfStages * kPfStageBytes + 256;  // + barriers, TMEM slot, abort flag
 
 struct PfGemmArgs {
     float *out;         // [R, ldo] fp32
@@ -49,16 +50,20 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t *full = (uint64_t *)(smem + (size_t)kPfStages * kPfStageBytes);
     uint64_t *empty = full + kPfStages;
-    uint64_t *acc_full = empty + kPfStages;
-    uint32_t *tmem_slot = (uint32_t *)(acc_full + 1);
+    uint64_t *acc_full = empty + kPfStages;  // [2]
+    uint64_t *acc_empty = acc_full + 2;      // [2]
+    uint32_t *tmem_slot = (uint32_t *)(acc_empty + 2);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.y * kPfTileM, n0 = blockIdx.x * kPfTileN;
     const int kchunks = (a.Kd + kTileK - 1) / kTileK;
+    const int tiles_m = (a.R + kPfTileM - 1) / kPfTileM, tiles_n = (a.N + kPfTileN - 1) / kPfTileN;
+    const int n_tiles = tiles_m * tiles_n;
+    // this CTA's tiles: blockIdx.x, + gridDim.x, ...; row tiles vary fastest, so the CTAs that run together share
+    // weight tiles in L2 (the activations of all rows stay there anyway)
 
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(256)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(512)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -67,7 +72,10 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             mbar_init(&full[s], 1);
             mbar_init(&empty[s], 1);
         }
-        mbar_init(acc_full, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&acc_full[i], 1);
+            mbar_init(&acc_empty[i], 4);  // one arrival per epilogue warp
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -76,64 +84,96 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    int issued = 0;
+    int issued = 0;  // stage fills issued by the producer thread
     if (warp == 0) {
         if (lane == 0) {
-            for (int kc = 0; kc < kchunks; ++kc, ++issued) {
-                const int s = kc % kPfStages;
-                if (kc >= kPfStages && !mbar_wait_limit(&empty[s], ((kc / kPfStages) - 1) & 1, a.wait_cycles)) {
-                    set_status(a.status, kTimeoutCode);
-                    *abort_flag = 1;
-                    break;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+                const int m0 = (tile % tiles_m) * kPfTileM, n0 = (tile / tiles_m) * kPfTileN;
+                for (int kc = 0; kc < kchunks; ++kc, ++issued) {
+                    const int s = issued % kPfStages;
+                    if (*abort_flag ||
+                        (issued >= kPfStages && !mbar_wait_limit(&empty[s], ((issued / kPfStages) - 1) & 1, a.wait_cycles))) {
+                        ok = false;
+                        break;
+                    }
+                    uint8_t *st = smem + (size_t)s * kPfStageBytes;
+                    mbar_expect_tx(&full[s], kPfStageBytes);
+                    tma_load_2d(st, &tmXhi, kc * kTileK, m0, &full[s]);
+                    tma_load_2d(st + kPfABytes, &tmXlo, kc * kTileK, m0, &full[s]);
+                    tma_load_2d(st + 2 * kPfABytes, &tmW, kc * kTileK, n0, &full[s]);
                 }
-                if (*abort_flag) break;
-                uint8_t *st = smem + (size_t)s * kPfStageBytes;
-                mbar_expect_tx(&full[s], kPfStageBytes);
-                tma_load_2d(st, &tmXhi, kc * kTileK, m0, &full[s]);
-                tma_load_2d(st + kPfABytes, &tmXlo, kc * kTileK, m0, &full[s]);
-                tma_load_2d(st + 2 * kPfABytes, &tmW, kc * kTileK, n0, &full[s]);
+            }
+            if (!ok) {
+                set_status(a.status, kTimeoutCode);
+                *abort_flag = 1;
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_bf16(kPfTileM, kPfTileN);
             bool ok = true;
-            for (int kc = 0; kc < kchunks; ++kc) {
-                const int s = kc % kPfStages;
-                if (*abort_flag || !mbar_wait_limit(&full[s], (kc / kPfStages) & 1, a.wait_cycles)) {
+            int it = 0, j = 0;
+            for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x, ++j) {
+                const int buf = j & 1;
+                if (j >= 2 && !mbar_wait_limit(&acc_empty[buf], ((j >> 1) - 1) & 1, 4 * a.wait_cycles)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t st = smem_u32(smem + (size_t)s * kPfStageBytes);
-                const uint64_t hi = umma_desc_sw128(st), lo = umma_desc_sw128(st + kPfABytes), w = umma_desc_sw128(st + 2 * kPfABytes);
+                const uint32_t d_tmem = tmem + (uint32_t)(buf * kPfTileN);
+                for (int kc = 0; kc < kchunks; ++kc, ++it) {
+                    const int s = it % kPfStages;
+                    if (*abort_flag || !mbar_wait_limit(&full[s], (it / kPfStages) & 1, a.wait_cycles)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t st = smem_u32(smem + (size_t)s * kPfStageBytes);
+                    const uint64_t hi = umma_desc_sw128(st), lo = umma_desc_sw128(st + kPfABytes), w = umma_desc_sw128(st + 2 * kPfABytes);
 #pragma unroll
-                for (int ks = 0; ks < kTileK / 16; ++ks) tc_mma_bf16(tmem, hi + 2 * ks, w + 2 * ks, idesc, (kc | ks) ? 1u : 0u);
+                    for (int ks = 0; ks < kTileK / 16; ++ks) tc_mma_bf16(d_tmem, hi + 2 * ks, w + 2 * ks, idesc, (kc | ks) ? 1u : 0u);
 #pragma unroll
-                for (int ks = 0; ks < kTileK / 16; ++ks) tc_mma_bf16(tmem, lo + 2 * ks, w + 2 * ks, idesc, 1u);
-                tc_commit(&empty[s]);
+                    for (int ks = 0; ks < kTileK / 16; ++ks) tc_mma_bf16(d_tmem, lo + 2 * ks, w + 2 * ks, idesc, 1u);
+                    tc_commit(&empty[s]);
+                }
+                if (ok) tc_commit(&acc_full[buf]);
             }
             if (!ok) {
                 set_status(a.status, kTimeoutCode);
                 *abort_flag = 1;
             }
-            tc_commit(acc_full);  // (arrives once everything issued so far has completed: also on the error path)
         }
         __syncwarp();
     } else {
         // epilogue: accumulator row r sits in tensor-memory lane r; warp w reaches lanes 32 (w % 4) ..
-        const int quad = warp & 3, row = m0 + quad * 32 + lane;
-        const bool landed = mbar_wait_limit(acc_full, 0, 4 * a.wait_cycles);
-        if (!landed) set_status(a.status, kTimeoutCode);
-        tc_fence_after();
-        if (__all_sync(0xffffffffu, landed && !*abort_flag)) {  // (the tensor-memory loads are warp-wide)
+        const int quad = warp & 3;
+        const bool vec = ((uintptr_t)a.out & 15) == 0 && (a.ldo & 3) == 0 && (!a.bias || ((uintptr_t)a.bias & 15) == 0);
+        int j = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++j) {
+            const int buf = j & 1;
+            const int m0 = (tile % tiles_m) * kPfTileM, n0 = (tile / tiles_m) * kPfTileN;
+            const int row = m0 + quad * 32 + lane;
+            // (the wait ends early once another role has given up)
+            bool landed = false;
+            {
+                const long long t0 = clock64();
+                while (!(landed = mbar_try_wait(&acc_full[buf], (j >> 1) & 1))) {
+                    if (*abort_flag || clock64() - t0 > 8 * a.wait_cycles) break;
+                }
+            }
+            if (!__all_sync(0xffffffffu, landed)) {  // (the tensor-memory loads are warp-wide)
+                set_status(a.status, kTimeoutCode);
+                *abort_flag = 1;
+                break;
+            }
+            tc_fence_after();
             float *orow = a.out + (size_t)row * a.ldo + n0;
-            const bool vec = ((uintptr_t)a.out & 15) == 0 && (a.ldo & 3) == 0 && (!a.bias || ((uintptr_t)a.bias & 15) == 0);
 #pragma unroll 1
             for (int cb = 0; cb < kPfTileN / 32; ++cb) {
                 if (n0 + cb * 32 >= a.N) break;
                 float v[32];
-                tc_ld_32(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(cb * 32), v);
+                tc_ld_32(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * kPfTileN + cb * 32), v);
                 if (row < a.R) {
                     if (vec && n0 + cb * 32 + 31 < a.N) {
                         if (a.bias) {
@@ -167,6 +207,9 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
                     }
                 }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);  // this warp has read its quadrant of the buffer
         }
         tc_fence_before();
     }
@@ -176,7 +219,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_consta
             for (int i = (issued > kPfStages ? issued - kPfStages : 0); i < issued; ++i) mbar_wait(&full[i % kPfStages], (i / kPfStages) & 1);
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(256) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(512) : "memory");
     }
 }
 

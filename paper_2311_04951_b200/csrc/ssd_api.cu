@@ -819,7 +819,8 @@ int gemm_wide(cudaStream_t st, const CUtensorMap *tw, const Operand &X, int rows
     g.out = out; g.bias = bias; g.accumulate = accumulate ? 1 : 0;
     g.ldo = ldo; g.N = N; g.Kd = Kd; g.R = R; g.status = status;
     g.wait_cycles = g_wait_cycles > 0 ? g_wait_cycles : kWaitCycles;
-    LAUNCH(prefill_gemm_kernel, dim3(ceil_div(N, kPfTileN), rows_pad / kPfTileM), kPfThreads, kPfSmem, st, *tw, th, tl, g);
+    const int n_tiles = ceil_div(N, kPfTileN) * ceil_div(R, kPfTileM), sms = g_num_sms > 0 ? g_num_sms : 148;
+    LAUNCH(prefill_gemm_kernel, n_tiles < sms ? n_tiles : sms, kPfThreads, kPfSmem, st, *tw, th, tl, g);
     return SSD_OK;
 }
 
