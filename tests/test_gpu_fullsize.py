@@ -161,6 +161,54 @@ def test_7b_shape_batch_of_eight_matches_the_oracle(llama7b):
     _check_pass_against_oracle(arch, model, omodel, kv, lens, [2, 5, 7], rows_np, K, T, q_np, u_np, S)
 
 
+def test_7b_shape_many_row_prompt_pass_matches_the_oracle(llama7b):
+    """The many-row prompt pass at the 7B shape, all 32 layers: three sequences with seeded caches of ragged
+    lengths are continued by 70, 49 and 3 prompt tokens in one pass (210 rows: two 128-row GEMM tiles at
+    d_ff = 11008 and 172 k-chunks, two 64-row attention tiles over hundreds of cached positions); the appended
+    cache rows of two sequences against the oracle, then a verification pass on top of them."""
+    arch, model = llama7b["arch"], llama7b["model"]
+    od.set_threads(16)
+    omodel = od.Model(arch, llama7b["host_weights"]())
+    Bn, S, P = 3, 1024, 70
+    lens0, n_new = [700, 321, 64], [70, 49, 3]
+    V = arch.vocab
+    kv = B.KV(model, Bn, S)
+    _seeded_fill(kv, 300)
+    B.kv_commit(kv, torch.tensor(lens0, dtype=torch.int32, device="cuda"))
+    prompts = synth.gen_prompt(301, Bn, P, V)
+    oracle = {}
+    for b in (0, 1):
+        oc = omodel.new_cache(S)
+        oc.kv[...] = kv.cache_view()[:, b].float().cpu().numpy()
+        oc.len = lens0[b]
+        oc.feed(prompts[b, :n_new[b]], want_logits=False)
+        oracle[b] = oc
+    B.set_prefill_mode(2)
+    try:
+        nbytes = model.prefill_workspace_bytes(Bn, P)
+        assert nbytes > 0
+        B.kv_prefill(model, kv, torch.from_numpy(prompts).cuda(), torch.tensor(n_new, dtype=torch.int32, device="cuda"),
+                     B.device_buffer(nbytes))
+    finally:
+        B.set_prefill_mode(0)
+    lens1 = [a + b for a, b in zip(lens0, n_new)]
+    assert kv.status() == 0 and kv.lengths().tolist() == lens1
+    for b in (0, 1):
+        g = kv.cache_view()[:, b, :, :, lens0[b]:lens1[b]].float().cpu().numpy()
+        r = oracle[b].kv[:, :, :, lens0[b]:lens1[b]]
+        # (70 rows x 32 layers: the relative term is taken against the row's largest entry - the error of a key or
+        #  value row is a vector whose size goes with the row, and a row whose attention is nearly tied between two
+        #  cached positions carries the roundings of the earlier layers' keys into every entry of the later ones)
+        bad = np.argwhere(np.abs(g - r) > gu.LOGIT_RTOL * np.abs(r).max(axis=-1, keepdims=True) + gu.LOGIT_ATOL)
+        assert bad.shape[0] == 0, (b, bad.shape[0], bad[:12].tolist(), [(float(g[tuple(i)]), float(r[tuple(i)])) for i in bad[:12]])
+        assert (g == r).mean() > 0.5      # (most bf16 entries are the oracle's bit for bit even after 32 layers)
+    K, T = 4, 1.0
+    rows_np = synth.gen_prompt(302, Bn, K + 1, V)
+    q_np = synth.gen_dirichlet_rows(303, Bn * K, V).reshape(Bn, K, V)
+    u_np = np.stack([synth.gen_uniforms(304, b, 0, K + 1) for b in range(Bn)])
+    _check_pass_against_oracle(arch, model, omodel, kv, lens1, [0], rows_np, K, T, q_np, u_np, S)
+
+
 @pytest.mark.parametrize("ctx,M", [(8192, 5), (8192, 17), (16384, 5), (16384, 17)])
 def test_7b_width_long_context_tensor_core_attention_matches_the_oracle(llama7b, ctx, M):
     """The long-context points of the verify sweep through target_verify with the default attention choice,
