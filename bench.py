@@ -42,10 +42,10 @@ NOMINAL_HBM_GBS = 8000.0
 # An entry is dropped (None) when the kernel has changed since its capture.
 NCU_TRAFFIC = {
     # workload: (captured workload, dram bytes of the captured launch, layers captured)
-    "llama-7b-b8": ("llama-7b-l4-b8", 3.1859e9, 4),        # profiles/forward_kernel_llama-7b-l4-b8_verify.md
-    "llama-7b-l4-b8": ("llama-7b-l4-b8", 3.1859e9, 4),
+    "llama-7b-b8": ("llama-7b-l4-b8", 3.1874e9, 4),        # profiles/forward_kernel_llama-7b-l4-b8_verify.md
+    "llama-7b-l4-b8": ("llama-7b-l4-b8", 3.1874e9, 4),
     "llama-7b-l4-ctx8k": ("llama-7b-l4-ctx8k", 2.4935e9, 4),  # profiles/forward_kernel_llama-7b-l4-ctx8k_verify.md
-    "neox-1.4b": ("neox-1.4b", 2.6746e9, 24),               # profiles/forward_kernel_neox-1.4b_verify.md
+    "neox-1.4b": ("neox-1.4b", 2.6756e9, 24),               # profiles/forward_kernel_neox-1.4b_verify.md
 }
 
 # bench workloads: name -> preset (+ overrides)
@@ -545,6 +545,19 @@ def prompt_pass(target, arch, torch, B, synth, Bn, P, seed):
             "frac_of_bf16_peak": 2 * useful / t / 1e12 / peak, "device_status": int(status)}
 
 
+def run_prompt_pass(args):
+    """The prompt pass alone: the workload's target, its batch, --prompt-pass tokens per sequence."""
+    import torch
+    from paper_2311_04951_b200 import binding as B, synth
+    torch.cuda.set_device(0)
+    cfg = resolve(args.workload)
+    arch = cfg["target"]
+    target = B.Model(arch, random_weights_on_device(arch, cfg["seeds"]["w"], torch, **late_scaling(cfg)))
+    out = prompt_pass(target, arch, torch, B, synth, cfg["batch"], args.prompt_pass, cfg["seeds"]["prompt"])
+    out["workload"] = args.workload
+    return out
+
+
 def verify_batch1(target, arch, torch, B, synth, reps, ctx=2048, rows_list=(1, 4, 5)):
     """One sequence, `ctx` cached positions (seeded N(0,1) fill), verification passes over 1, 4 and 5 rows:
     latency, algorithmic GB/s, fraction of the HBM peak, and the ratio to the one-row pass."""
@@ -770,13 +783,17 @@ def main(argv=None):
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="isolated verify-pass sweep at the 7B shape (one GPU)")
+    ap.add_argument("--prompt-pass", type=int, default=0, metavar="TOKENS",
+                    help="only the prompt pass of the workload's target: batch x TOKENS tokens (one GPU)")
     args = ap.parse_args(argv)
-    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.sweep:
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.sweep and not args.prompt_pass:
         return launch_replicas(args, argv)
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     if args.sweep:
         line = run_sweep(args) if rank == 0 else None
+    elif args.prompt_pass:
+        line = run_prompt_pass(args) if rank == 0 else None
     elif args.impl == "reference":
         line = run_reference(args, rank, world)
     else:
