@@ -54,6 +54,7 @@ WORKLOADS = {
     "llama-7b-b1": dict(preset="llama-7b", batch=1, prompt=2048),
     "neox-1.4b": dict(preset="neox-1.4b"),
     "neox-2.7b": dict(preset="neox-2.7b"),
+    "neox-12b": dict(preset="neox-12b"),
     # four-layer cuts of the 7B shape, small enough for a full profiler capture: the same per-layer phases;
     # time and bytes scale with the layers
     "llama-7b-l4-ctx8k": dict(preset="llama-7b", batch=1, prompt=8192, layers=4),
@@ -435,6 +436,9 @@ def run_ours(args, rank, world):
     # ---------------- the prompt pass (fills the cache before sampling starts) ----------------
     pp = prompt_pass(target, arch, torch, B, synth, Bn, min(P - 1, 1024), seeds["prompt"]) if arch.dtype and rank == 0 else None
 
+    # ---------------- whole generations of 40 and 100 new tokens, as a caller times them ----------------
+    wc = whole_call(engine, target, draft, Bn, K, T, prompts.cpu().numpy(), synth, seeds["u"] + 7, torch) if rank == 0 else None
+
     # ---------------- aggregate over ranks ----------------
     tot_tokens, tot_e2e_tokens, max_ms, max_e2e = aggregate_replicas(
         dist, [spec_tokens, e2e_tokens], [spec_ms, e2e_s], "cuda")
@@ -482,6 +486,8 @@ def run_ours(args, rank, world):
         line["verify_b1"] = vb1
     if pp is not None:
         line["prompt_pass"] = pp
+    if wc is not None:
+        line["whole_call"] = wc
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         host_w = (weights_to_host(t_dev, torch), None if d_dev is None else weights_to_host(d_dev, torch))
         del t_dev, d_dev, target, draft
@@ -543,6 +549,33 @@ def prompt_pass(target, arch, torch, B, synth, Bn, P, seed):
             "projection_tflops_useful": useful / t / 1e12, "projection_tflops_tensor": 2 * useful / t / 1e12,
             "bf16_peak_tflops": peak, "peak_source": which + " (sustained cuBLAS bf16)",
             "frac_of_bf16_peak": 2 * useful / t / 1e12 / peak, "device_status": int(status)}
+
+
+def whole_call(engine, target, draft, Bn, K, T, prompts_np, synth, seed, torch, n_list=(40, 100)):
+    """Wall-clock time of whole generations as a caller sees them - prompt pass, iterations until every sequence
+    has N new tokens, host polling of the counters included - for N = 40 and 100 new tokens, speculative and
+    autoregressive (the quantity the paper's Table of timings reports per prompt)."""
+    P = prompts_np.shape[1]
+    out = {"prompt_tokens": P, "n_new": list(n_list), "speculative_s": [], "autoregressive_s": [], "iterations": []}
+    for N in n_list:
+        for k, dm, key in ((K, draft, "speculative_s"), (0, None, "autoregressive_s")):
+            max_len = P + (N + 8) * (k + 1) + 16
+            if target.arch.pos == 0:
+                max_len = min(max_len, target.arch.max_pos)
+            eng = engine.Engine(target, dm, Bn, max_len, k, T, (N + 8) * (k + 1))
+            width = 2 * k + 1
+            u = lambda s_, it: synth.gen_uniforms(seed, s_, it, width)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            res = eng.generate(prompts_np, N, u)
+            torch.cuda.synchronize()
+            out[key].append(time.perf_counter() - t0)
+            if k:
+                out["iterations"].append(int(res["iterations"]))
+            del eng
+            torch.cuda.empty_cache()
+    out["speedup"] = [a / s for a, s in zip(out["autoregressive_s"], out["speculative_s"])]
+    return out
 
 
 def run_prompt_pass(args):

@@ -89,6 +89,13 @@ PRESETS: Dict[str, dict] = {
     "neox-2.7b": dict(target=neox_like(32, 2560, 32, 10240, 50304), draft="prefix:4",
                       batch=1, prompt=512, K=8, temperature=0.0, new_tokens=512,
                       seeds=dict(w=21, prompt=23, u=24)),
+    # the shape pair of the paper's own experiment (Section "Experimental results": a 12B target with a 3B draft,
+    # K = 5, 40 and 100 new tokens): NeoX-style blocks, 36 layers x 5120 (40 heads of 128, rotary on a quarter of
+    # the head) and 32 layers x 2560 (32 heads of 80); random-init stand-ins, batch 1
+    "neox-12b": dict(target=neox_like(36, 5120, 40, 20480, 50304).replace(rotary_dim=32),
+                     draft=neox_like(32, 2560, 32, 10240, 50304),
+                     batch=1, prompt=128, K=5, temperature=1.0, new_tokens=100,
+                     seeds=dict(w=41, wd=42, prompt=43, u=44)),
     "llama-7b": dict(target=llama_like(32, 4096, 32, 11008, 32000),
                      draft=llama_like(4, 1024, 16, 2752, 32000),
                      batch=8, prompt=2048, K=4, temperature=1.0, new_tokens=256,
