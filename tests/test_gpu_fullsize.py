@@ -232,6 +232,26 @@ def test_7b_width_long_context_tensor_core_attention_matches_the_oracle(llama7b,
     _check_pass_against_oracle(arch4, model4, omodel, kv, [ctx], [0], rows_np, K, T, q_np, u_np, S)
 
 
+def test_12b_width_pass_matches_the_oracle():
+    """The 12B NeoX shape at full width (d 5120: rows wider than the 4096 columns a norm phase keeps in registers,
+    40 heads of 128 with rotary on 32 of them, MLP 20480 = 320 k-chunks, vocabulary 50304), two layers, K = 5 at
+    T = 1 on a seeded cache of 300 positions, against the oracle."""
+    import bench
+    arch = synth.PRESETS["neox-12b"]["target"].replace(n_layers=2)
+    model = B.Model(arch, bench.random_weights_on_device(arch, 41, torch))
+    od.set_threads(16)
+    omodel = od.Model(arch, bench.weights_to_host(model.tensors, torch))
+    K, T, ctx, S = 5, 1.0, 300, 320
+    V = arch.vocab
+    kv = B.KV(model, 1, S)
+    _seeded_fill(kv, 12)
+    B.kv_commit(kv, torch.tensor([ctx], dtype=torch.int32, device="cuda"))
+    rows_np = synth.gen_prompt(121, 1, K + 1, V)
+    q_np = synth.gen_dirichlet_rows(122, K, V).reshape(1, K, V)
+    u_np = synth.gen_uniforms(123, 0, 0, K + 1).reshape(1, K + 1)
+    _check_pass_against_oracle(arch, model, omodel, kv, [ctx], [0], rows_np, K, T, q_np, u_np, S)
+
+
 def test_2p7b_width_greedy_pass_matches_the_oracle():
     """The 2.7B NeoX shape at full width (d 2560, 32 heads of 80, MLP 10240, vocabulary 50304), four layers,
     K = 8, greedy: 9 rows in one pass against the oracle; the greedy decisions are the oracle's unless the
