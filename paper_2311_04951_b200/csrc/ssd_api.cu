@@ -508,7 +508,8 @@ template <int NT>
 int launch_forward_nt(FwdParams p, const void *ws_base, size_t ws_bytes, cudaStream_t st) {
     constexpr size_t stage = kWTileBytesP + 2 * NT * 8 * kTileK * 2;
     size_t attn = align_up(attn_scratch_bytes(p.Dh), 128);
-    if (p.attn_tc && attn < (size_t)kTcScratchBytes) attn = kTcScratchBytes;
+    if (p.attn_tc == 1 && attn < (size_t)kTcScratchBytes) attn = kTcScratchBytes;
+    if (p.attn_tc == 2) attn = kRowsScratchBytes;
     const size_t tail = 24 * 32 + 64 + 16 + sizeof(Shared) + 16 * sizeof(double) + kEpiBytes + 256;  // barriers, small state, epilogue tile
     const size_t total = (size_t)kSmemBudget - 1024 - tail;
     // upper slots share their bytes with the attention scratch; two slots never do where they fit
@@ -615,7 +616,12 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     const int groups = kv->B * a.n_heads * ((M + 15) / 16);
     p.attn_tc = 0;
     p.kv_rows_per_layer = kv->B * 2 * a.n_heads * kv->S;
-    if (a.head_dim == 128 && kv->tm_rows_ok && g_attn_mode != 1) {
+    // Passes of one or two rows per sequence (draft steps, decode steps): items on the FP32 pipe.
+    const bool rows_form = M <= kRowsMax && (a.head_dim == 64 || a.head_dim == 128) && (g_attn_mode == 0 || g_attn_mode == 3);
+    if (rows_form) {
+        plan_split(groups, ctx, &p.chunk, &p.n_split, kAttnTile);
+        p.attn_tc = 2;
+    } else if (a.head_dim == 128 && kv->tm_rows_ok && g_attn_mode != 1 && g_attn_mode != 3) {
         plan_split(groups, ctx, &p.chunk, &p.n_split, kTcChunk);
         if (p.chunk >= 1024 || g_attn_mode == 2) {
             p.attn_tc = 1;
@@ -972,7 +978,7 @@ int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n
 }
 
 int ssd_set_attention_mode(int mode) {
-    if (mode < 0 || mode > 2) return SSD_E_ARG;
+    if (mode < 0 || mode > 3) return SSD_E_ARG;
     g_attn_mode = mode;
     return SSD_OK;
 }

@@ -74,13 +74,29 @@ def test_parallel_residual_out_projection_behind_the_attention_count(lens, M, mo
     _forward_over_seeded_cache(synth.neox_like(3, 256, 2, 512, 520), lens, M, mode)
 
 
+@pytest.mark.parametrize("arch,lens,M", [
+    (synth.llama_like(2, 256, 2, 512, 512), [3000, 120], 2),      # head 128: several splits per head, ragged lengths
+    (synth.llama_like(2, 256, 2, 512, 512), [1000, 0], 1),        # one row; an empty cache beside it
+    (synth.llama_like(2, 256, 2, 512, 512), [255, 7], 2),         # blocks that end inside a load; fewer positions than a block
+    (synth.llama_like(2, 256, 4, 512, 512), [2100, 77, 0], 2),    # head 64: 8 lanes per position, 16 positions per block
+    (synth.llama_like(2, 256, 4, 512, 512), [513, 64, 31], 1),
+    (synth.neox_like(3, 256, 4, 512, 520), [700, 90], 2),         # parallel residual: the out-projection waits for the attention count
+    (synth.llama_like(1, 4096, 32, 512, 512), [1151, 127, 1152, 64, 300], 2),   # 160 (sequence, head) items on 148 SMs
+])
+def test_few_row_passes_on_the_fp32_attention_items(arch, lens, M):
+    """Passes of one or two rows per sequence (draft steps, decode steps) take the FP32 attention items: per-warp
+    position blocks, copy ring private to the warp, the rows of the pass appended by the owning split, merge of the
+    eight warps and of the splits."""
+    _forward_over_seeded_cache(arch, lens, M, 3, scale=1.5 if arch.d_model == 4096 else 6.0)
+
+
 def _forward_over_seeded_cache(arch, lens, M, mode, scale=6.0):
     """Whole verification pass (single forward kernel) of a head-128 model over a seeded cache:
     logits of all rows and the appended cache rows against the oracle.  Exercises the tensor-core
     attention (mode 2) and the warp-MMA attention (mode 1): splits of several chunks, the merge of
     splits, empty splits, more than 16 rows per sequence, and rows of the pass that cross a chunk
     boundary."""
-    assert arch.head_dim == 128
+    assert arch.head_dim in (64, 128)
     from tests import gpu_util as gu
     ws_np = gu.scaled_weights(synth, arch, 11, scale)
     model = B.Model(arch, B.upload_weights(arch, ws_np))
@@ -104,7 +120,7 @@ def _forward_over_seeded_cache(arch, lens, M, mode, scale=6.0):
     u = torch.full((Bn, M), 0.5, device=dev)
     B.set_attention_mode(mode)
     try:
-        B.target_verify(model, kv, torch.from_numpy(rows).to(dev), K, q, u, 1.0, n_acc, nxt, 1, None, ws)
+        B.target_verify(model, kv, torch.from_numpy(rows).to(dev), K, q if K else None, u, 1.0, n_acc, nxt, 1, None, ws)
         got = B.last_logits(model, Bn, M, ws).cpu().numpy()
     finally:
         B.set_attention_mode(0)
