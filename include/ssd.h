@@ -105,13 +105,15 @@ int ssd_set_prefill_mode(int mode);
  * step instead (same results up to fp32 summation order; kept for comparison). */
 int ssd_set_persistent(int enable);
 
-/* The single forward kernel has two forms of the K-query attention over the cache (Section "KV Caching":
- * the new rows attend to the stored keys / values): items on warp-level MMAs, 64 positions per step,
- * and - head dimension 128 only - items on the tcgen05 tensor core with the scores in tensor memory,
- * 128 positions per step, which start more slowly but stream twice as fast.  mode 0 (default) picks
- * per pass (tensor-core items from 1024 positions per split), 1 forces the first form, 2 the second
- * wherever it applies.  Same results up to fp32 summation order; for comparison and tests.
- * SSD_E_ARG for any other mode. */
+/* The single forward kernel has three forms of the K-query attention over the cache (Section "KV Caching":
+ * the new rows attend to the stored keys / values): items on warp-level MMAs, 64 positions per step;
+ * - head dimension 128 only - items on the tcgen05 tensor core with the scores in tensor memory, 128
+ * positions per step, which start more slowly but stream twice as fast; and - passes of one or two rows
+ * per sequence at head dimension 64 or 128 (draft steps, decode steps) - items on the FP32 pipe with the
+ * queries and the output in registers.  mode 0 (default) picks per pass (FP32 items where they apply, else
+ * tensor-core items from 1024 positions per split), 1 forces the first form, 2 the second wherever it
+ * applies, 3 the third where it applies and the first elsewhere.  Same results up to fp32 summation order;
+ * for comparison and tests.  SSD_E_ARG for any other mode. */
 int ssd_set_attention_mode(int mode);
 
 /* A layer-skip draft: the first n_layers layers of `target` plus its final norm and LM head
