@@ -1896,7 +1896,9 @@ __device__ __forceinline__ void attention_phase(const FwdParams &p, int layer, u
     const int items = p.B * p.H * p.n_split * MT;
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
         if (p.attn_tc == 1) attention_item_tc(p, layer, item, scratch, sh);
+        else if (p.attn_tc == 2 && p.Dh == 128 && p.M == 1) attention_item_rows<16, 1>(p, layer, item, scratch, sh);
         else if (p.attn_tc == 2 && p.Dh == 128) attention_item_rows<16, kRowsMax>(p, layer, item, scratch, sh);
+        else if (p.attn_tc == 2 && p.M == 1) attention_item_rows<8, 1>(p, layer, item, scratch, sh);
         else if (p.attn_tc == 2) attention_item_rows<8, kRowsMax>(p, layer, item, scratch, sh);
         else attention_item(p, layer, item, scratch, sh);
     }
