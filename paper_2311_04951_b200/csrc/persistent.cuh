@@ -336,6 +336,23 @@ __device__ __forceinline__ void tc_ld_16x32(uint32_t taddr, float (&v)[16]) {
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// the same shape eight times along the columns: 16 lanes x 64 columns in one round trip
+__device__ __forceinline__ void tc_ld_16x64(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,"
+        "%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 __device__ __forceinline__ void red_add_v4(float *dst, float4 v) {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
                  : "memory");
@@ -2081,13 +2098,13 @@ __device__ __noinline__ void run_gemm(const FwdParams &p, int gi, uint8_t *smem)
                         const int wq = kM == 64 ? q : (q >> 1), half = kM == 64 ? 0 : (q & 1);
                         if (wq == warp) {
                             const uint32_t ta = tmem_base + ((uint32_t)(warp * 32 + half * 16) << 16) + (uint32_t)(b * kAccStride);
-                            for (int cg = 0; cg < kTileNP / 32; ++cg) {
-                                if (t * kTileNP + cg * 32 >= g.N) break;
-                                float v[16];
-                                tc_ld_16x32(ta + (uint32_t)(cg * 32), v);
+                            for (int cg = 0; cg < kTileNP / 64; ++cg) {  // 64 columns per tensor-memory round trip
+                                if (t * kTileNP + cg * 64 >= g.N) break;
+                                float v[32];
+                                tc_ld_16x64(ta + (uint32_t)(cg * 64), v);
 #pragma unroll
-                                for (int k = 0; k < 4; ++k)
-                                    *reinterpret_cast<float2 *>(epi_tile + g8 * kEpiPitch + cg * 32 + 8 * k + 2 * t4) =
+                                for (int k = 0; k < 8; ++k)
+                                    *reinterpret_cast<float2 *>(epi_tile + g8 * kEpiPitch + cg * 64 + 8 * k + 2 * t4) =
                                         make_float2(v[4 * k] + v[4 * k + 2], v[4 * k + 1] + v[4 * k + 3]);
                             }
                         }
