@@ -98,7 +98,9 @@ size_t ssd_model_desc_bytes(const ssd_arch *arch);
 size_t ssd_prefill_workspace_bytes(const ssd_model *m, int batch, int rows_per_seq);
 
 /* Which form kv_prefill takes: 0 (default) the many-row form from 256 rows per pass, 1 never,
- * 2 wherever the model and the workspace allow it (for tests on small shapes).  SSD_E_ARG otherwise. */
+ * 2 wherever the model and the workspace allow it (for tests on small shapes), 3 as 2 but with the
+ * causal attention on warp-level MMAs also where the tcgen05 form (head dimension 128) applies.
+ * SSD_E_ARG otherwise. */
 int ssd_set_prefill_mode(int mode);
 
 /* bf16 models run the whole forward as one cooperative kernel by default; 0 selects one launch per

@@ -515,4 +515,293 @@ __global__ void __launch_bounds__(kPaThreads) prefill_attn_kernel(const PfAttnAr
     }
 }
 
+// prefill_attn_tc_kernel (head dim 128): the same causal attention on the 5th-generation tensor core, 128 query rows
+// of one (sequence, head) per CTA, 128 positions per chunk, scores, probabilities and output in tensor memory:
+//   S [128 rows x 128 positions] = Q (bf16 hi + lo, 128-byte-swizzled tiles in shared memory) x K chunk^T (straight
+//                                  from the TMA copy of the cache): 2 x 8 MMAs of K = 16 head dims;
+//   thread r of warps 0-3 owns query row r = tensor-memory lane r: it reads its row of S, keeps the row's running
+//   maximum and sum in registers (no exchange between threads), and writes P = exp2(S - max) back over the same
+//   columns as packed bf16 hi and lo (per group of 32 positions: 16 columns hi, 16 columns lo);
+//   O [128 rows x 128 head dims] += P (hi, then lo: the A operand read from tensor memory) x V chunk (the B operand,
+//                                  head dims contiguous: MN-major): 2 x 8 MMAs of K = 16 positions.
+// S is double-buffered (256 columns) so that the scores of chunk c + 1 are computed while the threads work on chunk
+// c; O takes 128 columns.  The running maximum is only raised when a chunk exceeds it by more than 2^8 (the sums and
+// O absorb the factor), so that rescaling O - a read and a write of the thread's 128 columns - is rare.
+// Warp 4 issues the MMAs, warp 5 the K / V copies (two stages each).  Every wait is bounded.
+constexpr int kPtRows = 128, kPtChunk = 128, kPtThreads = 192;
+constexpr int kPtQBytes = 2 * 128 * 128;             // one of hi / lo: two 64-column panels of 128 rows x 128 bytes
+constexpr int kPtKvBytes = 2 * 128 * 128;            // one K or V chunk, the same shape
+constexpr size_t kPtSmem = 1024 + 2 * kPtQBytes + 4 * kPtKvBytes + 256;
+constexpr float kPtMaxSlack = 8.f;
+
+struct PtAttnArgs {
+    const float *q;              // [B * M, d] position-encoded queries
+    const int32_t *len;          // [B] committed lengths
+    const int32_t *n_eff;        // [B] rows fed per sequence
+    __nv_bfloat16 *out_hi, *out_lo;  // [B * M, d]
+    int M, H, S, d;
+    int kv_row0;                 // first row of this layer in the cache seen as rows of 128 bf16
+    float scale;
+    long long wait_cycles;
+    int32_t *status;
+};
+
+__device__ __forceinline__ void tc_st_16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n"
+        "tcgen05.wait::st.sync.aligned;\n" ::"r"(taddr),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+        "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] x B[smem descriptor]
+__device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__global__ void __launch_bounds__(kPtThreads, 1)
+prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmKV, const PtAttnArgs a) {
+    extern __shared__ uint8_t pt_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)pt_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *qhi = smem, *qlo = smem + kPtQBytes, *kring = smem + 2 * kPtQBytes, *vring = kring + 2 * kPtKvBytes;
+    uint64_t *bars = (uint64_t *)(vring + 2 * kPtKvBytes);
+    uint64_t *k_full = bars, *k_free = bars + 2, *v_full = bars + 4, *v_free = bars + 6, *s_full = bars + 8;
+    uint64_t *p_ready = bars + 10, *o_done = bars + 11;
+    uint32_t *tmem_slot = (uint32_t *)(bars + 12);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    constexpr int Dh = 128;
+    const int mt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int len = a.len[b], n = a.n_eff[b];
+    const int m_base = mt * kPtRows, r0 = b * a.M;
+    const int rows_fed = max(0, min(kPtRows, n - m_base));
+    if (rows_fed == 0) {  // nothing fed in this tile: zeros for its rows
+        for (int i = tid; i < kPtRows * (Dh / 8); i += kPtThreads) {
+            const int m = m_base + i / (Dh / 8);
+            if (m < a.M) {
+                const size_t off = (size_t)(r0 + m) * a.d + h * Dh + (i % (Dh / 8)) * 8;
+                *reinterpret_cast<uint4 *>(a.out_hi + off) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4 *>(a.out_lo + off) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        return;
+    }
+    const int p_end = min(len + m_base + rows_fed, a.S);  // positions any row of this tile sees
+    const int n_chunks = (p_end + kPtChunk - 1) / kPtChunk;
+    const int krow0 = a.kv_row0 + ((b * 2) * a.H + h) * a.S, vrow0 = krow0 + a.H * a.S;
+
+    if (warp == 4) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(512)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        for (int i = 0; i < 10; ++i) mbar_init(&bars[i], 1);
+        mbar_init(p_ready, 128);
+        mbar_init(o_done, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // Q rows of this tile as bf16 hi / lo: thread = row (warps 0-3)
+    if (tid < kPtRows) {
+        const int m = m_base + tid;
+        const float *src = a.q + (size_t)(r0 + m) * a.d + h * Dh;
+#pragma unroll 1
+        for (int g8 = 0; g8 < Dh / 8; ++g8) {
+            float qv[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) qv[u] = 0.f;
+            if (m < n) {
+                const float4 x0 = *reinterpret_cast<const float4 *>(src + g8 * 8), x1 = *reinterpret_cast<const float4 *>(src + g8 * 8 + 4);
+                qv[0] = x0.x; qv[1] = x0.y; qv[2] = x0.z; qv[3] = x0.w; qv[4] = x1.x; qv[5] = x1.y; qv[6] = x1.z; qv[7] = x1.w;
+            }
+            __nv_bfloat16 hq[8], lq[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                hq[u] = __float2bfloat16_rn(qv[u]);
+                lq[u] = __float2bfloat16_rn(qv[u] - __bfloat162float(hq[u]));
+            }
+            const uint32_t off = (uint32_t)(g8 >> 3) * 16384u + sw128(tid, g8 & 7);
+            *reinterpret_cast<uint4 *>(qhi + off) = *reinterpret_cast<uint4 *>(hq);
+            *reinterpret_cast<uint4 *>(qlo + off) = *reinterpret_cast<uint4 *>(lq);
+        }
+    }
+    fence_async_proxy();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t tS = tmem, tO = tmem + 256;  // S / P of chunk c at tS + 128 (c & 1)
+    auto wait = [&](uint64_t *bar, uint32_t parity) {  // keeps every role's control flow intact once anything has timed out
+        if (*abort_flag) return;
+        const long long t0 = clock64();
+        while (!mbar_try_wait(bar, parity)) {
+            if (*abort_flag) return;
+            if (clock64() - t0 > a.wait_cycles) {
+                set_status(a.status, kTimeoutCode);
+                *abort_flag = 1;
+                return;
+            }
+        }
+    };
+
+    if (warp == 5) {
+        if (lane == 0) {
+            int issued_k = 0, issued_v = 0;
+            for (int c = 0; c < n_chunks && !*abort_flag; ++c) {
+                const int s = c & 1;
+                if (c >= 2) wait(&k_free[s], ((c >> 1) - 1) & 1);
+                if (*abort_flag) break;
+                mbar_expect_tx(&k_full[s], kPtKvBytes);
+                tma_load_2d(kring + s * kPtKvBytes, &tmKV, 0, krow0 + c * kPtChunk, &k_full[s]);
+                tma_load_2d(kring + s * kPtKvBytes + 16384, &tmKV, 64, krow0 + c * kPtChunk, &k_full[s]);
+                ++issued_k;
+                if (c >= 2) wait(&v_free[s], ((c >> 1) - 1) & 1);
+                if (*abort_flag) break;
+                mbar_expect_tx(&v_full[s], kPtKvBytes);
+                tma_load_2d(vring + s * kPtKvBytes, &tmKV, 0, vrow0 + c * kPtChunk, &v_full[s]);
+                tma_load_2d(vring + s * kPtKvBytes + 16384, &tmKV, 64, vrow0 + c * kPtChunk, &v_full[s]);
+                ++issued_v;
+            }
+            if (*abort_flag) {  // error path only: copies still in flight into this CTA's shared memory
+                for (int c = max(0, issued_k - 2); c < issued_k; ++c) mbar_wait(&k_full[c & 1], (c >> 1) & 1);
+                for (int c = max(0, issued_v - 2); c < issued_v; ++c) mbar_wait(&v_full[c & 1], (c >> 1) & 1);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 4) {
+        if (lane == 0) {
+            const uint32_t idS = umma_idesc_bf16(128, 128), idO = umma_idesc_bf16(128, 128) | (1u << 16);  // B of P V: MN-major
+            auto issue_s = [&](int c) {
+                const int s = c & 1;
+                wait(&k_full[s], (c >> 1) & 1);
+                if (*abort_flag) return;
+                tc_fence_after();
+                const uint32_t ka = smem_u32(kring + s * kPtKvBytes), qa = smem_u32(qhi), ql = smem_u32(qlo);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)  // k = 16 head dims per step; panel ks / 4
+                    tc_mma_bf16(tS + 128 * s, umma_desc(qa + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                                umma_desc(ka + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024), idS, ks ? 1u : 0u);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    tc_mma_bf16(tS + 128 * s, umma_desc(ql + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                                umma_desc(ka + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024), idS, 1u);
+                tc_commit(&s_full[s]);
+                tc_commit(&k_free[s]);
+            };
+            issue_s(0);
+            for (int c = 0; c < n_chunks && !*abort_flag; ++c) {
+                const int s = c & 1;
+                if (c + 1 < n_chunks) issue_s(c + 1);
+                wait(p_ready, c & 1);
+                wait(&v_full[s], (c >> 1) & 1);
+                if (*abort_flag) break;
+                tc_fence_after();
+                const uint32_t va = smem_u32(vring + s * kPtKvBytes), tP = tS + 128 * s;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)  // k = 16 positions per step: two 8-row groups of the V tile; P hi
+                    tc_mma_bf16_ta(tO, tP + 32 * (ks >> 1) + 8 * (ks & 1), umma_desc(va + ks * 2048, 16384, 1024), idO, (c | ks) ? 1u : 0u);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)  // P lo
+                    tc_mma_bf16_ta(tO, tP + 32 * (ks >> 1) + 16 + 8 * (ks & 1), umma_desc(va + ks * 2048, 16384, 1024), idO, 1u);
+                tc_commit(o_done);
+                tc_commit(&v_free[s]);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------- softmax and output: thread = query row = tensor-memory lane ----------------
+        const int m = m_base + tid;
+        const int last = m < n ? len + m : -1;  // last visible position
+        const uint32_t lane_sel = (uint32_t)(warp * 32) << 16;
+        const float sc = a.scale * 1.4426950408889634f;
+        float m_run = -INFINITY, l_run = 0.f;
+        for (int c = 0; c < n_chunks; ++c) {
+            const uint32_t tSc = tS + 128 * (c & 1) + lane_sel;
+            const int pos0 = c * kPtChunk;
+            wait(&s_full[c & 1], (c >> 1) & 1);
+            tc_fence_after();
+            float mc = -INFINITY;
+#pragma unroll 1
+            for (int g = 0; g < 4; ++g) {
+                float v[32];
+                tc_ld_32(tSc + 32 * g, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (pos0 + 32 * g + i <= last) mc = fmaxf(mc, v[i] * sc);
+            }
+            const float m_new = (mc > m_run + kPtMaxSlack || m_run == -INFINITY) ? fmaxf(m_run, mc) : m_run;
+            const float f = m_new > -INFINITY ? exp2f(m_run - m_new) : 1.f;  // 0 on the first non-empty chunk
+            float sum = 0.f;
+#pragma unroll 1
+            for (int g = 0; g < 4; ++g) {
+                float v[32];
+                tc_ld_32(tSc + 32 * g, v);
+                uint32_t hi[16], lo[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int pos = pos0 + 32 * g + 2 * i;
+                    const float p0 = (pos <= last && m_new > -INFINITY) ? exp2f(v[2 * i] * sc - m_new) : 0.f;
+                    const float p1 = (pos + 1 <= last && m_new > -INFINITY) ? exp2f(v[2 * i + 1] * sc - m_new) : 0.f;
+                    sum += p0 + p1;
+                    const __nv_bfloat162 hv = __floats2bfloat162_rn(p0, p1);
+                    hi[i] = *reinterpret_cast<const uint32_t *>(&hv);
+                    lo[i] = pack_bf16x2(p0 - __low2float(hv), p1 - __high2float(hv));
+                }
+                tc_st_16(tSc + 32 * g, hi);
+                tc_st_16(tSc + 32 * g + 16, lo);
+            }
+            l_run = l_run * f + sum;
+            m_run = m_new;
+            // the accumulated O row moves to the new maximum, once P V of the previous chunk has written it; the
+            // tensor-memory loads and stores are warp-wide, so the warp goes together (f = 1 where nothing moved)
+            if (c > 0 && __any_sync(0xffffffffu, f != 1.f)) {
+                wait(o_done, (c - 1) & 1);
+                tc_fence_after();
+#pragma unroll 1
+                for (int g = 0; g < 4; ++g) {
+                    float o[32];
+                    tc_ld_32(tO + lane_sel + 32 * g, o);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] *= f;
+                    tc_st_32(tO + lane_sel + 32 * g, o);
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(p_ready);
+        }
+        wait(o_done, (n_chunks - 1) & 1);
+        tc_fence_after();
+        {
+            const bool store = m < a.M && !*abort_flag;  // (the loads are warp-wide: every lane takes them)
+            const float inv = (m < n && l_run > 0.f) ? 1.f / l_run : 0.f;
+            const size_t base = (size_t)(r0 + (store ? m : 0)) * a.d + h * Dh;
+#pragma unroll 1
+            for (int g = 0; g < 4; ++g) {
+                float o[32];
+                tc_ld_32(tO + lane_sel + 32 * g, o);
+                if (store) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        store_hilo4(a.out_hi, a.out_lo, base + 32 * g + 4 * i,
+                                    make_float4(o[4 * i] * inv, o[4 * i + 1] * inv, o[4 * i + 2] * inv, o[4 * i + 3] * inv));
+                }
+            }
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 4) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(512) : "memory");
+    }
+}
+
 }  // namespace ssd

@@ -165,6 +165,7 @@ int init_device_once() {
     rc |= set_smem(attn_partial_kernel<__nv_bfloat16, 32>, attn_smem<__nv_bfloat16, 32>(128));
     rc |= set_smem(prefill_gemm_kernel, kPfSmem);
     rc |= set_smem(prefill_attn_kernel, prefill_attn_smem(128));
+    rc |= set_smem(prefill_attn_tc_kernel, kPtSmem);
     if (rc) return SSD_E_CUDA;
     g_attr_done = true;
     return SSD_OK;
@@ -884,8 +885,20 @@ int forward_wide(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_stride
         at.out_hi = w.ao.hi; at.out_lo = w.ao.lo;
         at.M = C; at.H = a.n_heads; at.Dh = a.head_dim; at.S = kv->S; at.d = d;
         at.scale = 1.0f / sqrtf((float)a.head_dim);
-        LAUNCH(prefill_attn_kernel, dim3(ceil_div(C, kPaRows), a.n_heads, B), kPaThreads, prefill_attn_smem(a.head_dim), st,
-               at);
+        if (a.head_dim == 128 && kv->tm_rows_ok && g_prefill_mode != 3) {  // tensor-core form
+            PtAttnArgs pt;
+            pt.q = w.qrot; pt.len = kv->len; pt.n_eff = w.ri.n_eff;
+            pt.out_hi = w.ao.hi; pt.out_lo = w.ao.lo;
+            pt.M = C; pt.H = a.n_heads; pt.S = kv->S; pt.d = d;
+            pt.kv_row0 = l * (kv->B * 2 * a.n_heads * kv->S);
+            pt.scale = at.scale;
+            pt.wait_cycles = g_wait_cycles > 0 ? g_wait_cycles : kWaitCycles;
+            pt.status = kv->status;
+            LAUNCH(prefill_attn_tc_kernel, dim3(ceil_div(C, kPtRows), a.n_heads, B), kPtThreads, kPtSmem, st, kv->tm_rows, pt);
+        } else {
+            LAUNCH(prefill_attn_kernel, dim3(ceil_div(C, kPaRows), a.n_heads, B), kPaThreads, prefill_attn_smem(a.head_dim), st,
+                   at);
+        }
         if ((rc = gemm_wide(st, tm + 1, w.ao, Rp, R, d, d, w.x, d, b_o, true, kv->status))) return rc;
         if (!a.parallel_residual) {
             PfNormArgs n2 = norm_args((const float *)lw(m, l, L_LN2G), (const float *)lw(m, l, L_LN2B), w.xn1);
@@ -984,7 +997,7 @@ int ssd_set_attention_mode(int mode) {
 }
 
 int ssd_set_prefill_mode(int mode) {
-    if (mode < 0 || mode > 2) return SSD_E_ARG;
+    if (mode < 0 || mode > 3) return SSD_E_ARG;
     g_prefill_mode = mode;
     return SSD_OK;
 }
@@ -1120,7 +1133,7 @@ int kv_prefill(ssd_model *m, ssd_kv *kv, const int32_t *dev_tokens, const int32_
             int Cw = ceil_div(ceil_div(max_tokens, passes), 16) * 16;
             if (Cw > max_tokens) Cw = max_tokens;
             if (Cw > cap) Cw = cap;
-            if (g_prefill_mode == 2 || kv->B * Cw >= kWideMinRows) {
+            if (g_prefill_mode >= 2 || kv->B * Cw >= kWideMinRows) {
                 const WideWs ww = carve_wide(m, kv->B, Cw, (uint8_t *)dev_ws);
                 const int chunks = ceil_div(max_tokens, Cw);
                 for (int c = 0; c < chunks; ++c) {

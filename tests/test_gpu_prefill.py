@@ -13,9 +13,9 @@ pytestmark = pytest.mark.gpu
 BF16 = [n for n, a in ARCHS.items() if a.dtype == synth.DT_BF16]
 
 
-@pytest.fixture
-def many_row_mode():
-    B.set_prefill_mode(2)
+@pytest.fixture(params=[2, 3], ids=["tc-attention-where-it-applies", "mma-attention"])
+def many_row_mode(request):
+    B.set_prefill_mode(request.param)
     yield
     B.set_prefill_mode(0)
 
