@@ -554,6 +554,23 @@ __device__ __forceinline__ void tc_st_16(uint32_t taddr, const uint32_t (&v)[16]
         "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
         : "memory");
 }
+// 64 consecutive columns of this thread's lane in one round trip
+__device__ __forceinline__ void tc_ld_64(uint32_t taddr, float (&v)[64]) {
+    uint32_t r[64];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32,%33,%34,%35,%36,%37,%38,%39,%40,%41,%42,%43,%44,%45,%46,%47,%48,%49,%50,%51,%52,%53,%54,%55,%56,%57,%58,%59,%60,%61,%62,%63}, [%64];\n"
+        "tcgen05.wait::ld.sync.aligned;\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
+// 32 columns of this thread's lane; completion is awaited by tc_wait_st
+__device__ __forceinline__ void tc_st_32u_nowait(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n" ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31]) : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // D[tmem] (+)= A[tmem] x B[smem descriptor]
 __device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
@@ -609,26 +626,31 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmKV, const PtAttnArg
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // Q rows of this tile as bf16 hi / lo: thread = row (warps 0-3)
+    // Q rows of this tile as bf16 hi / lo (warps 0-3): consecutive threads take consecutive 8-column pieces of a row,
+    // all sixteen loads of a thread in flight together
     if (tid < kPtRows) {
-        const int m = m_base + tid;
-        const float *src = a.q + (size_t)(r0 + m) * a.d + h * Dh;
-#pragma unroll 1
-        for (int g8 = 0; g8 < Dh / 8; ++g8) {
-            float qv[8];
+        float4 x0[16], x1[16];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) qv[u] = 0.f;
+        for (int it = 0; it < 16; ++it) {
+            const int u = it * kPtRows + tid, row = u >> 4, g8 = u & 15, m = m_base + row;
+            x0[it] = x1[it] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (m < n) {
-                const float4 x0 = *reinterpret_cast<const float4 *>(src + g8 * 8), x1 = *reinterpret_cast<const float4 *>(src + g8 * 8 + 4);
-                qv[0] = x0.x; qv[1] = x0.y; qv[2] = x0.z; qv[3] = x0.w; qv[4] = x1.x; qv[5] = x1.y; qv[6] = x1.z; qv[7] = x1.w;
+                const float *src = a.q + (size_t)(r0 + m) * a.d + h * Dh + g8 * 8;
+                x0[it] = __ldg(reinterpret_cast<const float4 *>(src));
+                x1[it] = __ldg(reinterpret_cast<const float4 *>(src + 4));
             }
+        }
+#pragma unroll
+        for (int it = 0; it < 16; ++it) {
+            const int u = it * kPtRows + tid, row = u >> 4, g8 = u & 15;
+            const float qv[8] = {x0[it].x, x0[it].y, x0[it].z, x0[it].w, x1[it].x, x1[it].y, x1[it].z, x1[it].w};
             __nv_bfloat16 hq[8], lq[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                hq[u] = __float2bfloat16_rn(qv[u]);
-                lq[u] = __float2bfloat16_rn(qv[u] - __bfloat162float(hq[u]));
+            for (int e = 0; e < 8; ++e) {
+                hq[e] = __float2bfloat16_rn(qv[e]);
+                lq[e] = __float2bfloat16_rn(qv[e] - __bfloat162float(hq[e]));
             }
-            const uint32_t off = (uint32_t)(g8 >> 3) * 16384u + sw128(tid, g8 & 7);
+            const uint32_t off = (uint32_t)(g8 >> 3) * 16384u + sw128(row, g8 & 7);
             *reinterpret_cast<uint4 *>(qhi + off) = *reinterpret_cast<uint4 *>(hq);
             *reinterpret_cast<uint4 *>(qlo + off) = *reinterpret_cast<uint4 *>(lq);
         }
@@ -728,36 +750,39 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmKV, const PtAttnArg
             const int pos0 = c * kPtChunk;
             wait(&s_full[c & 1], (c >> 1) & 1);
             tc_fence_after();
+            // the row's 128 scores in two round trips, kept in registers for both passes
+            float v0[64], v1[64];
+            tc_ld_64(tSc, v0);
+            tc_ld_64(tSc + 64, v1);
             float mc = -INFINITY;
-#pragma unroll 1
-            for (int g = 0; g < 4; ++g) {
-                float v[32];
-                tc_ld_32(tSc + 32 * g, v);
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (pos0 + 32 * g + i <= last) mc = fmaxf(mc, v[i] * sc);
+            for (int i = 0; i < 64; ++i) {
+                v0[i] = pos0 + i <= last ? v0[i] * sc : -INFINITY;
+                v1[i] = pos0 + 64 + i <= last ? v1[i] * sc : -INFINITY;
+                mc = fmaxf(mc, fmaxf(v0[i], v1[i]));
             }
             const float m_new = (mc > m_run + kPtMaxSlack || m_run == -INFINITY) ? fmaxf(m_run, mc) : m_run;
             const float f = m_new > -INFINITY ? exp2f(m_run - m_new) : 1.f;  // 0 on the first non-empty chunk
+            const float m_ref = m_new > -INFINITY ? m_new : 0.f;             // (all masked: every p is exp2(-inf) = 0)
             float sum = 0.f;
-#pragma unroll 1
-            for (int g = 0; g < 4; ++g) {
-                float v[32];
-                tc_ld_32(tSc + 32 * g, v);
-                uint32_t hi[16], lo[16];
+            auto emit = [&](const float (&v)[64], int half) {  // P of 64 positions: per 32 of them 16 columns hi, 16 lo
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const int pos = pos0 + 32 * g + 2 * i;
-                    const float p0 = (pos <= last && m_new > -INFINITY) ? exp2f(v[2 * i] * sc - m_new) : 0.f;
-                    const float p1 = (pos + 1 <= last && m_new > -INFINITY) ? exp2f(v[2 * i + 1] * sc - m_new) : 0.f;
-                    sum += p0 + p1;
-                    const __nv_bfloat162 hv = __floats2bfloat162_rn(p0, p1);
-                    hi[i] = *reinterpret_cast<const uint32_t *>(&hv);
-                    lo[i] = pack_bf16x2(p0 - __low2float(hv), p1 - __high2float(hv));
+                for (int g = 0; g < 2; ++g) {
+                    uint32_t w[32];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float p0 = exp2f(v[32 * g + 2 * i] - m_ref), p1 = exp2f(v[32 * g + 2 * i + 1] - m_ref);
+                        sum += p0 + p1;
+                        const __nv_bfloat162 hv = __floats2bfloat162_rn(p0, p1);
+                        w[i] = *reinterpret_cast<const uint32_t *>(&hv);
+                        w[16 + i] = pack_bf16x2(p0 - __low2float(hv), p1 - __high2float(hv));
+                    }
+                    tc_st_32u_nowait(tSc + 64 * half + 32 * g, w);
                 }
-                tc_st_16(tSc + 32 * g, hi);
-                tc_st_16(tSc + 32 * g + 16, lo);
-            }
+            };
+            emit(v0, 0);
+            emit(v1, 1);
+            tc_wait_st();
             l_run = l_run * f + sum;
             m_run = m_new;
             // the accumulated O row moves to the new maximum, once P V of the previous chunk has written it; the
@@ -784,14 +809,23 @@ prefill_attn_tc_kernel(const __grid_constant__ CUtensorMap tmKV, const PtAttnArg
             const float inv = (m < n && l_run > 0.f) ? 1.f / l_run : 0.f;
             const size_t base = (size_t)(r0 + (store ? m : 0)) * a.d + h * Dh;
 #pragma unroll 1
-            for (int g = 0; g < 4; ++g) {
-                float o[32];
-                tc_ld_32(tO + lane_sel + 32 * g, o);
+            for (int g = 0; g < 2; ++g) {
+                float o[64];
+                tc_ld_64(tO + lane_sel + 64 * g, o);
                 if (store) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        store_hilo4(a.out_hi, a.out_lo, base + 32 * g + 4 * i,
-                                    make_float4(o[4 * i] * inv, o[4 * i + 1] * inv, o[4 * i + 2] * inv, o[4 * i + 3] * inv));
+                    for (int i = 0; i < 8; ++i) {  // eight head dims: 16 bytes of hi, 16 bytes of lo
+                        uint32_t hw[4], lw[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float y0 = o[8 * i + 2 * e] * inv, y1 = o[8 * i + 2 * e + 1] * inv;
+                            const __nv_bfloat162 hv = __floats2bfloat162_rn(y0, y1);
+                            hw[e] = *reinterpret_cast<const uint32_t *>(&hv);
+                            lw[e] = pack_bf16x2(y0 - __low2float(hv), y1 - __high2float(hv));
+                        }
+                        *reinterpret_cast<uint4 *>(a.out_hi + base + 64 * g + 8 * i) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                        *reinterpret_cast<uint4 *>(a.out_lo + base + 64 * g + 8 * i) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+                    }
                 }
             }
         }
