@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libssd_b200.so")
 SOURCES = ["ssd_api.cu"]
-DEPS = ["ssd_api.cu", "common.cuh", "gemm.cuh", "rowops.cuh", "attention.cuh", "tail.cuh", "persistent.cuh", "prefill.cuh",
+DEPS = ["ssd_api.cu", "common.cuh", "gemm.cuh", "rowops.cuh", "attention.cuh", "tail.cuh", "persistent.cuh", "prefill.cuh", "attn_mma8.cuh",
         os.path.join("..", "..", "include", "ssd.h")]
 
 

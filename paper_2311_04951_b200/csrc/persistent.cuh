@@ -116,7 +116,7 @@ struct alignas(64) FwdParams {
     // tensor-core attention (head dim 128): the whole cache as rows of Dh bf16, box 64 x 128 rows
     CUtensorMap tm_kv;
     const CUtensorMap *tm_kv_ptr;  // where the copy engine can read tm_kv (set by the kernel: see params copy)
-    int attn_tc;             // 0: attention_item (warp MMAs); 1: attention_item_tc; 2: attention_item_rows (FP32, few rows)
+    int attn_tc;             // 0: attention_item (warp MMAs); 1: attention_item_tc; 2: attention_item_rows (FP32, one or two rows); 3: attention_item_mma8 (up to eight rows, hi and lo in one MMA tile)
     int kv_rows_per_layer;   // B * 2 * H * S
     int attn_ctas;           // min(attention items, CTAs): set by the host together with the split plan
     int overlap_out;         // parallel-residual block and at most half of the CTAs on attention
@@ -1431,6 +1431,8 @@ __device__ __noinline__ void attention_item_rows(const FwdParams &p, int layer, 
     named_bar(3, kAttnThreadsP);  // scratch is free for the next item
 }
 
+#include "attn_mma8.cuh"
+
 // ---- attention on tcgen05 (head dim 128) ----------------------------------------------------------
 // The same item as attention_item - up to 16 query rows of one (sequence, head) over one split of the
 // position axis - with the two products on the 5th-generation tensor core and the scores and the
@@ -1917,6 +1919,8 @@ __device__ __forceinline__ void attention_phase(const FwdParams &p, int layer, u
         else if (p.attn_tc == 2 && p.Dh == 128) attention_item_rows<16, kRowsMax>(p, layer, item, scratch, sh);
         else if (p.attn_tc == 2 && p.M == 1) attention_item_rows<8, 1>(p, layer, item, scratch, sh);
         else if (p.attn_tc == 2) attention_item_rows<8, kRowsMax>(p, layer, item, scratch, sh);
+        else if (p.attn_tc == 3 && p.Dh == 128) attention_item_mma8<128>(p, layer, item, scratch, sh);
+        else if (p.attn_tc == 3) attention_item_mma8<64>(p, layer, item, scratch, sh);
         else attention_item(p, layer, item, scratch, sh);
     }
 }

@@ -90,6 +90,23 @@ def test_few_row_passes_on_the_fp32_attention_items(arch, lens, M):
     _forward_over_seeded_cache(arch, lens, M, 3, scale=1.5 if arch.d_model == 4096 else 6.0)
 
 
+@pytest.mark.parametrize("arch,lens,M", [
+    (synth.llama_like(2, 256, 2, 512, 512), [3000, 120], 5),      # head 128: several splits per head, ragged lengths
+    (synth.llama_like(2, 256, 2, 512, 512), [1000, 0], 8),        # a full tile of rows; an empty cache beside it
+    (synth.llama_like(2, 256, 2, 512, 512), [255, 7], 3),         # blocks that end inside the range; fewer positions than a block
+    (synth.llama_like(2, 256, 2, 512, 512), [16, 17, 15], 6),     # exactly one block / one more / one less
+    (synth.llama_like(2, 256, 4, 512, 512), [2100, 77, 0], 5),    # head 64
+    (synth.llama_like(2, 256, 4, 512, 512), [513, 64, 31], 4),
+    (synth.neox_like(3, 256, 4, 512, 520), [700, 90], 6),         # parallel residual: the out-projection waits for the attention count
+    (synth.llama_like(1, 4096, 32, 512, 512), [1151, 127, 1152, 64, 300], 5),   # 160 (sequence, head) items on 148 SMs
+])
+def test_passes_of_up_to_eight_rows_on_the_packed_mma_items(arch, lens, M):
+    """Passes of three to eight rows per sequence take the warp-MMA items that carry the hi and lo parts of the
+    queries and of the probabilities in one 16-row tile: per-warp position blocks through private copy rings, the
+    rows of the pass as one more block, merge of the eight warps and of the splits."""
+    _forward_over_seeded_cache(arch, lens, M, 4, scale=1.5 if arch.d_model == 4096 else 6.0)
+
+
 def _forward_over_seeded_cache(arch, lens, M, mode, scale=6.0):
     """Whole verification pass (single forward kernel) of a head-128 model over a seeded cache:
     logits of all rows and the appended cache rows against the oracle.  Exercises the tensor-core
