@@ -108,14 +108,15 @@ int ssd_set_prefill_mode(int mode);
 int ssd_set_persistent(int enable);
 
 /* The single forward kernel has three forms of the K-query attention over the cache (Section "KV Caching":
- * the new rows attend to the stored keys / values): items on warp-level MMAs, 64 positions per step;
- * - head dimension 128 only - items on the tcgen05 tensor core with the scores in tensor memory, 128
- * positions per step, which start more slowly but stream twice as fast; and - passes of one or two rows
- * per sequence at head dimension 64 or 128 (draft steps, decode steps) - items on the FP32 pipe with the
- * queries and the output in registers.  mode 0 (default) picks per pass (FP32 items where they apply, else
- * tensor-core items from 1024 positions per split), 1 forces the first form, 2 the second wherever it
- * applies, 3 the third where it applies and the first elsewhere.  Same results up to fp32 summation order;
- * for comparison and tests.  SSD_E_ARG for any other mode. */
+ * the new rows attend to the stored keys / values): items on warp-level MMAs over 16-row tiles, 64 positions
+ * per step; - head dimension 128 only - items on the tcgen05 tensor core with the scores in tensor memory,
+ * 128 positions per step; and - passes of at most eight rows per sequence at head dimension 64 or 128 (draft
+ * steps, decode steps, verification with K <= 7) - warp-level MMA items that carry the bf16 hi and lo parts of
+ * the queries and of the probabilities in one 16-row tile, each warp on position blocks of its own.  mode 0
+ * (default) picks per pass (the third form where it applies, else tensor-core items from 1024 positions per
+ * split, else the first), 1 forces the first form, 2 the second wherever it applies, 3 the third where it
+ * applies and the first elsewhere.  Same results up to fp32 summation order; for comparison and tests.
+ * SSD_E_ARG for any other mode. */
 int ssd_set_attention_mode(int mode);
 
 /* A layer-skip draft: the first n_layers layers of `target` plus its final norm and LM head

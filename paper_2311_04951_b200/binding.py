@@ -335,8 +335,8 @@ def set_persistent(enable: bool) -> None:
 
 
 def set_attention_mode(mode: int) -> None:
-    """0: per pass (default); 1: warp-MMA attention items; 2: tensor-core items wherever they apply;
-    3: FP32 items for passes of one or two rows, warp-MMA items otherwise."""
+    """0: per pass (default); 1: warp-MMA items over 16-row tiles; 2: tensor-core items wherever they apply;
+    3: the hi-and-lo-in-one-tile MMA items for passes of at most eight rows, the first form otherwise."""
     _check(load().ssd_set_attention_mode(int(mode)), "ssd_set_attention_mode")
 
 

@@ -116,7 +116,7 @@ struct alignas(64) FwdParams {
     // tensor-core attention (head dim 128): the whole cache as rows of Dh bf16, box 64 x 128 rows
     CUtensorMap tm_kv;
     const CUtensorMap *tm_kv_ptr;  // where the copy engine can read tm_kv (set by the kernel: see params copy)
-    int attn_tc;             // 0: attention_item (warp MMAs); 1: attention_item_tc; 2: attention_item_rows (FP32, one or two rows); 3: attention_item_mma8 (up to eight rows, hi and lo in one MMA tile)
+    int attn_tc;             // 0: attention_item (warp MMAs, 16-row tiles); 1: attention_item_tc; 2: attention_item_mma8 (up to eight rows, hi and lo in one MMA tile)
     int kv_rows_per_layer;   // B * 2 * H * S
     int attn_ctas;           // min(attention items, CTAs): set by the host together with the split plan
     int overlap_out;         // parallel-residual block and at most half of the CTAs on attention
@@ -1169,266 +1169,8 @@ __device__ __noinline__ void attention_item(const FwdParams &p, int layer, int i
     named_bar(3, kAttnThreadsP);  // scratch is free for the next item
 }
 
-// ---- attention of a few query rows on the FP32 pipe ------------------------------------------------
-// The same item as attention_item for passes of at most MR rows per sequence (draft steps, decode steps): with so
-// few rows the two products of a position are 2 MR Dh multiply-adds, which the FP32 lanes retire far faster than
-// the position's 4 Dh bytes of K and V arrive, while the MMA forms pay 16-row tiles and a chain of block-wide
-// steps per 64 positions.  Here nothing is shared inside the loop:
-//   * a warp owns every eighth block of positions; LPP = Dh / 8 lanes hold one position's K (then V) row, 16 bytes
-//     each, so one load instruction of the warp brings 32 / LPP positions, coalesced; a block is four such loads of
-//     K and four of V (4 KB), copied with cp.async into a ring of four stages private to the warp: three blocks
-//     are on their way while one is used (8 warps x 3 x 4 KB = 96 KB per SM in flight), and since a lane reads
-//     back only the 16 bytes it copied itself, waiting for its own copy groups is the only synchronisation;
-//   * q (rotary applied, pre-scaled to log2 units) and the output accumulators of the lane's eight head dims
-//     stay in registers; a score is eight multiply-adds per lane and log2(LPP) shuffles; running maximum and sum
-//     per warp in registers; K, V widen exactly, Q, the scores and P stay fp32: nothing is split or rounded;
-//   * the rows of this pass (positions >= len) are appended by warp 0 of the split that owns them, from qkv
-//     (rotary, cache rounding), after its blocks;
-//   * the eight warps' (max, sum, output) meet once, in shared memory, at the end; the result goes to the
-//     out-projection operand (one split) or to the partials the last-finishing split merges.
-__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-__device__ __forceinline__ void widen8(const uint4 &w, float (&f)[8]) {
-    f[0] = bf_lo(w.x); f[1] = bf_hi(w.x); f[2] = bf_lo(w.y); f[3] = bf_hi(w.y);
-    f[4] = bf_lo(w.z); f[5] = bf_hi(w.z); f[6] = bf_lo(w.w); f[7] = bf_hi(w.w);
-}
-constexpr int kRowsMax = 2;  // rows per sequence the FP32 items are instantiated for
-constexpr int kRowsStages = 4, kRowsStageBytes = 4096;  // per warp: blocks in flight + the one in use; a block = 4 + 4 loads of 512 bytes
-constexpr int kRowsMergeBytes = 2 * 8 * kRowsMax * 4 + 8 * kRowsMax * 128 * 4 + 256;  // the warps' (max, sum, output) at the end
-constexpr int kRowsScratchBytes = (kRowsMergeBytes + 1023) / 1024 * 1024 + 8 * kRowsStages * kRowsStageBytes;
 __device__ __forceinline__ void cp_async16_zfill(void *dst, const void *src, bool valid) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(valid ? 16 : 0) : "memory");
-}
-
-template <int LPP, int MR>
-__device__ __noinline__ void attention_item_rows(const FwdParams &p, int layer, int item, uint8_t *scratch, Shared *sh) {
-    constexpr int Dh = 8 * LPP, PPI = 32 / LPP, PB = 4 * PPI;  // head dim; positions per load; positions per block
-    static_assert(MR <= 4, "the rows of a pass are handled as one block of four positions");
-    const int split = item % p.n_split, bh = item / p.n_split, b = bh / p.H, h = bh % p.H;
-    const int d = p.d;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int sub = lane / LPP, seg = lane % LPP;
-    const int n_rows = staged_len(sh)[64 + b];
-    const int len = staged_len(sh)[b];
-    const int r0 = b * p.M;
-    const int chunk = split_chunk(p, len + n_rows, kAttnTile);
-    const int p_begin = split * chunk;
-    const int p_end = min(p_begin + chunk, len + n_rows);
-    const int c1 = min(p_end, len);                      // cached positions of this split: [p_begin, c1)
-    const int nb = c1 > p_begin ? (c1 - p_begin + PB - 1) / PB : 0;
-    const float sc = p.attn_scale * 1.4426950408889634f;  // scores in log2 units
-    __nv_bfloat16 *kc = (__nv_bfloat16 *)(p.cache + (size_t)layer * p.layer_bytes) + ((size_t)(b * 2) * p.H + h) * p.S * Dh;
-    __nv_bfloat16 *vc = kc + (size_t)p.H * p.S * Dh;
-    float *mw = reinterpret_cast<float *>(scratch);  // [8][MR] running maxima, then [8][MR] sums, then [8][MR][Dh] outputs
-    float *lw = mw + 8 * MR, *ow = lw + 8 * MR;
-
-    // per-warp stages in shared memory: [stage][K: four loads x 512 bytes][V: the same]; a lane reads back only
-    // what it copied itself, so waiting for its own copy groups is all the synchronisation there is
-    uint8_t *wbuf = scratch + (kRowsMergeBytes + 1023) / 1024 * 1024 + (size_t)warp * (kRowsStages * kRowsStageBytes) + lane * 16;
-    auto issue = [&](int i) {  // block warp + 8 i of this warp into stage i % kRowsStages
-        const int blk = warp + 8 * i;
-        uint8_t *st = wbuf + (i % kRowsStages) * kRowsStageBytes;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int pos = p_begin + blk * PB + j * PPI + sub;
-            const bool in = blk < nb && pos < c1;
-            const size_t off = in ? (size_t)pos * Dh + seg * 8 : 0;
-            cp_async16_zfill(st + j * 512, kc + off, in);
-            cp_async16_zfill(st + 2048 + j * 512, vc + off, in);
-        }
-        cp_async_commit();
-    };
-    const int my_blocks = nb > warp ? (nb - warp + 7) / 8 : 0;
-#pragma unroll
-    for (int i = 0; i < kRowsStages - 1; ++i) issue(i);
-
-    float q[MR][8], o[MR][8], m_run[MR], l_run[MR];
-#pragma unroll
-    for (int r = 0; r < MR; ++r) {
-        m_run[r] = -INFINITY;
-        l_run[r] = 0.f;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) q[r][i] = o[r][i] = 0.f;
-        if (r < n_rows) {
-            rope_vec8(p, p.qkv + (size_t)(r0 + r) * 3 * d + h * Dh, r0 + r, seg * 8, q[r]);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) q[r][i] *= sc;
-        }
-    }
-    // four positions of this lane's subgroup: scores against the MR rows, running maximum / sum, output.
-    // vis(j, r): position j of the block counts for row r.
-    auto update = [&](const uint4 (&kq)[4], const uint4 (&vq)[4], auto vis) {
-        float s[4][MR];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            float kf[8];
-            widen8(kq[j], kf);
-#pragma unroll
-            for (int r = 0; r < MR; ++r) {
-                float a = 0.f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) a = fmaf(q[r][i], kf[i], a);
-                s[j][r] = a;
-            }
-        }
-#pragma unroll
-        for (int off = 1; off < LPP; off <<= 1)
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-#pragma unroll
-                for (int r = 0; r < MR; ++r) s[j][r] += __shfl_xor_sync(0xffffffffu, s[j][r], off);
-        float f[MR];
-#pragma unroll
-        for (int r = 0; r < MR; ++r) {
-            float bm = -INFINITY;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                s[j][r] = vis(j, r) ? s[j][r] : -INFINITY;
-                bm = fmaxf(bm, s[j][r]);
-            }
-#pragma unroll
-            for (int off = LPP; off < 32; off <<= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, off));
-            const float m_new = fmaxf(m_run[r], bm);
-            f[r] = 1.f;
-            float sum = 0.f;
-            if (m_new > -INFINITY) {
-                f[r] = exp2f(m_run[r] - m_new);  // 0 on the first non-empty block
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    s[j][r] = exp2f(s[j][r] - m_new);
-                    sum += s[j][r];
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) s[j][r] = 0.f;
-            }
-            m_run[r] = m_new;
-            l_run[r] = l_run[r] * f[r] + sum;  // this subgroup's positions; the subgroups are summed at the end
-#pragma unroll
-            for (int i = 0; i < 8; ++i) o[r][i] *= f[r];
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            float vf[8];
-            widen8(vq[j], vf);
-#pragma unroll
-            for (int r = 0; r < MR; ++r)
-#pragma unroll
-                for (int i = 0; i < 8; ++i) o[r][i] = fmaf(s[j][r], vf[i], o[r][i]);
-        }
-    };
-#pragma unroll 1
-    for (int i = 0; i < my_blocks; ++i) {
-        issue(i + kRowsStages - 1);
-        cp_async_wait<kRowsStages - 1>();
-        const uint8_t *st = wbuf + (i % kRowsStages) * kRowsStageBytes;
-        uint4 kq[4], vq[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            kq[j] = *reinterpret_cast<const uint4 *>(st + j * 512);
-            vq[j] = *reinterpret_cast<const uint4 *>(st + 2048 + j * 512);
-        }
-        const int base = p_begin + (warp + 8 * i) * PB + sub;
-        update(kq, vq, [&](int j, int) { return base + j * PPI < c1; });
-    }
-    cp_async_wait<0>();
-    // ---- rows of this pass inside this split: warp 0, lanes of subgroup 0 carry them (position j = row j) ----
-    if (warp == 0 && p_end > len && p_end > p_begin) {
-        uint4 kq[4], vq[4];
-        const int first = max(p_begin, len) - len;  // first new row of this split
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            kq[j] = vq[j] = make_uint4(0, 0, 0, 0);
-            const int rn = first + j, pos = len + rn;
-            if (j < MR && rn < n_rows && pos < p_end) {
-                const int r = r0 + rn;
-                const float *krow = p.qkv + (size_t)r * 3 * d + d + h * Dh;
-                float kf[8];
-                rope_vec8(p, krow, r, seg * 8, kf);
-                const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(krow + d + seg * 8));
-                const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(krow + d + seg * 8 + 4));
-                kq[j] = make_uint4(pack_bf16x2(kf[0], kf[1]), pack_bf16x2(kf[2], kf[3]), pack_bf16x2(kf[4], kf[5]), pack_bf16x2(kf[6], kf[7]));
-                vq[j] = make_uint4(pack_bf16x2(v0.x, v0.y), pack_bf16x2(v0.z, v0.w), pack_bf16x2(v1.x, v1.y), pack_bf16x2(v1.z, v1.w));
-                if (sub == 0) {  // append: exactly one split owns this position
-                    *reinterpret_cast<uint4 *>(kc + (size_t)pos * Dh + seg * 8) = kq[j];
-                    *reinterpret_cast<uint4 *>(vc + (size_t)pos * Dh + seg * 8) = vq[j];
-                }
-            }
-        }
-        update(kq, vq, [&](int j, int r) {
-            const int rn = first + j;
-            return sub == 0 && j < MR && rn < n_rows && len + rn < p_end && rn <= r;
-        });
-    }
-    // ---- the subgroups of a warp, then the eight warps ----
-#pragma unroll
-    for (int r = 0; r < MR; ++r) {
-#pragma unroll
-        for (int off = LPP; off < 32; off <<= 1) {
-            l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], off);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) o[r][i] += __shfl_xor_sync(0xffffffffu, o[r][i], off);
-        }
-        if (lane == 0) {
-            mw[warp * MR + r] = m_run[r];
-            lw[warp * MR + r] = l_run[r];
-        }
-        if (sub == 0) {
-            float *dst = ow + ((size_t)warp * MR + r) * Dh + seg * 8;
-            *reinterpret_cast<float4 *>(dst) = make_float4(o[r][0], o[r][1], o[r][2], o[r][3]);
-            *reinterpret_cast<float4 *>(dst + 4) = make_float4(o[r][4], o[r][5], o[r][6], o[r][7]);
-        }
-    }
-    named_bar(3, kAttnThreadsP);
-    const bool direct = p.n_split == 1;
-    constexpr int q4 = Dh >> 2;
-    const int rows_here = min(MR, p.M);
-    for (int i = tid; i < rows_here * q4; i += kAttnThreadsP) {
-        const int r = i / q4, e = (i % q4) * 4;
-        float mx = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) mx = fmaxf(mx, mw[w * MR + r]);
-        float L = 0.f;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (mx > -INFINITY) {
-#pragma unroll
-            for (int w = 0; w < 8; ++w) {
-                const float mq = mw[w * MR + r];
-                if (mq > -INFINITY) {
-                    const float f = exp2f(mq - mx);
-                    const float4 a = *reinterpret_cast<const float4 *>(ow + ((size_t)w * MR + r) * Dh + e);
-                    L = fmaf(lw[w * MR + r], f, L);
-                    acc.x = fmaf(a.x, f, acc.x); acc.y = fmaf(a.y, f, acc.y); acc.z = fmaf(a.z, f, acc.z); acc.w = fmaf(a.w, f, acc.w);
-                }
-            }
-        }
-        const bool live = r < n_rows && L > 0.f;
-        if (!live) acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (direct) {
-            const float inv = live ? 1.f / L : 0.f;
-            store_ao4(p, r0 + r, h * Dh + e, make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
-        } else {
-            const size_t slot = ((size_t)(r0 + r) * p.H + h) * p.n_split + split;
-            if (e == 0) {
-                p.part_m[slot] = live ? mx : -INFINITY;
-                p.part_l[slot] = live ? L : 0.f;
-            }
-            *reinterpret_cast<float4 *>(p.part_o + slot * Dh + e) = acc;
-        }
-    }
-    if (!direct) {
-        // ticket: the item that finishes last for this (sequence, head) merges all partials
-        __threadfence();
-        named_bar(3, kAttnThreadsP);
-        if (tid == 0) sh->flag = (atomicAdd(p.tickets + bh, 1u) == (unsigned)(p.n_split - 1));
-        named_bar(3, kAttnThreadsP);
-        if (sh->flag) {
-            __threadfence();
-            merge_splits(p, r0, h, Dh);
-            if (tid == 0) p.tickets[bh] = 0;  // ready for the next layer (a grid barrier lies between)
-        }
-    }
-    named_bar(3, kAttnThreadsP);  // scratch is free for the next item
 }
 
 #include "attn_mma8.cuh"
@@ -1915,12 +1657,8 @@ __device__ __forceinline__ void attention_phase(const FwdParams &p, int layer, u
     const int items = p.B * p.H * p.n_split * MT;
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
         if (p.attn_tc == 1) attention_item_tc(p, layer, item, scratch, sh);
-        else if (p.attn_tc == 2 && p.Dh == 128 && p.M == 1) attention_item_rows<16, 1>(p, layer, item, scratch, sh);
-        else if (p.attn_tc == 2 && p.Dh == 128) attention_item_rows<16, kRowsMax>(p, layer, item, scratch, sh);
-        else if (p.attn_tc == 2 && p.M == 1) attention_item_rows<8, 1>(p, layer, item, scratch, sh);
-        else if (p.attn_tc == 2) attention_item_rows<8, kRowsMax>(p, layer, item, scratch, sh);
-        else if (p.attn_tc == 3 && p.Dh == 128) attention_item_mma8<128>(p, layer, item, scratch, sh);
-        else if (p.attn_tc == 3) attention_item_mma8<64>(p, layer, item, scratch, sh);
+        else if (p.attn_tc == 2 && p.Dh == 128) attention_item_mma8<128>(p, layer, item, scratch, sh);
+        else if (p.attn_tc == 2) attention_item_mma8<64>(p, layer, item, scratch, sh);
         else attention_item(p, layer, item, scratch, sh);
     }
 }

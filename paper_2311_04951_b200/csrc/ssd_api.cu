@@ -510,8 +510,7 @@ int launch_forward_nt(FwdParams p, const void *ws_base, size_t ws_bytes, cudaStr
     constexpr size_t stage = kWTileBytesP + 2 * NT * 8 * kTileK * 2;
     size_t attn = align_up(attn_scratch_bytes(p.Dh), 128);
     if (p.attn_tc == 1 && attn < (size_t)kTcScratchBytes) attn = kTcScratchBytes;
-    if (p.attn_tc == 2) attn = kRowsScratchBytes;
-    if (p.attn_tc == 3) attn = m8_scratch_bytes(p.Dh);
+    if (p.attn_tc == 2) attn = m8_scratch_bytes(p.Dh);
     const size_t tail = 24 * 32 + 64 + 16 + sizeof(Shared) + 16 * sizeof(double) + kEpiBytes + 256;  // barriers, small state, epilogue tile
     const size_t total = (size_t)kSmemBudget - 1024 - tail;
     // upper slots share their bytes with the attention scratch; two slots never do where they fit
@@ -618,16 +617,13 @@ int forward_persistent(ssd_model *m, ssd_kv *kv, const int32_t *tokens, int tok_
     const int groups = kv->B * a.n_heads * ((M + 15) / 16);
     p.attn_tc = 0;
     p.kv_rows_per_layer = kv->B * 2 * a.n_heads * kv->S;
-    // Passes of one or two rows per sequence (draft steps, decode steps): items on the FP32 pipe.
-    const bool rows_form = M <= kRowsMax && (a.head_dim == 64 || a.head_dim == 128) && (g_attn_mode == 0 || g_attn_mode == 3);
-    const bool packed_form = M <= kM8Rows && (a.head_dim == 64 || a.head_dim == 128) && (g_attn_mode == 0 || g_attn_mode == 4);
-    if (rows_form) {
+    // Passes of at most eight rows per sequence (draft steps, decode steps, verification with K <= 7): the warp-MMA
+    // items that carry hi and lo in one tile.
+    const bool packed_form = M <= kM8Rows && (a.head_dim == 64 || a.head_dim == 128) && (g_attn_mode == 0 || g_attn_mode == 3);
+    if (packed_form) {
         plan_split(groups, ctx, &p.chunk, &p.n_split, kAttnTile);
         p.attn_tc = 2;
-    } else if (packed_form) {
-        plan_split(groups, ctx, &p.chunk, &p.n_split, kAttnTile);
-        p.attn_tc = 3;
-    } else if (a.head_dim == 128 && kv->tm_rows_ok && g_attn_mode != 1 && g_attn_mode != 3 && g_attn_mode != 4) {
+    } else if (a.head_dim == 128 && kv->tm_rows_ok && g_attn_mode != 1 && g_attn_mode != 3) {
         plan_split(groups, ctx, &p.chunk, &p.n_split, kTcChunk);
         if (p.chunk >= 1024 || g_attn_mode == 2) {
             p.attn_tc = 1;
@@ -996,7 +992,7 @@ int ssd_model_create(const ssd_arch *arch, const void *const *dev_weights, int n
 }
 
 int ssd_set_attention_mode(int mode) {
-    if (mode < 0 || mode > 4) return SSD_E_ARG;
+    if (mode < 0 || mode > 3) return SSD_E_ARG;
     g_attn_mode = mode;
     return SSD_OK;
 }

@@ -83,10 +83,9 @@ def test_parallel_residual_out_projection_behind_the_attention_count(lens, M, mo
     (synth.neox_like(3, 256, 4, 512, 520), [700, 90], 2),         # parallel residual: the out-projection waits for the attention count
     (synth.llama_like(1, 4096, 32, 512, 512), [1151, 127, 1152, 64, 300], 2),   # 160 (sequence, head) items on 148 SMs
 ])
-def test_few_row_passes_on_the_fp32_attention_items(arch, lens, M):
-    """Passes of one or two rows per sequence (draft steps, decode steps) take the FP32 attention items: per-warp
-    position blocks, copy ring private to the warp, the rows of the pass appended by the owning split, merge of the
-    eight warps and of the splits."""
+def test_one_and_two_row_passes_on_the_packed_mma_items(arch, lens, M):
+    """Passes of one or two rows per sequence (draft steps, decode steps) on the warp-MMA items that carry hi and lo in
+    one tile: blocks that end inside the range, empty caches, head 64 and head 128, splits and their merge."""
     _forward_over_seeded_cache(arch, lens, M, 3, scale=1.5 if arch.d_model == 4096 else 6.0)
 
 
@@ -104,7 +103,7 @@ def test_passes_of_up_to_eight_rows_on_the_packed_mma_items(arch, lens, M):
     """Passes of three to eight rows per sequence take the warp-MMA items that carry the hi and lo parts of the
     queries and of the probabilities in one 16-row tile: per-warp position blocks through private copy rings, the
     rows of the pass as one more block, merge of the eight warps and of the splits."""
-    _forward_over_seeded_cache(arch, lens, M, 4, scale=1.5 if arch.d_model == 4096 else 6.0)
+    _forward_over_seeded_cache(arch, lens, M, 3, scale=1.5 if arch.d_model == 4096 else 6.0)
 
 
 def _forward_over_seeded_cache(arch, lens, M, mode, scale=6.0):
