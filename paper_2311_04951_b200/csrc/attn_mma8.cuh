@@ -21,15 +21,18 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t &r0, u
 }
 constexpr int kM8Rows = 8, kM8Block = 16;             // query rows per item; positions per block
 constexpr int kM8Slack = 8;
-__host__ __device__ constexpr int m8_stage_bytes(int Dh) { return 2 * kM8Block * Dh * 2; }   // K rows, then V rows
+// bytes of a tile row in shared memory: the head's bf16 row padded to a power of two, so that the 16-byte pieces can be swizzled
+__host__ __device__ constexpr int m8_row_bytes(int Dh) { return Dh <= 32 ? 64 : Dh <= 64 ? 128 : 256; }
+__host__ __device__ constexpr int m8_stage_bytes(int Dh) { return 2 * kM8Block * m8_row_bytes(Dh); }   // K rows, then V rows
 __host__ __device__ constexpr int m8_scratch_bytes(int Dh) {
     // two stages per warp (the warps' (max, sum, output) lie over them at the end), then the staged queries
-    return 8 * 2 * m8_stage_bytes(Dh) + 16 * Dh * 2;
+    return 8 * 2 * m8_stage_bytes(Dh) + 16 * m8_row_bytes(Dh);
 }
 
 template <int DH>
 __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, int item, uint8_t *scratch, Shared *sh) {
-    constexpr int NK = DH / 16, ND = DH / 8, ROWB = DH * 2, GPR = DH / 8;  // k-steps; 8-column tiles; bytes and 16-byte pieces per row
+    constexpr int NK = DH / 16, ND = DH / 8, ROWB = m8_row_bytes(DH), GPR = DH / 8;  // k-steps; 8-column tiles; bytes of a tile row; 16-byte pieces of a head row
+    static_assert(DH % 16 == 0 && DH <= 128 && ND % 2 == 0, "head dims that are multiples of 16");
     constexpr int STAGE = m8_stage_bytes(DH);
     const int split = item % p.n_split, bh = item / p.n_split, b = bh / p.H, h = bh % p.H;
     const int d = p.d;
@@ -51,8 +54,9 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
         const int blk = warp + 8 * i;
         uint8_t *st = wst + (i & 1) * STAGE;
 #pragma unroll 1
-        for (int it = 0; it < kM8Block * GPR / 32; ++it) {
+        for (int it = 0; it < (kM8Block * GPR + 31) / 32; ++it) {
             const int idx = it * 32 + lane, r = idx / GPR, c = idx % GPR;
+            if (kM8Block * GPR % 32 != 0 && idx >= kM8Block * GPR) break;
             const int pos = p_begin + blk * kM8Block + r;
             const bool in = blk < nb && pos < c1;
             const size_t off = in ? (size_t)pos * DH + c * 8 : 0;
@@ -170,7 +174,7 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
         const int first = max(p_begin, len) - len;                // first new row of this split
         const int cnt = min(p_end - len, n_rows) - first;         // new rows here (at most 8)
         uint8_t *st = wst;
-        for (int i = lane; i < 2 * kM8Block * GPR; i += 32) reinterpret_cast<uint4 *>(st)[i] = make_uint4(0, 0, 0, 0);
+        for (int i = lane; i < STAGE / 16; i += 32) reinterpret_cast<uint4 *>(st)[i] = make_uint4(0, 0, 0, 0);
         __syncwarp();
         for (int i = lane; i < cnt * GPR; i += 32) {
             const int j = i / GPR, c = i % GPR, rn = first + j, pos = len + rn, r = r0 + rn;
