@@ -50,19 +50,24 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
     __nv_bfloat16 *vc = kc + (size_t)p.H * p.S * DH;
     uint8_t *wst = scratch + (size_t)warp * (2 * STAGE);   // this warp's two stages
     // piece c of row r of a tile sits at r * ROWB + ((c ^ (r & 7)) << 4)
+    // a lane copies 16-byte piece lc of rows lr, lr + RPI, ... of a block's K and V tiles
+    static_assert((GPR & (GPR - 1)) == 0, "pieces per row: a power of two");
+    constexpr int RPI = 32 / GPR;
+    const int lr = lane / GPR, lc = lane % GPR;
+    const uint32_t wst_u = smem_u32(wst) + (uint32_t)(lr * ROWB);
     auto issue = [&](int i) {  // block warp + 8 i of this warp into stage i & 1
-        const int blk = warp + 8 * i;
-        uint8_t *st = wst + (i & 1) * STAGE;
-#pragma unroll 1
-        for (int it = 0; it < (kM8Block * GPR + 31) / 32; ++it) {
-            const int idx = it * 32 + lane, r = idx / GPR, c = idx % GPR;
-            if (kM8Block * GPR % 32 != 0 && idx >= kM8Block * GPR) break;
-            const int pos = p_begin + blk * kM8Block + r;
-            const bool in = blk < nb && pos < c1;
-            const size_t off = in ? (size_t)pos * DH + c * 8 : 0;
-            const uint32_t so = (uint32_t)(r * ROWB + ((c ^ (r & 7)) << 4));
-            cp_async16_zfill(st + so, kc + off, in);
-            cp_async16_zfill(st + kM8Block * ROWB + so, vc + off, in);
+        const int blk = warp + 8 * i, pos0 = p_begin + blk * kM8Block + lr;
+        const uint32_t st = wst_u + (uint32_t)((i & 1) * STAGE);
+        const size_t off0 = (size_t)pos0 * DH + lc * 8;
+#pragma unroll 4
+        for (int it = 0; it < kM8Block / RPI; ++it) {
+            const int r = it * RPI + lr;
+            const bool in = blk < nb && pos0 + it * RPI < c1;
+            const size_t off = in ? off0 + (size_t)it * RPI * DH : 0;
+            const uint32_t so = st + (uint32_t)(it * RPI * ROWB + ((lc ^ (r & 7)) << 4));
+            const uint32_t nbytes = in ? 16u : 0u;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(so), "l"(kc + off), "r"(nbytes) : "memory");
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(so + kM8Block * ROWB), "l"(vc + off), "r"(nbytes) : "memory");
         }
         cp_async_commit();
     };
