@@ -163,22 +163,12 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
             }
         }
     };
-#pragma unroll 1
-    for (int i = 0; i < my_blocks; ++i) {
-        __syncwarp();            // every lane is done reading the stage block i - 1 used
-        issue(i + 1);
-        cp_async_wait<1>();      // this thread's copies of block i have landed ...
-        __syncwarp();            // ... and every other lane's
-        const int base = p_begin + (warp + 8 * i) * kM8Block;
-        update(wst + (i & 1) * STAGE, [&](int j) { return base + j < c1; });
-    }
-    cp_async_wait<0>();
-    __syncwarp();
-    // ---- rows of this pass inside this split: one more block of warp 0, built in its first stage ----
+    // ---- rows of this pass inside this split: a block of warp 0, built in its second stage while the copies of its
+    //      first block are on their way (the order of the blocks does not matter to the running maximum / sum) ----
     if (warp == 0 && p_end > len && p_end > p_begin) {
         const int first = max(p_begin, len) - len;                // first new row of this split
         const int cnt = min(p_end - len, n_rows) - first;         // new rows here (at most 8)
-        uint8_t *st = wst;
+        uint8_t *st = wst + STAGE;
         for (int i = lane; i < STAGE / 16; i += 32) reinterpret_cast<uint4 *>(st)[i] = make_uint4(0, 0, 0, 0);
         __syncwarp();
         for (int i = lane; i < cnt * GPR; i += 32) {
@@ -199,6 +189,17 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
         __syncwarp();
         update(st, [&](int j) { return j < cnt && first + j <= g; });
     }
+#pragma unroll 1
+    for (int i = 0; i < my_blocks; ++i) {
+        __syncwarp();            // every lane is done reading the stage block i - 1 used
+        issue(i + 1);
+        cp_async_wait<1>();      // this thread's copies of block i have landed ...
+        __syncwarp();            // ... and every other lane's
+        const int base = p_begin + (warp + 8 * i) * kM8Block;
+        update(wst + (i & 1) * STAGE, [&](int j) { return base + j < c1; });
+    }
+    cp_async_wait<0>();
+    __syncwarp();
     // ---- the four threads of a row, then the eight warps (their partial results lie over the stages) ----
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
