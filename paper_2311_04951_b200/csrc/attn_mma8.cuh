@@ -24,16 +24,18 @@ constexpr int kM8Slack = 8;
 // bytes of a tile row in shared memory: the head's bf16 row padded to a power of two, so that the 16-byte pieces can be swizzled
 __host__ __device__ constexpr int m8_row_bytes(int Dh) { return Dh <= 32 ? 64 : Dh <= 64 ? 128 : 256; }
 __host__ __device__ constexpr int m8_stage_bytes(int Dh) { return 2 * kM8Block * m8_row_bytes(Dh); }   // K rows, then V rows
+// stages of a warp's ring: two 8 KB stages at head 128; narrower heads take more of them for the same bytes on their way
+__host__ __device__ constexpr int m8_stages(int Dh) { return Dh <= 64 ? 4 : 2; }
 __host__ __device__ constexpr int m8_scratch_bytes(int Dh) {
     // two stages per warp (the warps' (max, sum, output) lie over them at the end), then the staged queries
-    return 8 * 2 * m8_stage_bytes(Dh) + 16 * m8_row_bytes(Dh);
+    return 8 * m8_stages(Dh) * m8_stage_bytes(Dh) + 16 * m8_row_bytes(Dh);
 }
 
 template <int DH>
 __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, int item, uint8_t *scratch, Shared *sh) {
     constexpr int NK = DH / 16, ND = DH / 8, ROWB = m8_row_bytes(DH), GPR = DH / 8;  // k-steps; 8-column tiles; bytes of a tile row; 16-byte pieces of a head row
     static_assert(DH % 16 == 0 && DH <= 128 && ND % 2 == 0, "head dims that are multiples of 16");
-    constexpr int STAGE = m8_stage_bytes(DH);
+    constexpr int STAGE = m8_stage_bytes(DH), NS = m8_stages(DH);
     const int split = item % p.n_split, bh = item / p.n_split, b = bh / p.H, h = bh % p.H;
     const int d = p.d;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
@@ -48,16 +50,16 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
     const float sc = p.attn_scale * 1.4426950408889634f;  // scores in log2 units
     __nv_bfloat16 *kc = (__nv_bfloat16 *)(p.cache + (size_t)layer * p.layer_bytes) + ((size_t)(b * 2) * p.H + h) * p.S * DH;
     __nv_bfloat16 *vc = kc + (size_t)p.H * p.S * DH;
-    uint8_t *wst = scratch + (size_t)warp * (2 * STAGE);   // this warp's two stages
+    uint8_t *wst = scratch + (size_t)warp * (NS * STAGE);   // this warp's stages
     // piece c of row r of a tile sits at r * ROWB + ((c ^ (r & 7)) << 4)
     // a lane copies 16-byte piece lc of rows lr, lr + RPI, ... of a block's K and V tiles
     static_assert((GPR & (GPR - 1)) == 0, "pieces per row: a power of two");
     constexpr int RPI = 32 / GPR;
     const int lr = lane / GPR, lc = lane % GPR;
     const uint32_t wst_u = smem_u32(wst) + (uint32_t)(lr * ROWB);
-    auto issue = [&](int i) {  // block warp + 8 i of this warp into stage i & 1
+    auto issue = [&](int i) {  // block warp + 8 i of this warp into stage i % NS
         const int blk = warp + 8 * i, pos0 = p_begin + blk * kM8Block + lr;
-        const uint32_t st = wst_u + (uint32_t)((i & 1) * STAGE);
+        const uint32_t st = wst_u + (uint32_t)((i % NS) * STAGE);
         const size_t off0 = (size_t)pos0 * DH + lc * 8;
 #pragma unroll 4
         for (int it = 0; it < kM8Block / RPI; ++it) {
@@ -72,11 +74,12 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
         cp_async_commit();
     };
     const int my_blocks = nb > warp ? (nb - warp + 7) / 8 : 0;
-    issue(0);
+#pragma unroll
+    for (int i = 0; i < NS - 1; ++i) issue(i);
 
     // ---- the queries (rotary applied, in log2 units), staged once behind the stages as the MMA's A tile: row r
     //      as bf16 hi in tile row r, lo in tile row r + 8, pieces swizzled like the K / V tiles ----
-    uint8_t *q_t = scratch + 8 * 2 * STAGE;  // [16][DH] bf16
+    uint8_t *q_t = scratch + 8 * NS * STAGE;  // [16][DH] bf16
     for (int i = tid; i < kM8Rows * GPR; i += kAttnThreadsP) {
         const int r = i / GPR, c = i % GPR;
         float q[8];
@@ -163,12 +166,12 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
             }
         }
     };
-    // ---- rows of this pass inside this split: a block of warp 0, built in its second stage while the copies of its
+    // ---- rows of this pass inside this split: a block of warp 0, built in its last stage while the copies of its
     //      first block are on their way (the order of the blocks does not matter to the running maximum / sum) ----
     if (warp == 0 && p_end > len && p_end > p_begin) {
         const int first = max(p_begin, len) - len;                // first new row of this split
         const int cnt = min(p_end - len, n_rows) - first;         // new rows here (at most 8)
-        uint8_t *st = wst + STAGE;
+        uint8_t *st = wst + (NS - 1) * STAGE;
         for (int i = lane; i < STAGE / 16; i += 32) reinterpret_cast<uint4 *>(st)[i] = make_uint4(0, 0, 0, 0);
         __syncwarp();
         for (int i = lane; i < cnt * GPR; i += 32) {
@@ -192,11 +195,11 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
 #pragma unroll 1
     for (int i = 0; i < my_blocks; ++i) {
         __syncwarp();            // every lane is done reading the stage block i - 1 used
-        issue(i + 1);
-        cp_async_wait<1>();      // this thread's copies of block i have landed ...
+        issue(i + NS - 1);
+        cp_async_wait<NS - 1>();   // this thread's copies of block i have landed ...
         __syncwarp();            // ... and every other lane's
         const int base = p_begin + (warp + 8 * i) * kM8Block;
-        update(wst + (i & 1) * STAGE, [&](int j) { return base + j < c1; });
+        update(wst + (i % NS) * STAGE, [&](int j) { return base + j < c1; });
     }
     cp_async_wait<0>();
     __syncwarp();
