@@ -28,7 +28,8 @@ __host__ __device__ constexpr int m8_stage_bytes(int Dh) { return 2 * kM8Block *
 __host__ __device__ constexpr int m8_stages(int Dh) { return Dh <= 64 ? 4 : 2; }
 __host__ __device__ constexpr int m8_scratch_bytes(int Dh) {
     // two stages per warp (the warps' (max, sum, output) lie over them at the end), then the staged queries
-    return 8 * m8_stages(Dh) * m8_stage_bytes(Dh) + 16 * m8_row_bytes(Dh);
+    // ... then the staged queries (one tile) and the block of the pass's own rows (a K tile and a V tile)
+    return 8 * m8_stages(Dh) * m8_stage_bytes(Dh) + 16 * m8_row_bytes(Dh) + m8_stage_bytes(Dh);
 }
 
 template <int DH>
@@ -98,6 +99,34 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
         *reinterpret_cast<uint4 *>(q_t + r * ROWB + so) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
         *reinterpret_cast<uint4 *>(q_t + (r + 8) * ROWB + so) = make_uint4(lw4[0], lw4[1], lw4[2], lw4[3]);
     }
+    // ---- the rows of this pass inside this split, as one more block (a K tile, a V tile) behind the query tile:
+    //      every thread builds one or two 16-byte pieces (rotary, cache rounding); the split that owns the rows
+    //      appends them to the cache ----
+    uint8_t *n_t = q_t + 16 * ROWB;
+    const bool has_new = p_end > len && p_end > p_begin;
+    const int first = max(p_begin, len) - len;                              // first new row of this split
+    const int cnt = has_new ? min(p_end - len, n_rows) - first : 0;         // new rows here (at most 8)
+    if (has_new) {
+        for (int i = tid; i < 2 * kM8Block * GPR; i += kAttnThreadsP) {
+            const int kv = i / (kM8Block * GPR), j = (i / GPR) % kM8Block, c = i % GPR;
+            uint4 w = make_uint4(0, 0, 0, 0);
+            if (j < cnt) {
+                const int rn = first + j, r = r0 + rn;
+                const float *krow = p.qkv + (size_t)r * 3 * d + d + h * DH;
+                float x[8];
+                if (kv == 0) {
+                    rope_vec8(p, krow, r, c * 8, x);
+                } else {
+                    const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(krow + d + c * 8));
+                    const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(krow + d + c * 8 + 4));
+                    x[0] = v0.x; x[1] = v0.y; x[2] = v0.z; x[3] = v0.w; x[4] = v1.x; x[5] = v1.y; x[6] = v1.z; x[7] = v1.w;
+                }
+                w = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]), pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7]));
+                *reinterpret_cast<uint4 *>((kv ? vc : kc) + (size_t)(len + rn) * DH + c * 8) = w;  // append: exactly one split owns this position
+            }
+            *reinterpret_cast<uint4 *>(n_t + kv * (kM8Block * ROWB) + j * ROWB + ((c ^ (j & 7)) << 4)) = w;
+        }
+    }
     named_bar(3, kAttnThreadsP);
     // ldmatrix x4 of the A tile: (rows 0-7, k lo), (rows 8-15, k lo), (rows 0-7, k hi), (rows 8-15, k hi)
     const uint32_t qaddr = smem_u32(q_t) + (uint32_t)((lane & 15) * ROWB);
@@ -166,32 +195,9 @@ __device__ __noinline__ void attention_item_mma8(const FwdParams &p, int layer, 
             }
         }
     };
-    // ---- rows of this pass inside this split: a block of warp 0, built in its last stage while the copies of its
-    //      first block are on their way (the order of the blocks does not matter to the running maximum / sum) ----
-    if (warp == 0 && p_end > len && p_end > p_begin) {
-        const int first = max(p_begin, len) - len;                // first new row of this split
-        const int cnt = min(p_end - len, n_rows) - first;         // new rows here (at most 8)
-        uint8_t *st = wst + (NS - 1) * STAGE;
-        for (int i = lane; i < STAGE / 16; i += 32) reinterpret_cast<uint4 *>(st)[i] = make_uint4(0, 0, 0, 0);
-        __syncwarp();
-        for (int i = lane; i < cnt * GPR; i += 32) {
-            const int j = i / GPR, c = i % GPR, rn = first + j, pos = len + rn, r = r0 + rn;
-            const float *krow = p.qkv + (size_t)r * 3 * d + d + h * DH;
-            float kf[8];
-            rope_vec8(p, krow, r, c * 8, kf);
-            const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(krow + d + c * 8));
-            const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(krow + d + c * 8 + 4));
-            const uint4 kq = make_uint4(pack_bf16x2(kf[0], kf[1]), pack_bf16x2(kf[2], kf[3]), pack_bf16x2(kf[4], kf[5]), pack_bf16x2(kf[6], kf[7]));
-            const uint4 vq = make_uint4(pack_bf16x2(v0.x, v0.y), pack_bf16x2(v0.z, v0.w), pack_bf16x2(v1.x, v1.y), pack_bf16x2(v1.z, v1.w));
-            const uint32_t so = (uint32_t)(j * ROWB + ((c ^ (j & 7)) << 4));
-            *reinterpret_cast<uint4 *>(st + so) = kq;
-            *reinterpret_cast<uint4 *>(st + kM8Block * ROWB + so) = vq;
-            *reinterpret_cast<uint4 *>(kc + (size_t)pos * DH + c * 8) = kq;  // append: exactly one split owns this position
-            *reinterpret_cast<uint4 *>(vc + (size_t)pos * DH + c * 8) = vq;
-        }
-        __syncwarp();
-        update(st, [&](int j) { return j < cnt && first + j <= g; });
-    }
+    // the block of the pass's own rows: warp 0, first (the order of the blocks does not matter to the running
+    // maximum / sum), while the copies of its first cached blocks are on their way
+    if (warp == 0 && has_new) update(n_t, [&](int j) { return j < cnt && first + j <= g; });
 #pragma unroll 1
     for (int i = 0; i < my_blocks; ++i) {
         __syncwarp();            // every lane is done reading the stage block i - 1 used
