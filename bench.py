@@ -42,10 +42,10 @@ NOMINAL_HBM_GBS = 8000.0
 # An entry is dropped (None) when the kernel has changed since its capture.
 NCU_TRAFFIC = {
     # workload: (captured workload, dram bytes of the captured launch, layers captured)
-    "llama-7b-b8": ("llama-7b-l4-b8", 3.1179e9, 4),        # profiles/forward_kernel_llama-7b-l4-b8_verify.md
-    "llama-7b-l4-b8": ("llama-7b-l4-b8", 3.1179e9, 4),
-    "llama-7b-l4-ctx8k": ("llama-7b-l4-ctx8k", 2.4820e9, 4),  # profiles/forward_kernel_llama-7b-l4-ctx8k_verify.md
-    "neox-1.4b": ("neox-1.4b", 2.6793e9, 24),               # profiles/forward_kernel_neox-1.4b_verify.md
+    "llama-7b-b8": ("llama-7b-l4-b8", 3.1158e9, 4),        # profiles/forward_kernel_llama-7b-l4-b8_verify.md
+    "llama-7b-l4-b8": ("llama-7b-l4-b8", 3.1158e9, 4),
+    "llama-7b-l4-ctx8k": ("llama-7b-l4-ctx8k", 2.4807e9, 4),  # profiles/forward_kernel_llama-7b-l4-ctx8k_verify.md
+    "neox-1.4b": ("neox-1.4b", 2.6746e9, 24),               # profiles/forward_kernel_neox-1.4b_verify.md
 }
 
 # bench workloads: name -> preset (+ overrides)
