@@ -211,10 +211,11 @@ def test_7b_shape_many_row_prompt_pass_matches_the_oracle(llama7b):
 
 @pytest.mark.parametrize("ctx,M", [(8192, 5), (8192, 17), (16384, 5), (16384, 17)])
 def test_7b_width_long_context_tensor_core_attention_matches_the_oracle(llama7b, ctx, M):
-    """The long-context points of the verify sweep through target_verify with the default attention choice,
-    which at these lengths is the tcgen05 form (2048 to 8192 positions per split, the K/V ring wrapping many
-    times, 2 to 4 splits merged; 17 rows = two 16-row tiles): first four layers of the 7B model at full width
-    + final norm + LM head, against the oracle on the seeded cache."""
+    """The long-context points of the verify sweep through target_verify with the default attention choice: at 5
+    rows the warp-MMA items that carry hi and lo in one tile (hundreds of position blocks per warp), at 17 rows the
+    tcgen05 form (2048 to 8192 positions per split, the K/V ring wrapping many times, two 16-row tiles); 2 to 4
+    splits merged; first four layers of the 7B model at full width + final norm + LM head, against the oracle on
+    the seeded cache."""
     arch4 = llama7b["arch"].replace(n_layers=4)
     model4 = llama7b["model"].share_prefix(4)
     od.set_threads(16)
